@@ -1,0 +1,6 @@
+"""CPU oracle for one Sketched-SGD compression step -- TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
+It shares no code with the CUDA library and never imports it.
+"""
+from .ssgd_oracle import Oracle, build, derive_params, select  # noqa: F401

@@ -1,0 +1,306 @@
+// ssgd_oracle.cpp -- plain CPU statement of one Sketched-SGD compression step.
+//
+// TEST INFRASTRUCTURE ONLY (see ssgd_oracle.h).  Single-threaded, no blocking, no fusion, no
+// reordering beyond what Algorithm 3 and Algorithm 4 of the paper state.  Compile with
+// -ffp-contract=off so that the only fused multiply-add is the explicit one in the momentum line.
+#include "ssgd_oracle.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace {
+
+constexpr uint64_t P31 = 2147483647ULL;  // p = 2^31 - 1
+
+struct Ctx {
+    int64_t d, c, k;
+    int32_t r, W;
+    uint32_t a[SSGD_ORACLE_MAX_R], b[SSGD_ORACLE_MAX_R];    // bucket hash h_j
+    uint32_t a2[SSGD_ORACLE_MAX_R], b2[SSGD_ORACLE_MAX_R];  // sign hash s_j
+};
+
+inline const Ctx* C(const ssgd_oracle_ctx* p) { return reinterpret_cast<const Ctx*>(p); }
+inline Ctx* C(ssgd_oracle_ctx* p) { return reinterpret_cast<Ctx*>(p); }
+
+// Bucket hash of row j: h_j(i) = ((a_j * i + b_j) mod p) mod c.
+inline int64_t bucket(const Ctx* x, int j, uint64_t i) {
+    return (int64_t)((((uint64_t)x->a[j] * i + (uint64_t)x->b[j]) % P31) % (uint64_t)x->c);
+}
+// Sign hash of row j: s_j(i) = 2 * (((a'_j * i + b'_j) mod p) & 1) - 1, i.e. low bit 1 -> +1.
+inline int sign(const Ctx* x, int j, uint64_t i) {
+    return 2 * (int)((((uint64_t)x->a2[j] * i + (uint64_t)x->b2[j]) % P31) & 1ULL) - 1;
+}
+
+inline uint32_t abs_bits(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    return u & 0x7FFFFFFFu;
+}
+
+template <typename TX>
+int sketch_any(const Ctx* x, const TX* vec, double* T, double* M) {
+    if (!x || !vec || !T) return -1;
+    // Algorithm 4, update(i, f_i) for each coordinate in turn.
+    for (int64_t i = 0; i < x->d; ++i) {
+        const double f = (double)vec[i];
+        for (int j = 0; j < x->r; ++j) {
+            const int64_t col = bucket(x, j, (uint64_t)i);
+            T[(int64_t)j * x->c + col] += (double)sign(x, j, (uint64_t)i) * f;
+            if (M) M[(int64_t)j * x->c + col] += std::fabs(f);
+        }
+    }
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ssgd_oracle_derive_params(uint64_t seed, int32_t r, uint32_t* out4r) {
+    if (!out4r || r < 1 || r > SSGD_ORACLE_MAX_R) return -1;
+    uint64_t s = seed;
+    auto next = [&s]() -> uint64_t {
+        s += 0x9E3779B97F4A7C15ULL;
+        uint64_t z = s;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+        return z ^ (z >> 31);
+    };
+    for (int j = 0; j < r; ++j) {
+        out4r[4 * j + 0] = (uint32_t)(1 + next() % (P31 - 1));
+        out4r[4 * j + 1] = (uint32_t)(next() % P31);
+        out4r[4 * j + 2] = (uint32_t)(1 + next() % (P31 - 1));
+        out4r[4 * j + 3] = (uint32_t)(next() % P31);
+    }
+    return 0;
+}
+
+int ssgd_oracle_create(ssgd_oracle_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k,
+                       int32_t W, uint64_t seed) {
+    if (!out) return -1;
+    *out = nullptr;
+    if (d < 1 || d >= (int64_t)P31) return -1;
+    if (r < 1 || r > SSGD_ORACLE_MAX_R || (r % 2) == 0) return -1;
+    if (c < 1 || c >= (int64_t)P31) return -1;
+    if (k < 1 || k > d || W < 1) return -1;
+    Ctx* x = new (std::nothrow) Ctx();
+    if (!x) return -2;
+    x->d = d; x->r = r; x->c = c; x->k = k; x->W = W;
+    uint32_t p4[4 * SSGD_ORACLE_MAX_R];
+    ssgd_oracle_derive_params(seed, r, p4);
+    for (int j = 0; j < r; ++j) {
+        x->a[j] = p4[4 * j]; x->b[j] = p4[4 * j + 1];
+        x->a2[j] = p4[4 * j + 2]; x->b2[j] = p4[4 * j + 3];
+    }
+    *out = reinterpret_cast<ssgd_oracle_ctx*>(x);
+    return 0;
+}
+
+void ssgd_oracle_destroy(ssgd_oracle_ctx* ctx) { delete C(ctx); }
+
+int ssgd_oracle_get_params(const ssgd_oracle_ctx* ctx, uint32_t* out4r) {
+    const Ctx* x = C(ctx);
+    if (!x || !out4r) return -1;
+    for (int j = 0; j < x->r; ++j) {
+        out4r[4 * j] = x->a[j]; out4r[4 * j + 1] = x->b[j];
+        out4r[4 * j + 2] = x->a2[j]; out4r[4 * j + 3] = x->b2[j];
+    }
+    return 0;
+}
+
+int ssgd_oracle_set_params(ssgd_oracle_ctx* ctx, const uint32_t* in4r) {
+    Ctx* x = C(ctx);
+    if (!x || !in4r) return -1;
+    for (int j = 0; j < x->r; ++j) {
+        if (in4r[4 * j] < 1 || in4r[4 * j] >= P31 || in4r[4 * j + 1] >= P31) return -1;
+        if (in4r[4 * j + 2] < 1 || in4r[4 * j + 2] >= P31 || in4r[4 * j + 3] >= P31) return -1;
+    }
+    for (int j = 0; j < x->r; ++j) {
+        x->a[j] = in4r[4 * j]; x->b[j] = in4r[4 * j + 1];
+        x->a2[j] = in4r[4 * j + 2]; x->b2[j] = in4r[4 * j + 3];
+    }
+    return 0;
+}
+
+int ssgd_oracle_hashes(const ssgd_oracle_ctx* ctx, int64_t n, const int64_t* idx,
+                       int32_t* h_out, int32_t* s_out) {
+    const Ctx* x = C(ctx);
+    if (!x || n < 0 || (n > 0 && (!idx || !h_out || !s_out))) return -1;
+    for (int64_t t = 0; t < n; ++t)
+        if (idx[t] < 0 || idx[t] >= (int64_t)P31) return -1;
+    for (int j = 0; j < x->r; ++j)
+        for (int64_t t = 0; t < n; ++t) {
+            h_out[(int64_t)j * n + t] = (int32_t)bucket(x, j, (uint64_t)idx[t]);
+            s_out[(int64_t)j * n + t] = (int32_t)sign(x, j, (uint64_t)idx[t]);
+        }
+    return 0;
+}
+
+int ssgd_oracle_accumulate(const ssgd_oracle_ctx* ctx, const float* g, int64_t ld_g, float rho,
+                           float* u, float* v, int64_t ld) {
+    const Ctx* x = C(ctx);
+    if (!x || !g || !u || !v || ld_g < x->d || ld < x->d) return -1;
+    for (int w = 0; w < x->W; ++w) {
+        const float* gw = g + (int64_t)w * ld_g;
+        float* uw = u + (int64_t)w * ld;
+        float* vw = v + (int64_t)w * ld;
+        for (int64_t i = 0; i < x->d; ++i) {
+            uw[i] = std::fmaf(rho, uw[i], gw[i]);  // Algorithm 3 line 5: u <- m*u + g
+            vw[i] = vw[i] + uw[i];                 // Algorithm 3 line 6: v <- v + u (new u)
+        }
+    }
+    return 0;
+}
+
+int ssgd_oracle_sketch_f32(const ssgd_oracle_ctx* ctx, const float* x, double* T, double* M) {
+    return sketch_any<float>(C(ctx), x, T, M);
+}
+
+int ssgd_oracle_sketch_f64(const ssgd_oracle_ctx* ctx, const double* x, double* T, double* M) {
+    return sketch_any<double>(C(ctx), x, T, M);
+}
+
+int ssgd_oracle_sketch_workers(const ssgd_oracle_ctx* ctx, const float* v, int64_t ld,
+                               double* T, double* M, double* Tw) {
+    const Ctx* x = C(ctx);
+    if (!x || !v || !T || ld < x->d) return -1;
+    const int64_t rc = (int64_t)x->r * x->c;
+    std::fill(T, T + rc, 0.0);
+    if (M) std::fill(M, M + rc, 0.0);
+    std::vector<double> own;  // one worker's table S^w when the caller does not want all of them
+    if (!Tw) own.resize((size_t)rc);
+    for (int w = 0; w < x->W; ++w) {
+        double* Sw = Tw ? Tw + (int64_t)w * rc : own.data();
+        std::fill(Sw, Sw + rc, 0.0);
+        // Algorithm 3 line 7: worker w sketches its own v.
+        int e = sketch_any<float>(x, v + (int64_t)w * ld, Sw, M);
+        if (e) return e;
+        // Algorithm 3 line 8: the server adds the sketches, w = 0, 1, ..., W-1.
+        for (int64_t t = 0; t < rc; ++t) T[t] += Sw[t];
+    }
+    return 0;
+}
+
+int ssgd_oracle_estimate(const ssgd_oracle_ctx* ctx, const float* Tf, float* est) {
+    const Ctx* x = C(ctx);
+    if (!x || !Tf || !est) return -1;
+    float e[SSGD_ORACLE_MAX_R];
+    for (int64_t i = 0; i < x->d; ++i) {
+        for (int j = 0; j < x->r; ++j)
+            e[j] = (float)sign(x, j, (uint64_t)i) * Tf[(int64_t)j * x->c + bucket(x, j, (uint64_t)i)];
+        // sort the r row estimates (insertion sort) and take the middle one (r is odd)
+        for (int p = 1; p < x->r; ++p) {
+            const float key = e[p];
+            int q = p - 1;
+            while (q >= 0 && e[q] > key) { e[q + 1] = e[q]; --q; }
+            e[q + 1] = key;
+        }
+        est[i] = e[x->r / 2];
+    }
+    return 0;
+}
+
+int ssgd_oracle_select(int64_t n, const float* val, const int32_t* ids, int64_t m, int32_t* out_pos) {
+    if (n < 0 || m < 0 || m > n || n >= (int64_t)P31) return -1;
+    if (n > 0 && !val) return -1;
+    if (m > 0 && !out_pos) return -1;
+    std::vector<int32_t> pos((size_t)n);
+    for (int64_t t = 0; t < n; ++t) pos[(size_t)t] = (int32_t)t;
+    auto better = [&](int32_t p, int32_t q) {
+        const uint32_t kp = abs_bits(val[p]), kq = abs_bits(val[q]);
+        if (kp != kq) return kp > kq;  // larger magnitude first
+        const int32_t ip = ids ? ids[p] : p, iq = ids ? ids[q] : q;
+        if (ip != iq) return ip < iq;  // then smaller coordinate index first
+        return p < q;                  // (duplicate ids: keep it a strict order)
+    };
+    std::sort(pos.begin(), pos.end(), better);
+    for (int64_t t = 0; t < m; ++t) out_pos[t] = pos[(size_t)t];
+    return 0;
+}
+
+int ssgd_oracle_second_round(const ssgd_oracle_ctx* ctx, const float* v, int64_t ld,
+                             const int32_t* cand, int64_t ncand, double* xs) {
+    const Ctx* x = C(ctx);
+    if (!x || !v || ld < x->d || ncand < 0 || (ncand > 0 && (!cand || !xs))) return -1;
+    for (int64_t t = 0; t < ncand; ++t) {
+        if (cand[t] < 0 || cand[t] >= x->d) return -1;
+        double s = 0.0;
+        for (int w = 0; w < x->W; ++w) s += (double)v[(int64_t)w * ld + cand[t]];
+        xs[t] = s;
+    }
+    return 0;
+}
+
+int ssgd_oracle_zero(const ssgd_oracle_ctx* ctx, float* u, float* v, int64_t ld,
+                     const int32_t* idx, int64_t n) {
+    const Ctx* x = C(ctx);
+    if (!x || !u || !v || ld < x->d || n < 0 || (n > 0 && !idx)) return -1;
+    for (int64_t t = 0; t < n; ++t) {
+        if (idx[t] < 0 || idx[t] >= x->d) return -1;
+        for (int w = 0; w < x->W; ++w) {
+            u[(int64_t)w * ld + idx[t]] = 0.0f;
+            v[(int64_t)w * ld + idx[t]] = 0.0f;
+        }
+    }
+    return 0;
+}
+
+int ssgd_oracle_step(const ssgd_oracle_ctx* ctx, const float* g, int64_t ld_g, float rho,
+                     float* u, float* v, int64_t ld, int64_t ncand,
+                     int32_t* out_idx, float* out_val,
+                     double* T_out, double* M_out, float* est_out,
+                     int32_t* cand_out, double* xs_out, int32_t zero_state) {
+    const Ctx* x = C(ctx);
+    if (!x || !out_idx || !out_val) return -1;
+    if (ncand < x->k || ncand > x->d) return -1;
+    const int64_t rc = (int64_t)x->r * x->c;
+    int e;
+
+    // lines 5-6: momentum and error accumulation on every worker
+    if ((e = ssgd_oracle_accumulate(ctx, g, ld_g, rho, u, v, ld))) return e;
+
+    // lines 7-8: per-worker sketches of v, summed by the server
+    std::vector<double> T((size_t)rc), M;
+    if (M_out) M.resize((size_t)rc);
+    if ((e = ssgd_oracle_sketch_workers(ctx, v, ld, T.data(), M_out ? M.data() : nullptr, nullptr)))
+        return e;
+    if (T_out) std::memcpy(T_out, T.data(), sizeof(double) * (size_t)rc);
+    if (M_out) std::memcpy(M_out, M.data(), sizeof(double) * (size_t)rc);
+
+    // line 9: query every coordinate (Algorithm 4 estimate) and keep the ncand = P*k largest by
+    // magnitude.  The counters are rounded to fp32 once; all decisions are on fp32 values.
+    std::vector<float> Tf((size_t)rc);
+    for (int64_t t = 0; t < rc; ++t) Tf[(size_t)t] = (float)T[(size_t)t];
+    std::vector<float> est((size_t)x->d);
+    if ((e = ssgd_oracle_estimate(ctx, Tf.data(), est.data()))) return e;
+    if (est_out) std::memcpy(est_out, est.data(), sizeof(float) * (size_t)x->d);
+    std::vector<int32_t> cand((size_t)ncand);
+    if ((e = ssgd_oracle_select(x->d, est.data(), nullptr, ncand, cand.data()))) return e;
+    if (cand_out) std::memcpy(cand_out, cand.data(), sizeof(int32_t) * (size_t)ncand);
+
+    // line 10: second round -- exact values of v at the candidates, summed over the workers
+    std::vector<double> xs((size_t)ncand);
+    if ((e = ssgd_oracle_second_round(ctx, v, ld, cand.data(), ncand, xs.data()))) return e;
+    if (xs_out) std::memcpy(xs_out, xs.data(), sizeof(double) * (size_t)ncand);
+
+    // line 11: the k-sparse update = the k candidates with the largest exact magnitude
+    std::vector<float> xsf((size_t)ncand);
+    for (int64_t t = 0; t < ncand; ++t) xsf[(size_t)t] = (float)xs[(size_t)t];
+    std::vector<int32_t> best((size_t)x->k);
+    if ((e = ssgd_oracle_select(ncand, xsf.data(), cand.data(), x->k, best.data()))) return e;
+    for (int64_t t = 0; t < x->k; ++t) {
+        out_idx[t] = cand[(size_t)best[(size_t)t]];
+        out_val[t] = xsf[(size_t)best[(size_t)t]];
+    }
+
+    // line 13: momentum-factor masking and error reset at the chosen coordinates
+    if (zero_state)
+        if ((e = ssgd_oracle_zero(ctx, u, v, ld, out_idx, x->k))) return e;
+    return 0;
+}
+
+}  // extern "C"
