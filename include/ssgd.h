@@ -1,0 +1,157 @@
+/*
+ * ssgd.h -- C ABI of the Sketched-SGD compression step for NVIDIA B200 (sm_100a).
+ *
+ * One step of the paper's empirical training procedure (Algorithm 3, lines 5-13) over W workers
+ * whose state lives, batched, on ONE GPU:
+ *
+ *   line 5   momentum                 u_w <- rho*u_w + g_w
+ *   line 6   error accumulation       v_w <- v_w + u_w                       (the new u_w)
+ *   line 7   Count Sketch of v_w      S_w[j][h_j(i)] += s_j(i) * v_w[i]      (Algorithm 4, update)
+ *   line 8   aggregate                S = sum_w S_w                           (plain sum, see below)
+ *   line 9   top-ncand by |estimate|  est[i] = median_j s_j(i)*S[j][h_j(i)]   (Algorithm 4, estimate)
+ *   line 10  second round             xs[m] = sum_w v_w[cand[m]]
+ *   line 11  k-sparse update          the k candidates with the largest |xs|
+ *   line 13  masking / error reset    u_w[i] = v_w[i] = 0 at those k coordinates, every worker
+ *
+ * Conventions
+ *  - Every call returns an int status: SSGD_OK (0) or a negative SSGD_E* code.  Nothing throws,
+ *    aborts or traps.  Arguments are checked on the host before anything is launched.
+ *  - "device" pointers are CUDA device pointers of the current device, owned by the caller.  The
+ *    library allocates no device memory: all scratch is the caller's workspace (ssgd_bind).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Stage calls and
+ *    ssgd_step only enqueue work; they never synchronise.  Results are valid once the stream
+ *    has reached that point.
+ *  - Worker-major layout: g, u, v are [W][ld] fp32, row w at base + w*ld, only the first d entries
+ *    of a row are read or written.  Bases must be 16-byte aligned and ld a multiple of 4
+ *    (SSGD_EALIGN otherwise), ld >= d.
+ *  - Hash family (fixed by the problem statement; Algorithm 4 line 2 leaves it open), p = 2^31-1:
+ *        h_j(i) = ((a_j*i  + b_j ) mod p) mod c
+ *        s_j(i) = 2*(((a'_j*i + b'_j) mod p) & 1) - 1
+ *    with i the 0-based coordinate and j the 0-based row.  a_j, b_j, a'_j, b'_j come from `seed`:
+ *    a 64-bit state s starts at seed; each draw does s += 0x9E3779B97F4A7C15, z = s,
+ *    z = (z^(z>>30))*0xBF58476D1CE4E5B9, z = (z^(z>>27))*0x94D049BB133111EB, out = z^(z>>31);
+ *    row j takes four draws in the order a, b, a', b' with a = 1 + out mod (p-1), b = out mod p.
+ *  - The aggregate is the SUM of the workers' sketches and out_val is the SUM of the workers'
+ *    values (Algorithm 3 line 10 stores the sum; the 1/W of line 8 does not change any selection).
+ *  - Selections use the total order "larger magnitude first (fp32 bit pattern of |x|), then smaller
+ *    coordinate index first", so they are unique given their inputs.
+ *  - Inputs must be finite.  fp32 throughout; the only fused multiply-add is the momentum line.
+ */
+#ifndef SSGD_H
+#define SSGD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SSGD_OK          0
+#define SSGD_EINVAL     -1  /* bad shape, size, NULL pointer, ld < d, k > ncand, ncand > d, even r ... */
+#define SSGD_EALIGN     -2  /* base pointer not 16-byte aligned, or ld not a multiple of 4             */
+#define SSGD_ENOTBOUND  -3  /* ssgd_bind has not been called                                           */
+#define SSGD_EWORKSPACE -4  /* workspace too small for the requested ncand                             */
+#define SSGD_ECUDA      -5  /* a CUDA runtime call failed; ssgd_last_error gives its text              */
+#define SSGD_EDEVICE    -6  /* a kernel recorded an error (index out of range in a caller's list)      */
+#define SSGD_ENOMEM     -7  /* host allocation failed                                                  */
+
+#define SSGD_MAX_R 15
+
+/* Insert variants of ssgd_step (ssgd_set_insert_mode) */
+#define SSGD_INSERT_AUTO   0
+#define SSGD_INSERT_GLOBAL 1  /* reductions straight into the L2-resident r x c table                   */
+#define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
+
+typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
+
+/* Algorithm 4 init(r, c) plus the shape of Algorithm 3: d coordinates, r rows (odd, 1..15), c columns,
+ * k final sparsity, W workers; 1 <= d < 2^31-1, 1 <= c < 2^31-1, 1 <= k <= d, W >= 1.  Host only. */
+int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int32_t W, uint64_t seed);
+int ssgd_destroy(ssgd_ctx* ctx);
+
+/* The 4r hash parameters, row j at out4r[4j..4j+3] = a_j, b_j, a'_j, b'_j (host memory). */
+int ssgd_get_hash_params(const ssgd_ctx* ctx, uint32_t* out4r);
+/* Replace them (for tests): a, a' in [1, p-1], b, b' in [0, p-1]. */
+int ssgd_set_hash_params(ssgd_ctx* ctx, const uint32_t* in4r);
+int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
+
+/* Bytes of device scratch needed to run steps with up to ncand_max candidates (host only). */
+int ssgd_workspace_bytes(const ssgd_ctx* ctx, int64_t ncand_max, size_t* out_bytes);
+
+/* Attach the caller-owned worker state u, v ([W][ld] fp32, device; Algorithm 3 line 1 wants them
+ * zero before the first step) and the caller-owned workspace (device, 256-byte aligned, at least
+ * ssgd_workspace_bytes(ncand_max)).  The buffers must stay valid while the context uses them. */
+int ssgd_bind(ssgd_ctx* ctx, float* u, float* v, int64_t ld, void* workspace, size_t workspace_bytes,
+              int64_t ncand_max);
+
+/* Algorithm 3 lines 5-7 (Algorithm 4 update): updates the bound u, v from g ([W][ld_g] fp32, device,
+ * read only) and writes each worker's own sketch to tables[w] ([W][r][c] fp32, device; zeroed by the
+ * call, then filled with reductions, so bucket sums are order-dependent in the last bits). */
+int ssgd_sketch_accumulate(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, float* tables,
+                           void* stream);
+
+/* Algorithm 3 line 8 (mergeability, Section 3): merged[j][b] = sum over w = 0..W-1, in that order,
+ * of tables[w][j][b].  merged is [r][c] fp32, device. */
+int ssgd_sketch_merge(ssgd_ctx* ctx, const float* tables, float* merged, void* stream);
+
+/* Algorithm 3 line 9 (Algorithm 4 estimate for every coordinate, Section 5.2): computes est[i] for
+ * all i < d from merged ([r][c] fp32, device) and writes the ncand coordinates with the largest
+ * |est| to cand_idx ([ncand] int32, device), in ASCENDING coordinate order.  cand_est ([ncand] fp32)
+ * and est_all ([d] fp32, 16-byte aligned) are optional device outputs (NULL to skip).  k <= ncand <= d. */
+int ssgd_unsketch_candidates(ssgd_ctx* ctx, const float* merged, int64_t ncand, int32_t* cand_idx,
+                             float* cand_est, float* est_all, void* stream);
+
+/* Algorithm 3 lines 10, 11 and 13: sums the bound v over workers at each candidate (fp64, w = 0..W-1),
+ * keeps the k largest by |sum| (ties: earlier position in cand_idx, which is the smaller coordinate
+ * when cand_idx is ascending), writes them to out_idx/out_val ([k], device, in cand_idx order), and
+ * then sets u and v to +0.0f at those k coordinates in every worker.  Entries of cand_idx must be
+ * distinct and in [0, d); an out-of-range entry is skipped and reported by ssgd_status. */
+int ssgd_exact_topk(ssgd_ctx* ctx, const int32_t* cand_idx, int64_t ncand, int32_t* out_idx,
+                    float* out_val, void* stream);
+
+/* Algorithm 3 lines 5-13 in one call: the stages above, with the workers' values summed before the
+ * insert (sum_w S(v_w) = S(sum_w v_w), Section 3), so no per-worker table is materialised.
+ * out_idx/out_val: [k] device outputs, ascending coordinate order. */
+int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t ncand,
+              int32_t* out_idx, float* out_val, void* stream);
+
+/* The same step for a caller whose gradients and results live in HOST memory: copies g_host
+ * ([W][ld_g] fp32; pinned memory makes the copy asynchronous) into g_stage (device, [W][ld_g]),
+ * runs ssgd_step, copies the k results back to out_idx_host/out_val_host and waits for the stream. */
+int ssgd_step_host(ssgd_ctx* ctx, const float* g_host, int64_t ld_g, float rho, int64_t ncand,
+                   float* g_stage, int32_t* out_idx_host, float* out_val_host, void* stream);
+
+/* Device pointers into the workspace holding, after ssgd_step, the merged [r][c] table, est[d] and
+ * the candidate list [ncand] (for tests and diagnostics).  Any of the outputs may be NULL. */
+int ssgd_step_buffers(const ssgd_ctx* ctx, const float** merged, const float** est,
+                      const int32_t** cand_idx, const float** cand_xs);
+
+/* h_j(i), s_j(i) for n coordinates idx[n] (device int32) -> h_out, s_out ([r][n] int32, device).
+ * The same device functions the step uses (Algorithm 4 lines 2, 6, 11); for bit-exactness checks. */
+int ssgd_hashes(ssgd_ctx* ctx, const int32_t* idx, int64_t n, int32_t* h_out, int32_t* s_out,
+                void* stream);
+
+/* Optional per-stage timing of ssgd_step with CUDA events recorded on the caller's stream (up to 256
+ * steps between collections).  Stages: 0 = the accumulate+insert kernel, 1 = the unsketch kernel,
+ * 2 = candidate selection, 3 = second round + final top-k + zero-out.  ssgd_get_stage_times waits for
+ * the stream, writes the summed milliseconds per stage to ms_out[SSGD_NSTAGES] and the number of steps
+ * they cover to steps_out (host memory), and starts a new collection. */
+#define SSGD_NSTAGES 4
+int ssgd_set_timing(ssgd_ctx* ctx, int32_t enable);
+int ssgd_get_stage_times(ssgd_ctx* ctx, void* stream, double* ms_out, int64_t* steps_out);
+
+/* Number of kernels (and memset nodes) the library has launched through this context so far. */
+int ssgd_launch_count(const ssgd_ctx* ctx, int64_t* out);
+
+/* Waits for the stream, then returns SSGD_EDEVICE if a kernel recorded an error since the last call
+ * (the flag is cleared), SSGD_ECUDA if the stream reports a CUDA error, else SSGD_OK. */
+int ssgd_status(ssgd_ctx* ctx, void* stream);
+
+const char* ssgd_strerror(int code);
+const char* ssgd_last_error(const ssgd_ctx* ctx); /* text of the last CUDA error seen, or "" */
+
+#ifdef __cplusplus
+}
+#endif
+#endif

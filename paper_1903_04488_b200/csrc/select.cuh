@@ -1,0 +1,285 @@
+// select.cuh -- exact top-m selection by magnitude (Algorithm 3 lines 9 and 11).
+//
+// Items are positions 0..n-1 of an fp32 array; the key of an item is the bit pattern of |value|
+// (31 bits, monotone in the magnitude, -0 == +0).  The m selected items are the first m under the
+// total order "larger key first, then smaller position first".  The method is a most-significant-
+// digit radix select on 12 + 11 + 8 key bits:
+//
+//   producer kernel   histogram H1 of key bits 30..19          (fused into the kernel that makes the values)
+//   k_sel_pass2       histogram H2 of bits 18..8 among items whose top digit is the threshold digit
+//   k_sel_pass3       histogram H3 of bits 7..0 among items matching the 23-bit threshold prefix
+//   k_sel_count       threshold key T and tie quota Q are now known: per-chunk counts of key > T, key == T
+//   k_sel_scan        exclusive scan of the chunk counts (one block)
+//   emit kernel       item i is selected iff key > T or (key == T and #equal before i < Q); its output
+//                     slot is #greater before i + min(#equal before i, Q): outputs come out in position
+//                     order, with no atomics and no dependence on scheduling.
+//
+// Each histogram is turned into its threshold digit by the LAST block of the kernel that filled it
+// (a fence + ticket counter tells a block that it is the last one to finish; nobody waits), so no
+// single-block "find threshold" launch sits between the passes.
+#pragma once
+#include <stdint.h>
+
+namespace ssgd {
+
+constexpr int SEL_THREADS = 256;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+constexpr int SEL_ITEMS = 16;                          // items per thread in count/emit
+constexpr int SEL_CHUNK = SEL_THREADS * SEL_ITEMS;     // 4096 items per chunk (one block)
+constexpr int H1_BITS = 12, H2_BITS = 11, H3_BITS = 8;
+constexpr int H1_BINS = 1 << H1_BITS, H2_BINS = 1 << H2_BITS, H3_BINS = 1 << H3_BITS;
+constexpr int H1_SHIFT = 31 - H1_BITS;                 // 19
+constexpr int H2_SHIFT = H1_SHIFT - H2_BITS;           // 8
+constexpr int SEL_HIST_WORDS = H1_BINS + H2_BINS + H3_BINS;
+
+// Per-selection state, zeroed before the producer runs.
+struct SelState {
+    uint32_t d1, rem1;   // threshold digit of H1 and how many items are still wanted inside it
+    uint32_t d2, rem2;   // same for H2
+    uint32_t thr_key;    // T: the full 31-bit threshold key
+    uint32_t quota_eq;   // Q >= 1: how many items with key == T are selected
+    uint32_t ticket[3];  // finished-block counters of the three histogram kernels
+    uint32_t pad[7];
+};
+
+struct SelBuffers {
+    uint32_t* h1;        // [H1_BINS]   zeroed before the producer runs
+    uint32_t* h2;        // [H2_BINS]   zeroed
+    uint32_t* h3;        // [H3_BINS]   zeroed
+    SelState* state;
+    uint32_t* chunk_gt;  // [nchunks] counts, then exclusive offsets
+    uint32_t* chunk_eq;  // [nchunks]
+};
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+struct SelShared {
+    uint32_t hist[H1_BINS];
+    uint32_t warp_sum[SEL_WARPS];
+    uint32_t found[2];
+    uint32_t last;
+};
+
+// True, in every thread of the block, iff this block is the last of the grid to get here.  Everything
+// the other blocks wrote to global memory before their own call is then visible to this block.
+__device__ __forceinline__ bool block_is_last(uint32_t* ticket, SelShared& sh) {
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) sh.last = (atomicAdd(ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    return sh.last != 0;
+}
+
+// Largest digit D with count(bins > D) < want <= count(bins >= D); rem = want - count(bins > D).
+// Whole block (SEL_THREADS threads) must call.  Requires 1 <= want <= total count.
+template <int NBINS>
+__device__ __forceinline__ void block_find_from_top(const uint32_t* __restrict__ gh, uint32_t want,
+                                                    SelShared& sh, uint32_t& digit, uint32_t& rem) {
+    constexpr int PER = NBINS / SEL_THREADS;  // 16, 8, 1
+    static_assert(PER >= 1 && PER * SEL_THREADS == NBINS, "bins must be a multiple of the block");
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    for (int b = t; b < NBINS; b += SEL_THREADS) sh.hist[b] = __ldcg(gh + b);  // L2: other blocks' atomics
+    if (t == 0) { sh.found[0] = 0; sh.found[1] = 1; }
+    __syncthreads();
+    uint32_t sum = 0;
+#pragma unroll
+    for (int s = 0; s < PER; ++s) sum += sh.hist[t * PER + ((s + t) % PER)];  // rotated: no bank conflicts
+    uint32_t incl = sum;  // sum over lanes >= lane of this warp
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    if (lane == 0) sh.warp_sum[warp] = incl;
+    __syncthreads();
+    uint32_t above = incl - sum;
+    for (int w2 = warp + 1; w2 < SEL_WARPS; ++w2) above += sh.warp_sum[w2];
+    if (above < want && want <= above + sum) {
+        uint32_t acc = above;
+        for (int b = t * PER + PER - 1; b >= t * PER; --b) {
+            const uint32_t h = sh.hist[b];
+            if (acc + h >= want) { sh.found[0] = (uint32_t)b; sh.found[1] = want - acc; break; }
+            acc += h;
+        }
+    }
+    __syncthreads();
+    digit = sh.found[0];
+    rem = sh.found[1];
+    __syncthreads();  // sh.hist may be reused by the caller
+}
+
+// Adds a block-private histogram (shared memory) into the global one, skipping empty bins.
+template <int NBINS>
+__device__ __forceinline__ void flush_hist(const uint32_t* s_hist, uint32_t* __restrict__ gh) {
+    for (int b = threadIdx.x; b < NBINS; b += blockDim.x) {
+        const uint32_t h = s_hist[b];
+        if (h) atomicAdd(&gh[b], h);
+    }
+}
+
+// ---- pass 2: H2 over items whose top digit equals the threshold digit -----------------------------
+__global__ void __launch_bounds__(SEL_THREADS)
+k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
+    __shared__ SelShared sh;
+    const uint32_t d1 = sb.state->d1;
+    for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
+    for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
+        const uint32_t key = key_of(val[i]);
+        if ((key >> H1_SHIFT) == d1) atomicAdd(&sh.hist[(key >> H2_SHIFT) & (H2_BINS - 1)], 1u);
+    }
+    __syncthreads();
+    flush_hist<H2_BINS>(sh.hist, sb.h2);
+    if (block_is_last(&sb.state->ticket[1], sh)) {
+        uint32_t d2, rem2;
+        block_find_from_top<H2_BINS>(sb.h2, sb.state->rem1, sh, d2, rem2);
+        if (threadIdx.x == 0) { sb.state->d2 = d2; sb.state->rem2 = rem2; }
+    }
+}
+
+// ---- pass 3: H3 over items matching the 23-bit prefix; its last block publishes T and Q -----------
+__global__ void __launch_bounds__(SEL_THREADS)
+k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
+    __shared__ SelShared sh;
+    const uint32_t d1 = sb.state->d1, d2 = sb.state->d2;
+    const uint32_t prefix = (d1 << H2_BITS) | d2;
+    for (int b = threadIdx.x; b < H3_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
+    for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
+        const uint32_t key = key_of(val[i]);
+        if ((key >> H2_SHIFT) == prefix) atomicAdd(&sh.hist[key & (H3_BINS - 1)], 1u);
+    }
+    __syncthreads();
+    flush_hist<H3_BINS>(sh.hist, sb.h3);
+    if (block_is_last(&sb.state->ticket[2], sh)) {
+        uint32_t d3, rem3;
+        block_find_from_top<H3_BINS>(sb.h3, sb.state->rem2, sh, d3, rem3);
+        if (threadIdx.x == 0) {
+            sb.state->thr_key = (d1 << H1_SHIFT) | (d2 << H2_SHIFT) | d3;
+            sb.state->quota_eq = rem3;
+        }
+    }
+}
+
+// For producer kernels (SEL_THREADS threads, histogram H1 already flushed): the last block turns H1
+// into the first threshold digit.  `want` = how many items the selection keeps.
+__device__ __forceinline__ void producer_epilogue(const SelBuffers& sb, uint32_t want, SelShared& sh) {
+    if (block_is_last(&sb.state->ticket[0], sh)) {
+        uint32_t d1, rem1;
+        block_find_from_top<H1_BINS>(sb.h1, want, sh, d1, rem1);
+        if (threadIdx.x == 0) { sb.state->d1 = d1; sb.state->rem1 = rem1; }
+    }
+}
+
+// Warp w of a block owns items [chunk*SEL_CHUNK + w*512, +512), read 32 at a time (coalesced).
+// Returns, as ballots per iteration, which lanes hold key > T (bg) and key == T (be).
+__device__ __forceinline__ void chunk_ballots(const float* __restrict__ val, int64_t n, int64_t warp_base,
+                                              uint32_t T, uint32_t (&bg)[SEL_ITEMS], uint32_t (&be)[SEL_ITEMS],
+                                              uint32_t& ngt, uint32_t& neq) {
+    const int lane = threadIdx.x & 31;
+    ngt = 0; neq = 0;
+#pragma unroll
+    for (int it = 0; it < SEL_ITEMS; ++it) {
+        const int64_t i = warp_base + it * 32 + lane;
+        uint32_t key = 0; bool ok = i < n;
+        if (ok) key = key_of(val[i]);
+        bg[it] = __ballot_sync(0xFFFFFFFFu, ok && key > T);
+        be[it] = __ballot_sync(0xFFFFFFFFu, ok && key == T);
+        ngt += __popc(bg[it]);
+        neq += __popc(be[it]);
+    }
+}
+
+// ---- count: per-chunk numbers of key > T and key == T ---------------------------------------------
+__global__ void __launch_bounds__(SEL_THREADS)
+k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb) {
+    __shared__ uint32_t s_cnt[2 * SEL_WARPS];
+    const uint32_t T = sb.state->thr_key;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
+    chunk_ballots(val, n, (int64_t)blockIdx.x * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS), T, bg, be, ngt, neq);
+    if (lane == 0) { s_cnt[warp] = ngt; s_cnt[SEL_WARPS + warp] = neq; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t a = 0, b = 0;
+        for (int w = 0; w < SEL_WARPS; ++w) { a += s_cnt[w]; b += s_cnt[SEL_WARPS + w]; }
+        sb.chunk_gt[blockIdx.x] = a;
+        sb.chunk_eq[blockIdx.x] = b;
+    }
+}
+
+// ---- scan: chunk counts -> exclusive offsets (single block of 1024 threads) ------------------------
+__global__ void __launch_bounds__(1024)
+k_sel_scan(SelBuffers sb, int64_t nchunks) {
+    __shared__ uint32_t s_g[32], s_e[32];
+    __shared__ uint32_t carry_g, carry_e;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    if (t == 0) { carry_g = 0; carry_e = 0; }
+    __syncthreads();
+    for (int64_t base = 0; base < nchunks; base += 1024) {
+        const int64_t i = base + t;
+        const uint32_t g = i < nchunks ? sb.chunk_gt[i] : 0, e = i < nchunks ? sb.chunk_eq[i] : 0;
+        uint32_t ig = g, ie = e;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t og = __shfl_up_sync(0xFFFFFFFFu, ig, off), oe = __shfl_up_sync(0xFFFFFFFFu, ie, off);
+            if (lane >= off) { ig += og; ie += oe; }
+        }
+        if (lane == 31) { s_g[warp] = ig; s_e[warp] = ie; }
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t wg = s_g[lane], we = s_e[lane];
+            uint32_t xg = wg, xe = we;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t og = __shfl_up_sync(0xFFFFFFFFu, xg, off), oe = __shfl_up_sync(0xFFFFFFFFu, xe, off);
+                if (lane >= off) { xg += og; xe += oe; }
+            }
+            s_g[lane] = xg - wg;  // exclusive over warps
+            s_e[lane] = xe - we;
+        }
+        __syncthreads();
+        const uint32_t cg = carry_g, ce = carry_e;
+        if (i < nchunks) {
+            sb.chunk_gt[i] = cg + s_g[warp] + ig - g;
+            sb.chunk_eq[i] = ce + s_e[warp] + ie - e;
+        }
+        __syncthreads();
+        if (t == 1023) { carry_g = cg + s_g[warp] + ig; carry_e = ce + s_e[warp] + ie; }
+        __syncthreads();
+    }
+}
+
+// ---- emit: ordered compaction of the selected items -----------------------------------------------
+// `sink(slot, i)` is called once for every selected item i with its output slot (0 .. m-1).
+template <typename Sink>
+__device__ __forceinline__ void sel_emit_chunk(const float* __restrict__ val, int64_t n, const SelBuffers& sb,
+                                               Sink sink) {
+    __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
+    const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t warp_base = (int64_t)blockIdx.x * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS);
+    uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
+    chunk_ballots(val, n, warp_base, T, bg, be, ngt, neq);
+    if (lane == 0) { s_wg[warp] = ngt; s_we[warp] = neq; }
+    __syncthreads();
+    uint32_t gt_before = sb.chunk_gt[blockIdx.x], eq_before = sb.chunk_eq[blockIdx.x];
+    for (int w = 0; w < warp; ++w) { gt_before += s_wg[w]; eq_before += s_we[w]; }
+    const uint32_t lt_mask = (1u << lane) - 1u;
+#pragma unroll
+    for (int it = 0; it < SEL_ITEMS; ++it) {
+        const uint32_t g = gt_before + __popc(bg[it] & lt_mask);
+        const uint32_t e = eq_before + __popc(be[it] & lt_mask);
+        const bool is_gt = (bg[it] >> lane) & 1u, is_eq = (be[it] >> lane) & 1u;
+        if (is_gt || (is_eq && e < Q)) sink(g + (e < Q ? e : Q), warp_base + it * 32 + lane);
+        gt_before += __popc(bg[it]);
+        eq_before += __popc(be[it]);
+    }
+}
+
+#endif  // __CUDACC__
+}  // namespace ssgd

@@ -1,0 +1,905 @@
+// ssgd.cu -- kernels and C ABI of the Sketched-SGD compression step for sm_100a.
+//
+// Kernels (Algorithm 3 lines 5-13, Algorithm 4):
+//   k_accum_insert      lines 5-7: streams g, u, v once (128-bit loads/stores), updates u and v, and
+//                       inserts into the sketch with reductions (red.global.add.f32) -- either the sum
+//                       over workers into one merged table (linearity, Section 3), or every worker's
+//                       value into its own table, or into a shared-memory table flushed per block.
+//   k_merge             line 8: sum of the per-worker tables in worker order.
+//   k_unsketch          line 9, first half: median-of-r estimate of every coordinate from the L2-resident
+//                       table, plus the first radix histogram of |estimate|.
+//   k_sel_*             lines 9 and 11: exact radix select (select.cuh).
+//   k_gather            line 10: second-round sums of v over workers at the candidates (fp64, fixed order).
+//   k_zero              line 13: u = v = 0 at the chosen coordinates.
+// HBM-bound work is the first kernel (20 bytes per worker-coordinate); nothing here is a dense
+// contraction, so there are no tensor-core instructions.
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "../../include/ssgd.h"
+#include "hash.cuh"
+#include "select.cuh"
+
+namespace ssgd {
+
+// ------------------------------------------------------------------------------------------------
+// small device helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void red_add(float* addr, float x) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(x) : "memory");
+}
+
+constexpr int ERR_BAD_INDEX = 1;
+
+// ------------------------------------------------------------------------------------------------
+// K1: momentum + error accumulation + sketch insert
+// ------------------------------------------------------------------------------------------------
+enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2 };
+
+struct AccumArgs {
+    const float* g; int64_t ld_g;
+    float* u; float* v; int64_t ld;
+    int32_t W; int64_t d; float rho;
+    float* table;        // merged [r][c], or per-worker [W][r][c]
+    int64_t c;
+    HashParams hp; Bucketizer bk;
+};
+
+constexpr int K1_THREADS = 256;
+constexpr int K1_UNROLL = 4;  // workers in flight per thread: 3 x 16 B loads each
+
+template <int R, bool POW2, int MODE>
+__global__ void __launch_bounds__(K1_THREADS)
+k_accum_insert(const AccumArgs A) {
+    extern __shared__ float s_table[];  // MODE == INS_MERGED_SMEM: [R][c]
+    const int64_t rc = (int64_t)R * A.c;
+    if (MODE == INS_MERGED_SMEM) {
+        for (int64_t t = threadIdx.x; t < rc; t += K1_THREADS) s_table[t] = 0.0f;
+        __syncthreads();
+    }
+    const int64_t groups = (A.d + 3) >> 2;
+    const int64_t stride = (int64_t)gridDim.x * K1_THREADS;
+    for (int64_t q = (int64_t)blockIdx.x * K1_THREADS + threadIdx.x; q < groups; q += stride) {
+        const int64_t i0 = q << 2;
+        uint32_t hb[R][4];
+        if (MODE == INS_PER_WORKER) {
+#pragma unroll
+            for (int j = 0; j < R; ++j) row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb[j]);
+        }
+        float x[4] = {0.f, 0.f, 0.f, 0.f};  // sum over workers of the new v (worker order)
+        if (i0 + 3 < A.d) {
+            for (int w0 = 0; w0 < A.W; w0 += K1_UNROLL) {
+                float4 gg[K1_UNROLL], uu[K1_UNROLL], vv[K1_UNROLL];
+#pragma unroll
+                for (int s = 0; s < K1_UNROLL; ++s) {
+                    if (w0 + s < A.W) {
+                        const int64_t w = w0 + s;
+                        gg[s] = __ldcs(reinterpret_cast<const float4*>(A.g + w * A.ld_g + i0));
+                        uu[s] = __ldcs(reinterpret_cast<const float4*>(A.u + w * A.ld + i0));
+                        vv[s] = __ldcs(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
+                    }
+                }
+#pragma unroll
+                for (int s = 0; s < K1_UNROLL; ++s) {
+                    if (w0 + s < A.W) {
+                        const int64_t w = w0 + s;
+                        float4 un, vn;
+                        un.x = __fmaf_rn(A.rho, uu[s].x, gg[s].x); vn.x = __fadd_rn(vv[s].x, un.x);
+                        un.y = __fmaf_rn(A.rho, uu[s].y, gg[s].y); vn.y = __fadd_rn(vv[s].y, un.y);
+                        un.z = __fmaf_rn(A.rho, uu[s].z, gg[s].z); vn.z = __fadd_rn(vv[s].z, un.z);
+                        un.w = __fmaf_rn(A.rho, uu[s].w, gg[s].w); vn.w = __fadd_rn(vv[s].w, un.w);
+                        __stcs(reinterpret_cast<float4*>(A.u + w * A.ld + i0), un);
+                        __stcs(reinterpret_cast<float4*>(A.v + w * A.ld + i0), vn);
+                        if (MODE == INS_PER_WORKER) {
+                            float* tw = A.table + w * rc;
+                            const float vals[4] = {vn.x, vn.y, vn.z, vn.w};
+#pragma unroll
+                            for (int j = 0; j < R; ++j)
+#pragma unroll
+                                for (int e = 0; e < 4; ++e)
+                                    if (vals[e] != 0.0f)
+                                        red_add(tw + (int64_t)j * A.c + (hb[j][e] & P31), apply_sign(vals[e], hb[j][e]));
+                        } else {
+                            x[0] = __fadd_rn(x[0], vn.x); x[1] = __fadd_rn(x[1], vn.y);
+                            x[2] = __fadd_rn(x[2], vn.z); x[3] = __fadd_rn(x[3], vn.w);
+                        }
+                    }
+                }
+            }
+        } else {
+            // ragged last group (d not a multiple of 4): scalar, bounds-checked
+            for (int e = 0; e < 4; ++e) {
+                const int64_t i = i0 + e;
+                if (i >= A.d) break;
+                for (int64_t w = 0; w < A.W; ++w) {
+                    const float un = __fmaf_rn(A.rho, A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
+                    const float vn = __fadd_rn(A.v[w * A.ld + i], un);
+                    A.u[w * A.ld + i] = un;
+                    A.v[w * A.ld + i] = vn;
+                    if (MODE == INS_PER_WORKER) {
+#pragma unroll
+                        for (int j = 0; j < R; ++j)
+                            if (vn != 0.0f)
+                                red_add(A.table + w * rc + (int64_t)j * A.c + (hb[j][e] & P31),
+                                        apply_sign(vn, hb[j][e]));
+                    } else {
+                        x[e] = __fadd_rn(x[e], vn);
+                    }
+                }
+            }
+        }
+        if (MODE != INS_PER_WORKER) {
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                uint32_t h1[4];
+                row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, h1);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (i0 + e < A.d && x[e] != 0.0f) {
+                        const float sx = apply_sign(x[e], h1[e]);
+                        if (MODE == INS_MERGED_SMEM) atomicAdd(&s_table[(int64_t)j * A.c + (h1[e] & P31)], sx);
+                        else red_add(A.table + (int64_t)j * A.c + (h1[e] & P31), sx);
+                    }
+                }
+            }
+        }
+    }
+    if (MODE == INS_MERGED_SMEM) {
+        __syncthreads();
+        for (int64_t t = threadIdx.x; t < rc; t += K1_THREADS) {
+            const float s = s_table[t];
+            if (s != 0.0f) red_add(A.table + t, s);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// K2: merge of the per-worker tables, worker order
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_merge(const float* __restrict__ tables, float* __restrict__ merged, int64_t rc, int32_t W) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if ((rc & 3) == 0) {
+        const int64_t n4 = rc >> 2;
+        for (int64_t q = t0; q < n4; q += stride) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int w0 = 0; w0 < W; w0 += 8) {
+                float4 t[8];
+#pragma unroll
+                for (int s = 0; s < 8; ++s)
+                    if (w0 + s < W) t[s] = __ldcs(reinterpret_cast<const float4*>(tables + (int64_t)(w0 + s) * rc) + q);
+#pragma unroll
+                for (int s = 0; s < 8; ++s)
+                    if (w0 + s < W) {
+                        acc.x = __fadd_rn(acc.x, t[s].x); acc.y = __fadd_rn(acc.y, t[s].y);
+                        acc.z = __fadd_rn(acc.z, t[s].z); acc.w = __fadd_rn(acc.w, t[s].w);
+                    }
+            }
+            reinterpret_cast<float4*>(merged)[q] = acc;
+        }
+    } else {
+        for (int64_t t = t0; t < rc; t += stride) {
+            float acc = 0.f;
+            for (int w = 0; w < W; ++w) acc = __fadd_rn(acc, tables[(int64_t)w * rc + t]);
+            merged[t] = acc;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// K3: estimate of every coordinate (median of r signed buckets) + first histogram of |estimate|
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cswap(float& a, float& b) {
+    const float lo = fminf(a, b), hi = fmaxf(a, b);
+    a = lo; b = hi;
+}
+
+template <int R>
+__device__ __forceinline__ float median_of(float (&a)[R]) {
+    if constexpr (R == 1) {
+        return a[0];
+    } else if constexpr (R == 3) {
+        return fmaxf(fminf(a[0], a[1]), fminf(fmaxf(a[0], a[1]), a[2]));
+    } else if constexpr (R == 5) {
+        // sort two pairs; the smaller of the two minima and the larger of the two maxima cannot be
+        // the median; the median of the remaining three is the median of five
+        cswap(a[0], a[1]); cswap(a[3], a[4]);
+        const float lo = fmaxf(a[0], a[3]);   // larger of the pair minima
+        const float hi = fminf(a[1], a[4]);   // smaller of the pair maxima
+        return fmaxf(fminf(lo, hi), fminf(fmaxf(lo, hi), a[2]));
+    } else {
+        // general odd R: odd-even transposition sort in registers, then the middle element
+#pragma unroll
+        for (int round = 0; round < R; ++round)
+#pragma unroll
+            for (int p = round & 1; p + 1 < R; p += 2) cswap(a[p], a[p + 1]);
+        return a[R / 2];
+    }
+}
+
+struct UnsketchArgs {
+    const float* table; int64_t c; int64_t d;
+    HashParams hp; Bucketizer bk;
+    float* est;          // [d], 16-byte aligned
+    SelBuffers sb;       // selection buffers of the candidate stage (H1 filled here)
+    uint32_t want;       // ncand
+};
+
+constexpr int K3_THREADS = 256;
+
+template <int R, bool POW2>
+__global__ void __launch_bounds__(K3_THREADS)
+k_unsketch(const UnsketchArgs A) {
+    __shared__ SelShared sh;
+    uint32_t* s_hist = sh.hist;
+    for (int b = threadIdx.x; b < H1_BINS; b += K3_THREADS) s_hist[b] = 0;
+    __syncthreads();
+    const int64_t groups = (A.d + 3) >> 2;
+    const int64_t stride = (int64_t)gridDim.x * K3_THREADS;
+    for (int64_t q = (int64_t)blockIdx.x * K3_THREADS + threadIdx.x; q < groups; q += stride) {
+        const int64_t i0 = q << 2;
+        float rowv[4][R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            uint32_t hb[4];
+            row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                rowv[e][j] = apply_sign(__ldg(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
+        }
+        float m[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m[e] = median_of<R>(rowv[e]);
+        if (i0 + 3 < A.d) {
+            *reinterpret_cast<float4*>(A.est + i0) = make_float4(m[0], m[1], m[2], m[3]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
+        } else {
+            for (int e = 0; e < 4 && i0 + e < A.d; ++e) {
+                A.est[i0 + e] = m[e];
+                atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(s_hist, A.sb.h1);
+    producer_epilogue(A.sb, A.want, sh);
+}
+
+// ------------------------------------------------------------------------------------------------
+// candidate emit (line 9, second half)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SEL_THREADS)
+k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32_t* __restrict__ cand_idx,
+                  float* __restrict__ cand_est) {
+    sel_emit_chunk(est, d, sb, [&](uint32_t slot, int64_t i) {
+        cand_idx[slot] = (int32_t)i;
+        if (cand_est) cand_est[slot] = est[i];
+    });
+}
+
+// ------------------------------------------------------------------------------------------------
+// K5: second round -- xs[m] = sum_w v_w[cand[m]] (fp64, w = 0..W-1), rounded once to fp32
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ v, int64_t ld, int32_t W,
+         int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag) {
+    __shared__ SelShared sh;
+    uint32_t* s_hist = sh.hist;
+    for (int b = threadIdx.x; b < H1_BINS; b += 256) s_hist[b] = 0;
+    __syncthreads();
+    const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (m < ncand) {
+        const int64_t i = cand[m];
+        float out = 0.0f;
+        if (i < 0 || i >= d) {
+            atomicExch(errflag, ERR_BAD_INDEX);
+        } else {
+            double acc = 0.0;
+            const float* p = v + i;
+            int w = 0;
+            for (; w + 8 <= W; w += 8) {
+                float t[8];
+#pragma unroll
+                for (int s = 0; s < 8; ++s) t[s] = __ldg(p + (int64_t)(w + s) * ld);
+#pragma unroll
+                for (int s = 0; s < 8; ++s) acc = __dadd_rn(acc, (double)t[s]);
+            }
+            for (; w < W; ++w) acc = __dadd_rn(acc, (double)__ldg(p + (int64_t)w * ld));
+            out = (float)acc;
+        }
+        xs[m] = out;
+        atomicAdd(&s_hist[key_of(out) >> H1_SHIFT], 1u);
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(s_hist, sb.h1);
+    producer_epilogue(sb, want, sh);
+}
+
+// ------------------------------------------------------------------------------------------------
+// final emit (line 11) and zero-out (line 13)
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SEL_THREADS)
+k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const int32_t* __restrict__ cand,
+             int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
+    sel_emit_chunk(xs, ncand, sb, [&](uint32_t slot, int64_t m) {
+        out_idx[slot] = cand[m];
+        out_val[slot] = xs[m];
+    });
+}
+
+__global__ void __launch_bounds__(256)
+k_zero(const int32_t* __restrict__ out_idx, int64_t k, float* __restrict__ u, float* __restrict__ v,
+       int64_t ld, int32_t W, int64_t d) {
+    const int64_t total = k * (int64_t)W;
+    const int64_t stride = (int64_t)gridDim.x * 256;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += stride) {
+        const int64_t w = t / k, m = t - w * k;   // consecutive threads: consecutive chosen coordinates
+        const int64_t i = out_idx[m];
+        if (i >= 0 && i < d) {
+            u[w * ld + i] = 0.0f;
+            v[w * ld + i] = 0.0f;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// hash dump for bit-exactness checks
+// ------------------------------------------------------------------------------------------------
+template <bool POW2>
+__global__ void __launch_bounds__(256)
+k_hashes(const int32_t* __restrict__ idx, int64_t n, int32_t r, HashParams hp, Bucketizer bk,
+         int32_t* __restrict__ h_out, int32_t* __restrict__ s_out) {
+    const int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (t >= n) return;
+    const uint32_t i = (uint32_t)idx[t];
+    for (int j = 0; j < r; ++j) {
+        uint32_t hb[1];
+        row_hashes<POW2, 1>(hp.row[j], bk, i, hb);
+        h_out[(int64_t)j * n + t] = (int32_t)(hb[0] & P31);
+        s_out[(int64_t)j * n + t] = (hb[0] >> 31) ? -1 : 1;
+    }
+}
+
+}  // namespace ssgd
+
+// ==================================================================================================
+// host side: context, argument checks, launch plans
+// ==================================================================================================
+using namespace ssgd;
+
+struct ssgd_ctx {
+    int64_t d, c, k;
+    int32_t r, W;
+    uint64_t seed;
+    HashParams hp;
+    Bucketizer bk;
+    bool pow2;
+    int32_t insert_mode;
+    // binding
+    float* u; float* v; int64_t ld;
+    char* ws; size_t ws_bytes; int64_t ncand_max;
+    // workspace layout (byte offsets)
+    size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
+    size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
+    int64_t nchunk_c, nchunk_f;
+    // device facts
+    int device; int sm_count; int max_smem_optin;
+    int64_t launches;
+    // optional per-stage timing of ssgd_step (CUDA events on the caller's stream)
+    bool timing;
+    cudaEvent_t* ev;        // [TIMING_SLOTS][SSGD_NSTAGES + 1]
+    int32_t ev_steps;       // steps recorded since the last collection
+    std::string last_error;
+};
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+constexpr int TIMING_SLOTS = 256;
+constexpr int EV_PER_STEP = SSGD_NSTAGES + 1;
+inline size_t up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+void derive_params(uint64_t seed, int32_t r, HashParams& hp) {
+    uint64_t s = seed;
+    auto next = [&s]() -> uint64_t {
+        s += 0x9E3779B97F4A7C15ull;
+        uint64_t z = s;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+        return z ^ (z >> 31);
+    };
+    const uint64_t p = P31;
+    for (int j = 0; j < r; ++j) {
+        hp.row[j].a = (uint32_t)(1 + next() % (p - 1));
+        hp.row[j].b = (uint32_t)(next() % p);
+        hp.row[j].a2 = (uint32_t)(1 + next() % (p - 1));
+        hp.row[j].b2 = (uint32_t)(next() % p);
+    }
+}
+
+void layout(ssgd_ctx* x, int64_t ncand_max) {
+    size_t o = 0;
+    x->off_table = o;   o += up((size_t)x->r * x->c * 4);
+    x->off_hist_c = o;  o += up(SEL_HIST_WORDS * 4);
+    x->off_state_c = o; o += up(sizeof(SelState));
+    x->off_hist_f = o;  o += up(SEL_HIST_WORDS * 4);
+    x->off_state_f = o; o += up(sizeof(SelState));
+    x->off_err = o;     o += up(16);
+    x->zero_bytes = o;
+    x->nchunk_c = (x->d + SEL_CHUNK - 1) / SEL_CHUNK;
+    x->nchunk_f = (ncand_max + SEL_CHUNK - 1) / SEL_CHUNK;
+    x->off_est = o;     o += up((size_t)x->d * 4);
+    x->off_chunk_c = o; o += up((size_t)x->nchunk_c * 8);
+    x->off_chunk_f = o; o += up((size_t)x->nchunk_f * 8);
+    x->off_cand = o;    o += up((size_t)ncand_max * 4);
+    x->off_xs = o;      o += up((size_t)ncand_max * 4);
+    x->off_oidx = o;    o += up((size_t)x->k * 4);
+    x->off_oval = o;    o += up((size_t)x->k * 4);
+    x->total_bytes = o;
+}
+
+SelBuffers sel_buffers(ssgd_ctx* x, bool final_stage) {
+    SelBuffers sb;
+    uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_hist_f : x->off_hist_c));
+    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
+    sb.state = reinterpret_cast<SelState*>(x->ws + (final_stage ? x->off_state_f : x->off_state_c));
+    uint32_t* ch = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_chunk_f : x->off_chunk_c));
+    const int64_t nch = final_stage ? x->nchunk_f : x->nchunk_c;
+    sb.chunk_gt = ch; sb.chunk_eq = ch + nch;
+    return sb;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int cuda_fail(ssgd_ctx* x, cudaError_t e, const char* what) {
+    x->last_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return SSGD_ECUDA;
+}
+
+#define CU(call, what)                                                   \
+    do {                                                                 \
+        cudaError_t e_ = (call);                                         \
+        if (e_ != cudaSuccess) return cuda_fail(x, e_, what);            \
+    } while (0)
+
+#define LAUNCHED(what)                                                   \
+    do {                                                                 \
+        x->launches++;                                                   \
+        cudaError_t e_ = cudaGetLastError();                             \
+        if (e_ != cudaSuccess) return cuda_fail(x, e_, what);            \
+    } while (0)
+
+int ensure_device(ssgd_ctx* x) {
+    if (x->device >= 0) return SSGD_OK;
+    int dev = 0;
+    CU(cudaGetDevice(&dev), "cudaGetDevice");
+    CU(cudaDeviceGetAttribute(&x->sm_count, cudaDevAttrMultiProcessorCount, dev), "sm count");
+    CU(cudaDeviceGetAttribute(&x->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev), "smem optin");
+    x->device = dev;
+    return SSGD_OK;
+}
+
+inline int grid_for(int64_t items, int threads, int64_t cap) {
+    int64_t b = (items + threads - 1) / threads;
+    if (b < 1) b = 1;
+    if (b > cap) b = cap;
+    return (int)b;
+}
+
+// ---- K1 dispatch over (R, POW2, MODE) ------------------------------------------------------------
+template <int R, bool POW2, int MODE>
+int launch_accum_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    if (MODE == INS_MERGED_SMEM) {
+        const size_t smem = (size_t)R * A.c * 4;
+        CU(cudaFuncSetAttribute(k_accum_insert<R, POW2, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)smem), "smem attribute");
+        const int grid = grid_for(groups, K1_THREADS, x->sm_count);
+        k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, smem, st>>>(A);
+    } else {
+        const int grid = grid_for(groups, K1_THREADS, (int64_t)1 << 30);
+        k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, 0, st>>>(A);
+    }
+    LAUNCHED("k_accum_insert");
+    return SSGD_OK;
+}
+
+template <int R, bool POW2>
+int launch_accum_m(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
+    switch (mode) {
+        case INS_MERGED_GLOBAL: return launch_accum_t<R, POW2, INS_MERGED_GLOBAL>(x, A, st);
+        case INS_PER_WORKER: return launch_accum_t<R, POW2, INS_PER_WORKER>(x, A, st);
+        default: return launch_accum_t<R, POW2, INS_MERGED_SMEM>(x, A, st);
+    }
+}
+
+#define DISPATCH_R(fn, ...)                                                       \
+    switch (x->r) {                                                               \
+        case 1: return x->pow2 ? fn<1, true>(__VA_ARGS__) : fn<1, false>(__VA_ARGS__);    \
+        case 3: return x->pow2 ? fn<3, true>(__VA_ARGS__) : fn<3, false>(__VA_ARGS__);    \
+        case 5: return x->pow2 ? fn<5, true>(__VA_ARGS__) : fn<5, false>(__VA_ARGS__);    \
+        case 7: return x->pow2 ? fn<7, true>(__VA_ARGS__) : fn<7, false>(__VA_ARGS__);    \
+        case 9: return x->pow2 ? fn<9, true>(__VA_ARGS__) : fn<9, false>(__VA_ARGS__);    \
+        case 11: return x->pow2 ? fn<11, true>(__VA_ARGS__) : fn<11, false>(__VA_ARGS__); \
+        case 13: return x->pow2 ? fn<13, true>(__VA_ARGS__) : fn<13, false>(__VA_ARGS__); \
+        case 15: return x->pow2 ? fn<15, true>(__VA_ARGS__) : fn<15, false>(__VA_ARGS__); \
+        default: return SSGD_EINVAL;                                              \
+    }
+
+int launch_accum(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
+    DISPATCH_R(launch_accum_m, x, A, mode, st)
+}
+
+template <int R, bool POW2>
+int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    // a few blocks per SM: each block pays one histogram flush
+    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * 8);
+    k_unsketch<R, POW2><<<grid, K3_THREADS, 0, st>>>(A);
+    LAUNCHED("k_unsketch");
+    return SSGD_OK;
+}
+
+int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_unsketch_t, x, A, st)
+}
+
+// Radix-select passes after the producer filled H1: leaves thresholds in sb.state and exclusive
+// chunk offsets in sb.chunk_*; the caller launches the emit kernel over `nchunks` blocks.
+int launch_select(ssgd_ctx* x, const float* val, int64_t n, const SelBuffers& sb, int64_t nchunks,
+                  cudaStream_t st) {
+    const int grid = grid_for(n, SEL_THREADS * 8, (int64_t)x->sm_count * 8);
+    k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(val, n, sb);
+    LAUNCHED("k_sel_pass2");
+    k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(val, n, sb);
+    LAUNCHED("k_sel_pass3");
+    k_sel_count<<<(int)nchunks, SEL_THREADS, 0, st>>>(val, n, sb);
+    LAUNCHED("k_sel_count");
+    k_sel_scan<<<1, 1024, 0, st>>>(sb, nchunks);
+    LAUNCHED("k_sel_scan");
+    return SSGD_OK;
+}
+
+int check_bound(const ssgd_ctx* x) {
+    if (!x) return SSGD_EINVAL;
+    if (!x->u || !x->v || !x->ws) return SSGD_ENOTBOUND;
+    return SSGD_OK;
+}
+
+int check_g(const ssgd_ctx* x, const float* g, int64_t ld_g) {
+    if (!g || ld_g < x->d) return SSGD_EINVAL;
+    if (!aligned16(g) || (ld_g & 3)) return SSGD_EALIGN;
+    return SSGD_OK;
+}
+
+// Stage boundary `which` of the step being recorded (no-op unless timing is on and a slot is free).
+int mark(ssgd_ctx* x, int which, cudaStream_t st) {
+    if (!x->timing || x->ev_steps >= TIMING_SLOTS) return SSGD_OK;
+    CU(cudaEventRecord(x->ev[x->ev_steps * EV_PER_STEP + which], st), "event record");
+    return SSGD_OK;
+}
+
+int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, float* cand_est,
+                    float* est, cudaStream_t st, bool timed = false) {
+    UnsketchArgs A;
+    A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk; A.est = est;
+    SelBuffers sb = sel_buffers(x, false);
+    A.sb = sb; A.want = (uint32_t)ncand;
+    int e = launch_unsketch(x, A, st);
+    if (e) return e;
+    if (timed && (e = mark(x, 2, st))) return e;
+    if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st))) return e;
+    k_emit_candidates<<<(int)x->nchunk_c, SEL_THREADS, 0, st>>>(est, x->d, sb, cand_idx, cand_est);
+    LAUNCHED("k_emit_candidates");
+    return SSGD_OK;
+}
+
+int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
+                       cudaStream_t st) {
+    float* xs = reinterpret_cast<float*>(x->ws + x->off_xs);
+    int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
+    SelBuffers sb = sel_buffers(x, true);
+    const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
+    k_gather<<<grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, st>>>(cand, ncand, x->v, x->ld, x->W, x->d, xs,
+                                                                      sb, (uint32_t)x->k, err);
+    LAUNCHED("k_gather");
+    int e = launch_select(x, xs, ncand, sb, nch, st);
+    if (e) return e;
+    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand, out_idx, out_val);
+    LAUNCHED("k_emit_final");
+    k_zero<<<grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, st>>>(out_idx, x->k, x->u, x->v,
+                                                                                            x->ld, x->W, x->d);
+    LAUNCHED("k_zero");
+    return SSGD_OK;
+}
+
+int resolve_insert_mode(const ssgd_ctx* x) {
+    const size_t table_bytes = (size_t)x->r * x->c * 4;
+    const bool fits = table_bytes <= (size_t)200 * 1024 && (int64_t)table_bytes <= x->max_smem_optin;
+    if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
+    if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
+    return INS_MERGED_GLOBAL;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int32_t W, uint64_t seed) {
+    if (!out) return SSGD_EINVAL;
+    *out = nullptr;
+    if (d < 1 || d >= (int64_t)P31) return SSGD_EINVAL;
+    if (r < 1 || r > SSGD_MAX_R || (r % 2) == 0) return SSGD_EINVAL;
+    if (c < 1 || c >= (int64_t)P31) return SSGD_EINVAL;
+    if (k < 1 || k > d || W < 1) return SSGD_EINVAL;
+    ssgd_ctx* x = new (std::nothrow) ssgd_ctx();
+    if (!x) return SSGD_ENOMEM;
+    x->d = d; x->r = r; x->c = c; x->k = k; x->W = W; x->seed = seed;
+    std::memset(&x->hp, 0, sizeof(x->hp));
+    derive_params(seed, r, x->hp);
+    x->bk = make_bucketizer((uint64_t)c);
+    x->pow2 = (c & (c - 1)) == 0;
+    x->insert_mode = SSGD_INSERT_AUTO;
+    x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
+    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0;
+    *out = x;
+    return SSGD_OK;
+}
+
+int ssgd_destroy(ssgd_ctx* ctx) {
+    if (ctx && ctx->ev) {
+        for (int i = 0; i < TIMING_SLOTS * EV_PER_STEP; ++i) cudaEventDestroy(ctx->ev[i]);
+        delete[] ctx->ev;
+    }
+    delete ctx;
+    return SSGD_OK;
+}
+
+int ssgd_get_hash_params(const ssgd_ctx* x, uint32_t* out4r) {
+    if (!x || !out4r) return SSGD_EINVAL;
+    for (int j = 0; j < x->r; ++j) {
+        out4r[4 * j] = x->hp.row[j].a; out4r[4 * j + 1] = x->hp.row[j].b;
+        out4r[4 * j + 2] = x->hp.row[j].a2; out4r[4 * j + 3] = x->hp.row[j].b2;
+    }
+    return SSGD_OK;
+}
+
+int ssgd_set_hash_params(ssgd_ctx* x, const uint32_t* in4r) {
+    if (!x || !in4r) return SSGD_EINVAL;
+    for (int j = 0; j < x->r; ++j) {
+        if (in4r[4 * j] < 1 || in4r[4 * j] >= P31 || in4r[4 * j + 1] >= P31) return SSGD_EINVAL;
+        if (in4r[4 * j + 2] < 1 || in4r[4 * j + 2] >= P31 || in4r[4 * j + 3] >= P31) return SSGD_EINVAL;
+    }
+    for (int j = 0; j < x->r; ++j) {
+        x->hp.row[j].a = in4r[4 * j]; x->hp.row[j].b = in4r[4 * j + 1];
+        x->hp.row[j].a2 = in4r[4 * j + 2]; x->hp.row[j].b2 = in4r[4 * j + 3];
+    }
+    return SSGD_OK;
+}
+
+int ssgd_set_insert_mode(ssgd_ctx* x, int32_t mode) {
+    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_SMEM) return SSGD_EINVAL;
+    x->insert_mode = mode;
+    return SSGD_OK;
+}
+
+int ssgd_workspace_bytes(const ssgd_ctx* x, int64_t ncand_max, size_t* out_bytes) {
+    if (!x || !out_bytes || ncand_max < x->k || ncand_max > x->d) return SSGD_EINVAL;
+    ssgd_ctx tmp = *x;
+    layout(&tmp, ncand_max);
+    *out_bytes = tmp.total_bytes;
+    return SSGD_OK;
+}
+
+int ssgd_bind(ssgd_ctx* x, float* u, float* v, int64_t ld, void* workspace, size_t workspace_bytes,
+              int64_t ncand_max) {
+    if (!x || !u || !v || !workspace || ld < x->d) return SSGD_EINVAL;
+    if (ncand_max < x->k || ncand_max > x->d) return SSGD_EINVAL;
+    if (!aligned16(u) || !aligned16(v) || (ld & 3)) return SSGD_EALIGN;
+    if (reinterpret_cast<uintptr_t>(workspace) % ALIGN) return SSGD_EALIGN;
+    layout(x, ncand_max);
+    if (workspace_bytes < x->total_bytes) return SSGD_EWORKSPACE;
+    x->u = u; x->v = v; x->ld = ld;
+    x->ws = static_cast<char*>(workspace); x->ws_bytes = workspace_bytes; x->ncand_max = ncand_max;
+    int e = ensure_device(x);
+    if (e) return e;
+    CU(cudaMemset(x->ws + x->off_err, 0, 16), "clear error flag");
+    return SSGD_OK;
+}
+
+int ssgd_sketch_accumulate(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, float* tables, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if ((e = check_g(x, g, ld_g))) return e;
+    if (!tables) return SSGD_EINVAL;
+    if ((e = ensure_device(x))) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemsetAsync(tables, 0, (size_t)x->W * x->r * x->c * 4, st), "memset tables");
+    x->launches++;
+    AccumArgs A;
+    A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
+    A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
+    return launch_accum(x, A, INS_PER_WORKER, st);
+}
+
+int ssgd_sketch_merge(ssgd_ctx* x, const float* tables, float* merged, void* stream) {
+    if (!x || !tables || !merged) return SSGD_EINVAL;
+    const int64_t rc = (int64_t)x->r * x->c;
+    if ((rc & 3) == 0 && (!aligned16(tables) || !aligned16(merged))) return SSGD_EALIGN;
+    int e = ensure_device(x);
+    if (e) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    k_merge<<<grid_for((rc + 3) / 4, 256, (int64_t)x->sm_count * 16), 256, 0, st>>>(tables, merged, rc, x->W);
+    LAUNCHED("k_merge");
+    return SSGD_OK;
+}
+
+int ssgd_unsketch_candidates(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx,
+                             float* cand_est, float* est_all, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!merged || !cand_idx || ncand < x->k || ncand > x->d) return SSGD_EINVAL;
+    if (est_all && !aligned16(est_all)) return SSGD_EALIGN;
+    if ((e = ensure_device(x))) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->off_hist_f - x->off_hist_c, st), "memset hist");
+    x->launches++;
+    float* est = est_all ? est_all : reinterpret_cast<float*>(x->ws + x->off_est);
+    return unsketch_select(x, merged, ncand, cand_idx, cand_est, est, st);
+}
+
+int ssgd_exact_topk(ssgd_ctx* x, const int32_t* cand_idx, int64_t ncand, int32_t* out_idx, float* out_val,
+                    void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!cand_idx || !out_idx || !out_val || ncand < x->k || ncand > x->d) return SSGD_EINVAL;
+    if (ncand > x->ncand_max) return SSGD_EWORKSPACE;
+    if ((e = ensure_device(x))) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_err - x->off_hist_f, st), "memset hist");
+    x->launches++;
+    return gather_select_zero(x, cand_idx, ncand, out_idx, out_val, st);
+}
+
+int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncand, int32_t* out_idx,
+              float* out_val, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if ((e = check_g(x, g, ld_g))) return e;
+    if (!out_idx || !out_val || ncand < x->k || ncand > x->d) return SSGD_EINVAL;
+    if (ncand > x->ncand_max) return SSGD_EWORKSPACE;
+    if ((e = ensure_device(x))) return e;
+    const int mode = resolve_insert_mode(x);
+    if (mode < 0) return SSGD_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // table, histograms, selection state: one memset (the error flag is sticky until ssgd_status)
+    CU(cudaMemsetAsync(x->ws, 0, x->off_err, st), "memset workspace head");
+    x->launches++;
+    float* merged = reinterpret_cast<float*>(x->ws + x->off_table);
+    AccumArgs A;
+    A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
+    A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
+    if ((e = mark(x, 0, st))) return e;
+    if ((e = launch_accum(x, A, mode, st))) return e;
+    if ((e = mark(x, 1, st))) return e;
+    int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
+    float* est = reinterpret_cast<float*>(x->ws + x->off_est);
+    if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
+    if ((e = mark(x, 3, st))) return e;
+    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st))) return e;
+    if ((e = mark(x, 4, st))) return e;
+    if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
+    return SSGD_OK;
+}
+
+int ssgd_set_timing(ssgd_ctx* x, int32_t enable) {
+    if (!x) return SSGD_EINVAL;
+    if (enable && !x->ev) {
+        x->ev = new (std::nothrow) cudaEvent_t[TIMING_SLOTS * EV_PER_STEP];
+        if (!x->ev) return SSGD_ENOMEM;
+        for (int i = 0; i < TIMING_SLOTS * EV_PER_STEP; ++i) CU(cudaEventCreate(&x->ev[i]), "event create");
+    }
+    x->timing = enable != 0;
+    x->ev_steps = 0;
+    return SSGD_OK;
+}
+
+int ssgd_get_stage_times(ssgd_ctx* x, void* stream, double* ms_out, int64_t* steps_out) {
+    if (!x || !ms_out || !steps_out) return SSGD_EINVAL;
+    CU(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)), "stream synchronize");
+    for (int sgi = 0; sgi < SSGD_NSTAGES; ++sgi) ms_out[sgi] = 0.0;
+    for (int t = 0; t < x->ev_steps; ++t)
+        for (int sgi = 0; sgi < SSGD_NSTAGES; ++sgi) {
+            float ms = 0.f;
+            CU(cudaEventElapsedTime(&ms, x->ev[t * EV_PER_STEP + sgi], x->ev[t * EV_PER_STEP + sgi + 1]), "event elapsed");
+            ms_out[sgi] += ms;
+        }
+    *steps_out = x->ev_steps;
+    x->ev_steps = 0;
+    return SSGD_OK;
+}
+
+int ssgd_step_host(ssgd_ctx* x, const float* g_host, int64_t ld_g, float rho, int64_t ncand, float* g_stage,
+                   int32_t* out_idx_host, float* out_val_host, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!g_host || !g_stage || !out_idx_host || !out_val_host) return SSGD_EINVAL;
+    if ((e = check_g(x, g_stage, ld_g))) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpyAsync(g_stage, g_host, (size_t)x->W * ld_g * 4, cudaMemcpyHostToDevice, st), "copy g to device");
+    int32_t* oidx = reinterpret_cast<int32_t*>(x->ws + x->off_oidx);
+    float* oval = reinterpret_cast<float*>(x->ws + x->off_oval);
+    if ((e = ssgd_step(x, g_stage, ld_g, rho, ncand, oidx, oval, stream))) return e;
+    CU(cudaMemcpyAsync(out_idx_host, oidx, (size_t)x->k * 4, cudaMemcpyDeviceToHost, st), "copy out_idx to host");
+    CU(cudaMemcpyAsync(out_val_host, oval, (size_t)x->k * 4, cudaMemcpyDeviceToHost, st), "copy out_val to host");
+    CU(cudaStreamSynchronize(st), "stream synchronize");
+    return SSGD_OK;
+}
+
+int ssgd_step_buffers(const ssgd_ctx* x, const float** merged, const float** est, const int32_t** cand_idx,
+                      const float** cand_xs) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (merged) *merged = reinterpret_cast<const float*>(x->ws + x->off_table);
+    if (est) *est = reinterpret_cast<const float*>(x->ws + x->off_est);
+    if (cand_idx) *cand_idx = reinterpret_cast<const int32_t*>(x->ws + x->off_cand);
+    if (cand_xs) *cand_xs = reinterpret_cast<const float*>(x->ws + x->off_xs);
+    return SSGD_OK;
+}
+
+int ssgd_hashes(ssgd_ctx* x, const int32_t* idx, int64_t n, int32_t* h_out, int32_t* s_out, void* stream) {
+    if (!x || n < 0 || (n > 0 && (!idx || !h_out || !s_out))) return SSGD_EINVAL;
+    if (n == 0) return SSGD_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = grid_for(n, 256, (int64_t)1 << 30);
+    if (x->pow2) k_hashes<true><<<grid, 256, 0, st>>>(idx, n, x->r, x->hp, x->bk, h_out, s_out);
+    else k_hashes<false><<<grid, 256, 0, st>>>(idx, n, x->r, x->hp, x->bk, h_out, s_out);
+    LAUNCHED("k_hashes");
+    return SSGD_OK;
+}
+
+int ssgd_launch_count(const ssgd_ctx* x, int64_t* out) {
+    if (!x || !out) return SSGD_EINVAL;
+    *out = x->launches;
+    return SSGD_OK;
+}
+
+int ssgd_status(ssgd_ctx* x, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    CU(cudaStreamSynchronize(st), "stream synchronize");
+    int32_t flag = 0;
+    CU(cudaMemcpy(&flag, x->ws + x->off_err, 4, cudaMemcpyDeviceToHost), "read error flag");
+    if (flag) {
+        CU(cudaMemset(x->ws + x->off_err, 0, 4), "clear error flag");
+        return SSGD_EDEVICE;
+    }
+    return SSGD_OK;
+}
+
+const char* ssgd_strerror(int code) {
+    switch (code) {
+        case SSGD_OK: return "ok";
+        case SSGD_EINVAL: return "invalid argument";
+        case SSGD_EALIGN: return "pointer not 16-byte aligned or leading dimension not a multiple of 4";
+        case SSGD_ENOTBOUND: return "no state/workspace bound (call ssgd_bind)";
+        case SSGD_EWORKSPACE: return "workspace too small for this ncand";
+        case SSGD_ECUDA: return "CUDA runtime error (see ssgd_last_error)";
+        case SSGD_EDEVICE: return "a kernel reported an out-of-range index";
+        case SSGD_ENOMEM: return "out of host memory";
+        default: return "unknown error";
+    }
+}
+
+const char* ssgd_last_error(const ssgd_ctx* x) { return x ? x->last_error.c_str() : ""; }
+
+}  // extern "C"

@@ -1,0 +1,111 @@
+"""Staged parity protocol: one ssgd_step of the CUDA library against the CPU oracle.
+
+Both sides get the same g and start from bit-identical u, v.  Because reductions into the sketch
+happen in an unspecified order on the GPU, later stages are compared *conditionally*:
+
+  1. u, v after momentum/error accumulation ........ bit-exact (outside the zeroed coordinates)
+  2. merged table .................................. |S_gpu - T| <= 1e-5 * M per bucket, M = L1 mass of the bucket
+     estimates ..................................... |est_gpu - est| <= tau_i = 1e-5 * max_j M[j][h_j(i)]
+  3. candidates .................................... exactly the top-ncand of the GPU's own estimates
+                                                     (total order), and admissible w.r.t. the oracle:
+                                                     contains every i with |est_i| - tau_i above the highest
+                                                     possible threshold, none with |est_i| + tau_i below the lowest
+  4. final k ....................................... the oracle's lines 10-11 applied to the GPU's candidates:
+                                                     identical index set, identical values
+  5. zero-out ...................................... exactly the GPU's k coordinates, every worker, u and v, +0.0f
+  6. lock step ..................................... the oracle adopts the GPU's (admissible) selection, so both
+                                                     sides enter the next step with bit-identical state.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import select as oracle_select
+
+TABLE_RTOL = 1e-5   # relative to the L1 mass hashed into the bucket
+
+
+def bucket_tau(orc, M, idx=None, chunk=1 << 20):
+    """tau_i = TABLE_RTOL * max_j M[j][h_j(i)] for the listed coordinates (all if idx is None)."""
+    if idx is None:
+        idx = np.arange(orc.d, dtype=np.int64)
+    tau = np.zeros(idx.size)
+    for s in range(0, idx.size, chunk):
+        h, _ = orc.hashes(idx[s:s + chunk])
+        m = np.zeros(h.shape[1])
+        for j in range(orc.r):
+            m = np.maximum(m, M[j, h[j]])
+        tau[s:s + chunk] = TABLE_RTOL * m
+    return tau
+
+
+def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=None):
+    """Runs eng.step on g_dev and the oracle on the same g; asserts the protocol; adopts.
+
+    orc: oracle.Oracle; eng: bound Ssgd; u_o, v_o: the oracle's numpy state, bit-identical to the
+    engine's bound state on entry and again on exit.  Returns (out_idx, out_val) as numpy arrays."""
+    d, W, k = orc.d, orc.W, orc.k
+    dev = g_dev.device
+    out_idx = torch.empty(k, dtype=torch.int32, device=dev)
+    out_val = torch.empty(k, dtype=torch.float32, device=dev)
+    eng.step(g_dev, rho, ncand, out_idx, out_val)
+    assert eng.status() == 0
+    u_g, v_g, _ = eng._keep
+    merged_g, est_g, cand_g, xs_g = [t.cpu().numpy() for t in eng.step_buffers(ncand)]
+    out_idx_g, out_val_g = out_idx.cpu().numpy(), out_val.cpu().numpy()
+    u_g_h, v_g_h = u_g.cpu().numpy(), v_g.cpu().numpy()
+
+    # oracle, without its own zero-out
+    g_h = g_dev.cpu().numpy()
+    o = orc.step(g_h, rho, u_o, v_o, ncand, zero_state=False, full=True)
+
+    # 5 + 1: chosen coordinates are +0.0f everywhere, everything else equals the oracle bit for bit
+    assert len(np.unique(out_idx_g)) == k and out_idx_g.min() >= 0 and out_idx_g.max() < d
+    assert (np.diff(out_idx_g) > 0).all(), "out_idx must be ascending"
+    chosen = np.zeros(u_o.shape[1], bool)
+    chosen[out_idx_g] = True
+    for name, got, want in (("u", u_g_h, u_o), ("v", v_g_h, v_o)):
+        assert (got[:, chosen].view(np.uint32) == 0).all(), f"{name}: chosen coordinates must be +0.0f"
+        assert (got[:, ~chosen].view(np.uint32) == want[:, ~chosen].view(np.uint32)).all(), \
+            f"{name}: momentum/error accumulation is not bit-exact"
+
+    # 2: table and estimates
+    T, M = o["T"], o["M"]
+    err = np.abs(merged_g.astype(np.float64) - T)
+    assert (err <= TABLE_RTOL * M).all(), f"table: worst error/mass {np.max(err / np.maximum(M, 1e-300)):.3e}"
+    tau = None
+    if check_est:
+        tau = bucket_tau(orc, M)
+        e_err = np.abs(est_g.astype(np.float64) - o["est"].astype(np.float64))
+        assert (e_err <= tau).all(), "estimates outside tolerance"
+
+    # 3: candidates -- exact given the GPU's own estimates, admissible against the oracle's
+    assert (np.diff(cand_g) > 0).all(), "cand_idx must be ascending and distinct"
+    want_c = np.sort(oracle_select(est_g, ncand))
+    assert (cand_g == want_c).all(), "candidates are not the top-ncand of the GPU's estimates"
+    if check_est and ncand < d:
+        a = np.abs(o["est"].astype(np.float64))
+        hi = np.partition(a + tau, d - ncand)[d - ncand]   # ncand-th largest upper bound
+        lo = np.partition(a - tau, d - ncand)[d - ncand]   # ncand-th largest lower bound
+        inc = np.zeros(d, bool)
+        inc[cand_g] = True
+        assert inc[(a - tau) > hi].all(), "a coordinate surely above the threshold is missing"
+        assert not inc[(a + tau) < lo].any(), "a coordinate surely below the threshold was selected"
+    if report is not None:
+        report.append(dict(cand_sym_diff=int(np.setxor1d(cand_g, o["cand"]).size)))
+
+    # 4: final top-k -- the oracle's second round and top-k on the GPU's candidates
+    xs = orc.second_round(v_o, cand_g)
+    assert (xs_g == xs.astype(np.float32)).all(), "second-round sums differ"
+    want_idx, want_val = orc.final_topk(cand_g, xs)
+    order = np.argsort(want_idx)
+    assert (out_idx_g == want_idx[order]).all(), "final k-set differs from the oracle's on the same candidates"
+    assert (out_val_g.view(np.uint32) == want_val[order].view(np.uint32)).all(), "out_val differs"
+    if report is not None:
+        report[-1]["final_sym_diff_vs_unadopted"] = int(np.setxor1d(out_idx_g, o["out_idx"]).size)
+
+    # 6: adopt the GPU's selection
+    orc.zero(u_o, v_o, out_idx_g)
+    assert (u_g_h.view(np.uint32) == u_o.view(np.uint32)).all() and (v_g_h.view(np.uint32) == v_o.view(np.uint32)).all()
+    return out_idx_g, out_val_g

@@ -1,0 +1,302 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, stage by stage and as a
+whole step, on the same seeded inputs.  Integer work (hashes, signs, selections given their inputs,
+the zero-out mask, u and v) is compared bit for bit; the sketch table within 1e-5 of the L1 mass of
+each bucket, because the order of the reductions is not fixed."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import Oracle, select as oracle_select
+from paper_1903_04488_b200 import ssgd as S
+from paper_1903_04488_b200 import workloads as wl
+from tests.protocol import TABLE_RTOL, bucket_tau, check_step
+
+pytestmark = pytest.mark.gpu
+P = 2**31 - 1
+
+
+def make(cfg, dev, ncand_max=None, seed=None):
+    seed = cfg.sketch_seed if seed is None else seed
+    eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, seed)
+    orc = Oracle(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, seed)
+    u, v = wl.zero_state(cfg, dev)
+    eng.bind(u, v, ncand_max or cfg.ncand)
+    return eng, orc, u, v
+
+
+def random_state(cfg, dev, seed):
+    gen = torch.Generator(device=dev).manual_seed(seed)
+    u = torch.zeros((cfg.W, cfg.ld), device=dev)
+    v = torch.zeros((cfg.W, cfg.ld), device=dev)
+    u[:, :cfg.d] = torch.randn((cfg.W, cfg.d), generator=gen, device=dev)
+    v[:, :cfg.d] = torch.randn((cfg.W, cfg.d), generator=gen, device=dev)
+    return u, v
+
+
+# ------------------------------------------------------------------------------------------------
+# hashes and signs: bit-exact
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("c", [1, 2, 7, 40, 16384, 180000, 262144, 2**30, 2**31 - 2, 2**31 - 3])
+def test_hashes_bit_exact(cuda_device, c):
+    r, seed = 7, 1234 + c % 97
+    d = 2**31 - 2
+    eng = S.Ssgd(d, r, c, 1, 1, seed)
+    orc = Oracle(d, r, c, 1, 1, seed)
+    assert (eng.get_hash_params().numpy() == orc.params().astype(np.int64)).all()
+    rng = np.random.default_rng(c)
+    idx = np.concatenate([np.arange(0, 70000), [P - 2, P - 3, 2**30, 2**30 - 1, 2**30 + 1],
+                          rng.integers(0, P - 1, 200000)]).astype(np.int64)
+    h, s = eng.hashes(torch.tensor(idx, dtype=torch.int32, device=cuda_device))
+    ho, so = orc.hashes(idx)
+    assert (h.cpu().numpy() == ho).all() and (s.cpu().numpy() == so).all()
+
+
+def test_hashes_extreme_parameters(cuda_device):
+    d, c = 2**31 - 2, 1000003
+    for params in ([[P - 1, P - 1, P - 1, P - 1]] * 3, [[1, 0, 1, 0]] * 3, [[P - 1, 0, 1, P - 1]] * 3):
+        eng = S.Ssgd(d, 3, c, 1, 1, 0)
+        orc = Oracle(d, 3, c, 1, 1, 0)
+        eng.set_hash_params(params)
+        orc.set_params(params)
+        idx = np.array([0, 1, 2, P - 2, P - 3, 12345678], np.int64)
+        h, s = eng.hashes(torch.tensor(idx, dtype=torch.int32, device=cuda_device))
+        ho, so = orc.hashes(idx)
+        assert (h.cpu().numpy() == ho).all() and (s.cpu().numpy() == so).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# stage calls
+# ------------------------------------------------------------------------------------------------
+STAGE_CASES = [
+    wl.C2.scaled(d=100_003, W=3, c=1024, ncand=600, k=200),        # ragged d, several tiles
+    wl.C1.scaled(d=65_536, W=4, c=4096, ncand=400, k=200),
+    wl.C3.scaled(d=40_001, W=5, r=7, c=40, ncand=300, k=100),      # the paper's small sketch shape, c not 2^n
+    wl.C4.scaled(d=90_002, W=2, r=15, c=18_000, ncand=900, k=300), # r = 15 rows, c not a power of two
+    wl.C2.scaled(d=5, W=1, r=1, c=1, ncand=3, k=2),
+    wl.C2.scaled(d=4099, W=9, r=3, c=7, ncand=4099, k=4099),
+]
+
+
+@pytest.mark.parametrize("cfg", STAGE_CASES, ids=lambda c: f"{c.name}-d{c.d}-W{c.W}-r{c.r}-c{c.c}")
+def test_stage_calls_against_oracle(cuda_device, cfg):
+    dev = cuda_device
+    eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+    orc = Oracle(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+    u, v = random_state(cfg, dev, 7)
+    eng.bind(u, v, cfg.ncand)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    g = wl.gradients(wl.Structure(cfg, dev), 0)
+
+    # lines 5-7: u, v bit-exact; every worker's table within tolerance of its own bucket masses
+    tables = torch.full((cfg.W, cfg.r, cfg.c), 123.0, device=dev)   # the call must zero it
+    eng.sketch_accumulate(g, cfg.rho, tables)
+    orc.accumulate(g.cpu().numpy(), cfg.rho, u_o, v_o)
+    assert (u.cpu().numpy().view(np.uint32) == u_o.view(np.uint32)).all()
+    assert (v.cpu().numpy().view(np.uint32) == v_o.view(np.uint32)).all()
+    T, M, Tw = orc.sketch_workers(v_o, per_worker=True)
+    tables_h = tables.cpu().numpy().astype(np.float64)
+    for w in range(cfg.W):
+        Mw = orc.sketch(v_o[w, :cfg.d].copy(), with_mass=True)[1]
+        assert (np.abs(tables_h[w] - Tw[w]) <= TABLE_RTOL * Mw).all()
+
+    # line 8: merge in worker order -- reproduce it exactly from the GPU's own tables, then vs oracle
+    merged = torch.empty((cfg.r, cfg.c), device=dev)
+    eng.sketch_merge(tables, merged)
+    acc = np.zeros((cfg.r, cfg.c), np.float32)
+    for w in range(cfg.W):
+        acc = acc + tables.cpu().numpy()[w]
+    assert (merged.cpu().numpy() == acc).all()
+    assert (np.abs(merged.cpu().numpy().astype(np.float64) - T) <= TABLE_RTOL * M).all()
+
+    # line 9 on the ORACLE's table: estimates and candidates must then be identical
+    Tf = T.astype(np.float32)
+    cand = torch.empty(cfg.ncand, dtype=torch.int32, device=dev)
+    cand_est = torch.empty(cfg.ncand, device=dev)
+    est = torch.empty(cfg.d + 4, device=dev)[:cfg.d]
+    eng.unsketch_candidates(torch.tensor(Tf, device=dev), cfg.ncand, cand, cand_est, est)
+    est_o = orc.estimate(Tf)
+    assert (est.cpu().numpy() == est_o).all()
+    cand_o = np.sort(oracle_select(est_o, cfg.ncand))
+    assert (cand.cpu().numpy() == cand_o).all()
+    assert (cand_est.cpu().numpy() == est_o[cand_o]).all()
+
+    # lines 10, 11, 13 on those candidates
+    out_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    out_val = torch.empty(cfg.k, device=dev)
+    eng.exact_topk(cand, out_idx, out_val)
+    assert eng.status() == S.OK
+    xs = orc.second_round(v_o, cand_o)
+    want_idx, want_val = orc.final_topk(cand_o, xs)
+    order = np.argsort(want_idx)
+    assert (out_idx.cpu().numpy() == want_idx[order]).all()
+    assert (out_val.cpu().numpy().view(np.uint32) == want_val[order].view(np.uint32)).all()
+    orc.zero(u_o, v_o, want_idx)
+    assert (u.cpu().numpy().view(np.uint32) == u_o.view(np.uint32)).all()
+    assert (v.cpu().numpy().view(np.uint32) == v_o.view(np.uint32)).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# whole step, lock step with the oracle over several steps
+# ------------------------------------------------------------------------------------------------
+STEP_CASES = [
+    (wl.C1.scaled(d=131_072, c=4096, ncand=500, k=250), 1),
+    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), 4),
+    (wl.C3.scaled(d=200_003, W=6, c=16_384, ncand=2000, k=1000), 3),
+    (wl.C4.scaled(d=270_002, W=3, c=32_768, ncand=1500, k=700), 3),
+    (wl.C2.scaled(d=50_001, W=2, r=7, c=40, ncand=500, k=10), 3),          # r=7, c=40 (MNIST shape)
+    (wl.C3.scaled(d=60_000, W=3, r=15, c=1800, ncand=1600, k=100), 2),     # r=15, P=16
+    (wl.C2.scaled(d=70_001, W=17, r=3, c=999, ncand=300, k=300), 2),       # k == ncand, odd W
+    (wl.C2.scaled(d=20_000, W=1, r=1, c=64, ncand=20_000, k=50), 2),       # ncand == d: true top-k
+    (wl.C1.scaled(d=3, W=2, r=5, c=16, ncand=2, k=1), 2),                  # d < 4
+]
+
+
+@pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
+@pytest.mark.parametrize("mode", [S.INSERT_GLOBAL, S.INSERT_SMEM])
+def test_step_lockstep(cuda_device, cfg, steps, mode):
+    if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
+        pytest.skip("table does not fit the shared-memory variant")
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_insert_mode(mode)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    report = []
+    for t in range(steps):
+        g = wl.gradients(st, t)
+        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report)
+    if cfg.ncand == cfg.d:
+        assert all(r["final_sym_diff_vs_unadopted"] == 0 for r in report)
+
+
+def test_all_zero_gradient_ties_break_by_index(cuda_device):
+    cfg = wl.C2.scaled(d=10_001, W=3, c=256, ncand=700, k=300)
+    eng, orc, u, v = make(cfg, cuda_device)
+    g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
+    assert idx.tolist() == list(range(cfg.k)) and (val == 0).all()
+
+
+def test_heavy_ties_at_the_threshold(cuda_device):
+    """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
+    cfg = wl.C2.scaled(d=40_000, W=2, r=1, c=40_000, ncand=1000, k=400)
+    eng, orc, u, v = make(cfg, cuda_device)
+    ident = [[1, 0, 1, 0]]
+    eng.set_hash_params(ident)
+    orc.set_params(ident)          # table = signed copy of the summed vector: estimates are exact
+    g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
+    g[:, 5:30_000:7] = 1.0         # 4286 coordinates tie at |x| = 2
+    g[:, 11:500:13] = 3.0          # 38 coordinates above them
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
+    big = set(range(11, 500, 13))
+    assert big <= set(idx.tolist())
+
+
+def test_planted_heavy_coordinates_recovered(cuda_device):
+    cfg = wl.C1.scaled(d=262_144, c=8192, ncand=512, k=256)
+    eng, orc, u, v = make(cfg, cuda_device)
+    st = wl.Structure(cfg, cuda_device)
+    g = wl.gradients(st, 0)
+    # make the planted coordinates dominate: 5000 x the median instead of 50 x
+    g[:, st.planted_idx] *= 100.0
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    idx, _ = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
+    assert set(st.planted_idx.cpu().tolist()) <= set(idx.tolist())
+
+
+def test_fused_step_equals_stage_pipeline_selection(cuda_device):
+    """ssgd_step (sum over workers before the insert) and the faithful pipeline (per-worker tables,
+    merge) agree on u, v exactly and on the table within tolerance."""
+    cfg = wl.C2.scaled(d=150_001, W=8, c=4096, ncand=1200, k=600)
+    dev = cuda_device
+    g = wl.gradients(wl.Structure(cfg, dev), 0)
+    eng, orc, u, v = make(cfg, dev)
+    out_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    out_val = torch.empty(cfg.k, device=dev)
+    eng.step(g, cfg.rho, cfg.ncand, out_idx, out_val)
+    merged_fused = eng.step_buffers(cfg.ncand)[0].clone()
+    eng2, _, u2, v2 = make(cfg, dev)
+    tables = torch.empty((cfg.W, cfg.r, cfg.c), device=dev)
+    merged = torch.empty((cfg.r, cfg.c), device=dev)
+    eng2.sketch_accumulate(g, cfg.rho, tables)
+    eng2.sketch_merge(tables, merged)
+    T, M = orc.sketch_workers(v2.cpu().numpy())
+    for m in (merged_fused, merged):
+        assert (np.abs(m.cpu().numpy().astype(np.float64) - T) <= TABLE_RTOL * M).all()
+    cand = torch.empty(cfg.ncand, dtype=torch.int32, device=dev)
+    eng2.unsketch_candidates(merged, cfg.ncand, cand)
+    o_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    o_val = torch.empty(cfg.k, device=dev)
+    eng2.exact_topk(cand, o_idx, o_val)
+    assert eng2.status() == S.OK and eng.status() == S.OK
+    # the heavy part of the selection is common to both
+    common = np.intersect1d(out_idx.cpu().numpy(), o_idx.cpu().numpy()).size
+    assert common >= 0.95 * cfg.k
+
+
+def test_step_host_matches_step(cuda_device):
+    cfg = wl.C2.scaled(d=120_002, W=4, c=4096, ncand=900, k=300)
+    dev = cuda_device
+    g = wl.gradients(wl.Structure(cfg, dev), 0)
+    eng, _, u, v = make(cfg, dev)
+    out_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    out_val = torch.empty(cfg.k, device=dev)
+    eng.step(g, cfg.rho, cfg.ncand, out_idx, out_val)
+    eng2, _, u2, v2 = make(cfg, dev)
+    g_host = g.cpu().pin_memory()
+    stage = torch.empty_like(g)
+    oi = torch.empty(cfg.k, dtype=torch.int32).pin_memory()
+    ov = torch.empty(cfg.k, dtype=torch.float32).pin_memory()
+    eng2.step_host(g_host, cfg.rho, cfg.ncand, stage, oi, ov)
+    assert (u2 == u).all() and (v2 == v).all()
+    # same table up to reduction order -> the selections agree except near ties; values of common ones match
+    a, b = out_idx.cpu().numpy(), oi.numpy()
+    common, ia, ib = np.intersect1d(a, b, return_indices=True)
+    assert common.size >= 0.98 * cfg.k
+    assert (out_val.cpu().numpy()[ia] == ov.numpy()[ib]).all()
+
+
+# ------------------------------------------------------------------------------------------------
+# argument checking (host side; nothing is launched)
+# ------------------------------------------------------------------------------------------------
+def test_argument_errors(cuda_device):
+    dev = cuda_device
+    cfg = wl.C2.scaled(d=1000, W=2, c=64, ncand=100, k=50)
+    eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, 1)
+    g = torch.zeros((cfg.W, cfg.ld), device=dev)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    ov = torch.empty(cfg.k, device=dev)
+    with pytest.raises(S.SsgdError) as e:
+        eng.step(g, 0.9, cfg.ncand, oi, ov)
+    assert e.value.code == S.ENOTBOUND
+    u, v = wl.zero_state(cfg, dev)
+    small = torch.empty(16, dtype=torch.uint8, device=dev)
+    with pytest.raises(S.SsgdError) as e:
+        eng.bind(u, v, cfg.ncand, small)
+    assert e.value.code == S.EWORKSPACE
+    big = torch.empty(cfg.W * cfg.ld + 1, device=dev)
+    with pytest.raises(S.SsgdError) as e:
+        eng.bind(big[1:].view(cfg.W, cfg.ld), v, cfg.ncand)
+    assert e.value.code == S.EALIGN
+    eng.bind(u, v, cfg.ncand)
+    for ncand, code in ((cfg.k - 1, S.EINVAL), (cfg.d + 1, S.EINVAL), (cfg.ncand + 1, S.EWORKSPACE)):
+        with pytest.raises(S.SsgdError) as e:
+            eng.step(g, 0.9, ncand, oi, ov)
+        assert e.value.code == code
+    with pytest.raises(S.SsgdError) as e:
+        eng.step(big[1:].view(cfg.W, cfg.ld), 0.9, cfg.ncand, oi, ov)
+    assert e.value.code == S.EALIGN
+    g_short = torch.zeros((cfg.W, cfg.d - 8), device=dev)
+    with pytest.raises(S.SsgdError) as e:
+        eng.step(g_short, 0.9, cfg.ncand, oi, ov)
+    assert e.value.code == S.EINVAL
+    with pytest.raises(S.SsgdError):
+        eng.set_insert_mode(7)
+    # an out-of-range candidate is skipped and reported, never dereferenced
+    cand = torch.arange(cfg.ncand, dtype=torch.int32, device=dev)
+    cand[3] = cfg.d + 5
+    eng.exact_topk(cand, oi, ov)
+    assert eng.status() == S.EDEVICE
+    assert eng.status() == S.OK
+    assert eng.launch_count() > 0
