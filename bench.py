@@ -201,7 +201,7 @@ def run_ours(args, cfg):
     # replicas differ only in their seeds
     rcfg = cfg.scaled(base_seed=cfg.base_seed + 100 * rank)
     st = wl.Structure(rcfg, dev)
-    n_sets = cfg.steps
+    n_sets = args.sets or cfg.steps
     g_sets = [wl.gradients(st, t) for t in range(n_sets)]
     u, v = wl.zero_state(cfg, dev)
     eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
@@ -241,13 +241,13 @@ def run_ours(args, cfg):
     value = world * cfg.W * cfg.d / (ms_step * 1e-3)
 
     # ---- end to end: host gradients in, host results out, through ssgd_step_host ------------------
-    e2e_steps = max(1, min(args.steps, 20))
-    g_host = [g_sets[i].cpu().pin_memory() for i in range(2)]
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
+    g_host = [g_sets[i % n_sets].cpu().pin_memory() for i in range(2 if e2e_steps else 0)]
     g_stage = torch.empty_like(g_sets[0])
     oi_h = torch.empty(cfg.k, dtype=torch.int32).pin_memory()
     ov_h = torch.empty(cfg.k, dtype=torch.float32).pin_memory()
     u.zero_(); v.zero_()
-    for t in range(2):
+    for t in range(2 if e2e_steps else 0):
         eng.step_host(g_host[t % 2], cfg.rho, cfg.ncand, g_stage, oi_h, ov_h)
     u.zero_(); v.zero_()
     barrier(); torch.cuda.synchronize()
@@ -262,7 +262,7 @@ def run_ours(args, cfg):
         tmax = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         e2e_ms = float(tmax.item())
-    e2e_value = world * cfg.W * cfg.d / (e2e_ms / e2e_steps * 1e-3)
+    e2e_value = world * cfg.W * cfg.d / (e2e_ms / e2e_steps * 1e-3) if e2e_steps else None
 
     # ---- roofline of the dominant kernel and of the whole step -----------------------------------
     peak, peak_kind = peaks()
@@ -286,7 +286,7 @@ def run_ours(args, cfg):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": workload_config(cfg, args),
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": cfg.W * cfg.ld * 4,
-                "d2h_bytes_per_step": 8 * cfg.k, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps},
+                "d2h_bytes_per_step": 8 * cfg.k, "steps": e2e_steps, "ms_per_step": e2e_ms / max(1, e2e_steps)},
         "roofline": roofline,
         "step_hbm": {"algorithmic_bytes_per_step": step_bytes, "achieved": step_gbs, "peak": peak, "unit": "GB/s",
                      "frac": step_gbs / peak, "peak_source": f"of {peak_kind}", "frac_of_8000_nominal": step_gbs / 8000.0},
@@ -315,9 +315,14 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="C2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--d", type=int, default=0, help="override the number of coordinates (small profiling cases)")
+    ap.add_argument("--sets", type=int, default=0, help="resident gradient sets (default: the workload's steps)")
     args = ap.parse_args()
     from paper_1903_04488_b200 import workloads as wl
     cfg = wl.CONFIGS[args.workload]
+    if args.d:
+        cfg = cfg.scaled(name=f"{cfg.name}[d={args.d}]", d=args.d)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

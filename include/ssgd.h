@@ -53,15 +53,16 @@ extern "C" {
 #define SSGD_ENOTBOUND  -3  /* ssgd_bind has not been called                                           */
 #define SSGD_EWORKSPACE -4  /* workspace too small for the requested ncand                             */
 #define SSGD_ECUDA      -5  /* a CUDA runtime call failed; ssgd_last_error gives its text              */
-#define SSGD_EDEVICE    -6  /* a kernel recorded an error (index out of range in a caller's list)      */
+#define SSGD_EDEVICE    -6  /* a kernel recorded an error: bad index in a caller's list, or a wait gave up */
 #define SSGD_ENOMEM     -7  /* host allocation failed                                                  */
 
 #define SSGD_MAX_R 15
 
 /* Insert variants of ssgd_step (ssgd_set_insert_mode) */
-#define SSGD_INSERT_AUTO   0
-#define SSGD_INSERT_GLOBAL 1  /* reductions straight into the L2-resident r x c table                   */
+#define SSGD_INSERT_AUTO   0  /* = SSGD_INSERT_TMA                                                      */
+#define SSGD_INSERT_GLOBAL 1  /* plain 128-bit loads; reductions straight into the L2-resident table    */
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
+#define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
 
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
 

@@ -1,0 +1,217 @@
+// accum_tma.cuh -- the streaming form of Algorithm 3 lines 5-7 used by ssgd_step on sm_100a.
+//
+// One persistent CTA owns tiles of KT_TC consecutive coordinates.  For a tile it walks the W workers;
+// each (tile, worker) is one pipeline stage: three bulk asynchronous copies (cp.async.bulk, the TMA
+// engine) bring that worker's g, u and v slices into a ring of shared-memory slots, completion is
+// signalled on an mbarrier.  A dedicated producer warp keeps the ring full, so the bytes in flight do
+// not depend on what the consumer warps are doing; eight consumer warps take a slot, compute
+//     u' = fma(rho, u, g),  v' = v + u',  x += v'        (x: sum over workers, in worker order)
+// write u', v' straight back to global memory (coalesced 128-bit stores) and release the slot.
+// After the last worker each consumer thread hashes its four coordinates and issues the r reductions
+// per coordinate into the L2-resident merged table (sum_w S(v_w) = S(sum_w v_w), Section 3).
+// Several CTAs share an SM, so one CTA's reduction phase overlaps the others' streaming.
+//
+// Every mbarrier wait is bounded: after KT_WAIT_NS nanoseconds the waiter records ERR_TIMEOUT in the
+// error word, raises the CTA's abort flag and leaves; the producer then waits (bounded again) for the
+// copies it still has in flight before the CTA exits.
+#pragma once
+#include <stdint.h>
+
+#include "hash.cuh"
+
+namespace ssgd {
+
+constexpr int ERR_BAD_INDEX = 1;
+constexpr int ERR_TIMEOUT = 2;
+
+struct AccumArgs {
+    const float* g; int64_t ld_g;
+    float* u; float* v; int64_t ld;
+    int32_t W; int64_t d; float rho;
+    float* table;        // merged [r][c], or per-worker [W][r][c]
+    int64_t c;
+    HashParams hp; Bucketizer bk;
+};
+
+#ifndef SSGD_KT_STAGES
+#define SSGD_KT_STAGES 6
+#endif
+constexpr int KT_CONSUMER_WARPS = 8;
+constexpr int KT_CONSUMERS = KT_CONSUMER_WARPS * 32;
+constexpr int KT_THREADS = KT_CONSUMERS + 32;       // + one producer warp
+constexpr int KT_TC = KT_CONSUMERS * 4;             // coordinates per tile: one float4 per consumer thread
+constexpr int KT_STAGES = SSGD_KT_STAGES;
+constexpr uint64_t KT_WAIT_NS = 2000000000ull;      // a wait gives up after two seconds
+
+struct alignas(128) KtSlot { float g[KT_TC]; float u[KT_TC]; float v[KT_TC]; };
+struct KtShared {
+    KtSlot slot[KT_STAGES];
+    uint64_t full[KT_STAGES];
+    uint64_t empty[KT_STAGES];
+    volatile int abort;
+};
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void red_add(float* addr, float x) {
+    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(x) : "memory");
+}
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait; false if it gave up (KT_WAIT_NS elapsed) or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*abort || global_ns() - t0 > KT_WAIT_NS) return false;
+            __nanosleep(64);
+        }
+    }
+}
+__device__ __forceinline__ uint64_t policy_evict_first() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+// global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+}
+
+template <int R, bool POW2>
+__global__ void __launch_bounds__(KT_THREADS)
+k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
+    extern __shared__ __align__(128) unsigned char kt_raw[];
+    KtShared& S = *reinterpret_cast<KtShared*>(kt_raw);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int64_t d_main = A.d & ~(int64_t)3;                      // bulk copies cover whole float4 groups
+    const int64_t ntiles = (d_main + KT_TC - 1) / KT_TC;
+
+    if (tid == 0) {
+        for (int s = 0; s < KT_STAGES; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], KT_CONSUMER_WARPS); }
+        S.abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == KT_CONSUMER_WARPS) {
+        // ---------------- producer warp: one thread feeds the ring ----------------
+        if (lane == 0) {
+            const uint64_t pol = policy_evict_first();
+            uint32_t n = 0;
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+                const int64_t i0 = tile * KT_TC;
+                const uint32_t bytes = (uint32_t)((d_main - i0 < KT_TC ? d_main - i0 : KT_TC) * 4);
+                for (int w = 0; w < A.W; ++w, ++n) {
+                    const int s = n % KT_STAGES;
+                    if (n >= KT_STAGES && !mbar_wait(&S.empty[s], ((n / KT_STAGES) - 1) & 1, &S.abort)) { ok = false; break; }
+                    mbar_expect_tx(&S.full[s], 3 * bytes);
+                    bulk_load(S.slot[s].g, A.g + (int64_t)w * A.ld_g + i0, bytes, &S.full[s], pol);
+                    bulk_load(S.slot[s].u, A.u + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
+                    bulk_load(S.slot[s].v, A.v + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
+                }
+            }
+            if (!ok) {
+                // give up: report, tell the consumers, and let the copies already issued land before exit
+                atomicExch(errflag, ERR_TIMEOUT);
+                S.abort = 1;
+                const uint32_t first = n > KT_STAGES ? n - KT_STAGES : 0;
+                for (uint32_t m = first; m < n; ++m) {
+                    uint64_t* bar = &S.full[m % KT_STAGES];
+                    const uint64_t t0 = global_ns();
+                    while (!mbar_try_wait(bar, (m / KT_STAGES) & 1) && global_ns() - t0 < KT_WAIT_NS) __nanosleep(64);
+                }
+            }
+        }
+    } else {
+        // ---------------- consumer warps ----------------
+        uint32_t n = 0;
+        bool ok = true;
+        for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            const int64_t i0 = tile * KT_TC + 4 * tid;
+            const bool active = i0 < d_main;
+            float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;   // sum over workers of the new v, worker order
+            for (int w = 0; w < A.W; ++w, ++n) {
+                const int s = n % KT_STAGES;
+                if (!mbar_wait(&S.full[s], (n / KT_STAGES) & 1, &S.abort)) { ok = false; break; }
+                if (active) {
+                    const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[4 * tid]);
+                    const float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * tid]);
+                    const float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * tid]);
+                    float4 un, vn;
+                    un.x = __fmaf_rn(A.rho, u4.x, g4.x); vn.x = __fadd_rn(v4.x, un.x);
+                    un.y = __fmaf_rn(A.rho, u4.y, g4.y); vn.y = __fadd_rn(v4.y, un.y);
+                    un.z = __fmaf_rn(A.rho, u4.z, g4.z); vn.z = __fadd_rn(v4.z, un.z);
+                    un.w = __fmaf_rn(A.rho, u4.w, g4.w); vn.w = __fadd_rn(v4.w, un.w);
+                    __stcs(reinterpret_cast<float4*>(A.u + (int64_t)w * A.ld + i0), un);
+                    __stcs(reinterpret_cast<float4*>(A.v + (int64_t)w * A.ld + i0), vn);
+                    x0 = __fadd_rn(x0, vn.x); x1 = __fadd_rn(x1, vn.y);
+                    x2 = __fadd_rn(x2, vn.z); x3 = __fadd_rn(x3, vn.w);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S.empty[s]);
+            }
+            if (!ok) break;
+            if (active) {
+                const float x[4] = {x0, x1, x2, x3};
+#pragma unroll
+                for (int j = 0; j < R; ++j) {
+                    uint32_t hb[4];
+                    row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (x[e] != 0.0f) red_add(A.table + (int64_t)j * A.c + (hb[e] & P31), apply_sign(x[e], hb[e]));
+                }
+            }
+        }
+        if (!ok && lane == 0) { atomicExch(errflag, ERR_TIMEOUT); S.abort = 1; }
+        // ragged tail (d not a multiple of 4): at most three coordinates, plain loads, one thread
+        if (ok && blockIdx.x == 0 && tid == 0) {
+            for (int64_t i = d_main; i < A.d; ++i) {
+                float x = 0.f;
+                for (int64_t w = 0; w < A.W; ++w) {
+                    const float un = __fmaf_rn(A.rho, A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
+                    const float vn = __fadd_rn(A.v[w * A.ld + i], un);
+                    A.u[w * A.ld + i] = un;
+                    A.v[w * A.ld + i] = vn;
+                    x = __fadd_rn(x, vn);
+                }
+                for (int j = 0; j < R; ++j) {
+                    uint32_t hb[1];
+                    row_hashes<POW2, 1>(A.hp.row[j], A.bk, (uint32_t)i, hb);
+                    if (x != 0.0f) red_add(A.table + (int64_t)j * A.c + (hb[0] & P31), apply_sign(x, hb[0]));
+                }
+            }
+        }
+    }
+}
+
+#endif  // __CUDACC__
+}  // namespace ssgd

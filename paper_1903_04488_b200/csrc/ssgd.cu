@@ -24,37 +24,28 @@
 #include "../../include/ssgd.h"
 #include "hash.cuh"
 #include "select.cuh"
+#include "accum_tma.cuh"
 
 namespace ssgd {
 
 // ------------------------------------------------------------------------------------------------
-// small device helpers
+// K1 (plain-load form): momentum + error accumulation + sketch insert.  ssgd_step uses the bulk-copy
+// pipeline of accum_tma.cuh; this form serves the per-worker tables of ssgd_sketch_accumulate and the
+// shared-memory table variant.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void red_add(float* addr, float x) {
-    asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(x) : "memory");
-}
+enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
 
-constexpr int ERR_BAD_INDEX = 1;
-
-// ------------------------------------------------------------------------------------------------
-// K1: momentum + error accumulation + sketch insert
-// ------------------------------------------------------------------------------------------------
-enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2 };
-
-struct AccumArgs {
-    const float* g; int64_t ld_g;
-    float* u; float* v; int64_t ld;
-    int32_t W; int64_t d; float rho;
-    float* table;        // merged [r][c], or per-worker [W][r][c]
-    int64_t c;
-    HashParams hp; Bucketizer bk;
-};
-
+#ifndef SSGD_K1_UNROLL
+#define SSGD_K1_UNROLL 4
+#endif
+#ifndef SSGD_K1_MINBLOCKS
+#define SSGD_K1_MINBLOCKS 1
+#endif
 constexpr int K1_THREADS = 256;
-constexpr int K1_UNROLL = 4;  // workers in flight per thread: 3 x 16 B loads each
+constexpr int K1_UNROLL = SSGD_K1_UNROLL;  // workers in flight per thread: 3 x 16 B loads each
 
 template <int R, bool POW2, int MODE>
-__global__ void __launch_bounds__(K1_THREADS)
+__global__ void __launch_bounds__(K1_THREADS, SSGD_K1_MINBLOCKS)
 k_accum_insert(const AccumArgs A) {
     extern __shared__ float s_table[];  // MODE == INS_MERGED_SMEM: [R][c]
     const int64_t rc = (int64_t)R * A.c;
@@ -143,7 +134,11 @@ k_accum_insert(const AccumArgs A) {
                     if (i0 + e < A.d && x[e] != 0.0f) {
                         const float sx = apply_sign(x[e], h1[e]);
                         if (MODE == INS_MERGED_SMEM) atomicAdd(&s_table[(int64_t)j * A.c + (h1[e] & P31)], sx);
+#ifndef SSGD_EXP_NOATOMICS
                         else red_add(A.table + (int64_t)j * A.c + (h1[e] & P31), sx);
+#else
+                        else if (sx == 1.2345e-30f) A.table[0] = sx;
+#endif
                     }
                 }
             }
@@ -231,7 +226,24 @@ struct UnsketchArgs {
     uint32_t want;       // ncand
 };
 
+#ifndef SSGD_K3_NC
+#define SSGD_K3_NC 4
+#endif
+#ifndef SSGD_K3_LOAD
+#define SSGD_K3_LOAD 0
+#endif
 constexpr int K3_THREADS = 256;
+constexpr int K3_NC = SSGD_K3_NC;  // consecutive coordinates per thread (multiple of 4)
+
+__device__ __forceinline__ float table_load(const float* p) {
+#if SSGD_K3_LOAD == 0
+    return __ldg(p);
+#elif SSGD_K3_LOAD == 1
+    return __ldcg(p);
+#else
+    return *p;
+#endif
+}
 
 template <int R, bool POW2>
 __global__ void __launch_bounds__(K3_THREADS)
@@ -240,28 +252,32 @@ k_unsketch(const UnsketchArgs A) {
     uint32_t* s_hist = sh.hist;
     for (int b = threadIdx.x; b < H1_BINS; b += K3_THREADS) s_hist[b] = 0;
     __syncthreads();
-    const int64_t groups = (A.d + 3) >> 2;
+    const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     const int64_t stride = (int64_t)gridDim.x * K3_THREADS;
     for (int64_t q = (int64_t)blockIdx.x * K3_THREADS + threadIdx.x; q < groups; q += stride) {
-        const int64_t i0 = q << 2;
-        float rowv[4][R];
+        const int64_t i0 = q * K3_NC;
+        float rowv[K3_NC][R];
 #pragma unroll
         for (int j = 0; j < R; ++j) {
-            uint32_t hb[4];
-            row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+            uint32_t hb[K3_NC];
+            row_hashes<POW2, K3_NC>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-                rowv[e][j] = apply_sign(__ldg(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
+            for (int e = 0; e < K3_NC; ++e)
+                rowv[e][j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
         }
-        float m[4];
+        float m[K3_NC];
 #pragma unroll
-        for (int e = 0; e < 4; ++e) m[e] = median_of<R>(rowv[e]);
-        if (i0 + 3 < A.d) {
-            *reinterpret_cast<float4*>(A.est + i0) = make_float4(m[0], m[1], m[2], m[3]);
+        for (int e = 0; e < K3_NC; ++e) m[e] = median_of<R>(rowv[e]);
+        if (i0 + K3_NC - 1 < A.d) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
+            for (int e = 0; e < K3_NC; e += 4)
+                *reinterpret_cast<float4*>(A.est + i0 + e) = make_float4(m[e], m[e + 1], m[e + 2], m[e + 3]);
+#ifndef SSGD_EXP_NOHIST
+#pragma unroll
+            for (int e = 0; e < K3_NC; ++e) atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
+#endif
         } else {
-            for (int e = 0; e < 4 && i0 + e < A.d; ++e) {
+            for (int e = 0; e < K3_NC && i0 + e < A.d; ++e) {
                 A.est[i0 + e] = m[e];
                 atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
             }
@@ -277,8 +293,9 @@ k_unsketch(const UnsketchArgs A) {
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32_t* __restrict__ cand_idx,
-                  float* __restrict__ cand_est) {
+                  float* __restrict__ cand_est, uint32_t cap) {
     sel_emit_chunk(est, d, sb, [&](uint32_t slot, int64_t i) {
+        if (slot >= cap) return;  // cannot happen with consistent histograms; never write past the list
         cand_idx[slot] = (int32_t)i;
         if (cand_est) cand_est[slot] = est[i];
     });
@@ -327,8 +344,9 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const int32_t* __restrict__ cand,
-             int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
+             int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap) {
     sel_emit_chunk(xs, ncand, sb, [&](uint32_t slot, int64_t m) {
+        if (slot >= cap) return;
         out_idx[slot] = cand[m];
         out_val[slot] = xs[m];
     });
@@ -391,6 +409,7 @@ struct ssgd_ctx {
     int64_t nchunk_c, nchunk_f;
     // device facts
     int device; int sm_count; int max_smem_optin;
+    int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
     int64_t launches;
     // optional per-stage timing of ssgd_step (CUDA events on the caller's stream)
     bool timing;
@@ -520,6 +539,11 @@ int launch_accum_m(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
     }
 }
 
+#ifdef SSGD_EXP_ONLY_R5
+#define DISPATCH_R(fn, ...)                                                       \
+    if (x->r == 5 && x->pow2) return fn<5, true>(__VA_ARGS__);                    \
+    return SSGD_EINVAL;
+#else
 #define DISPATCH_R(fn, ...)                                                       \
     switch (x->r) {                                                               \
         case 1: return x->pow2 ? fn<1, true>(__VA_ARGS__) : fn<1, false>(__VA_ARGS__);    \
@@ -532,14 +556,36 @@ int launch_accum_m(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
         case 15: return x->pow2 ? fn<15, true>(__VA_ARGS__) : fn<15, false>(__VA_ARGS__); \
         default: return SSGD_EINVAL;                                              \
     }
+#endif
 
 int launch_accum(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
     DISPATCH_R(launch_accum_m, x, A, mode, st)
 }
 
 template <int R, bool POW2>
+int launch_accum_tma_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
+    auto kern = k_accum_insert_tma<R, POW2>;
+    const size_t smem = sizeof(KtShared);
+    if (x->kt_blocks_per_sm == 0) {
+        CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "smem attribute");
+        int nb = 0;
+        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, KT_THREADS, smem), "occupancy query");
+        x->kt_blocks_per_sm = nb < 1 ? 1 : nb;
+    }
+    const int64_t ntiles = ((A.d & ~(int64_t)3) + KT_TC - 1) / KT_TC;
+    const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->kt_blocks_per_sm);
+    kern<<<grid, KT_THREADS, smem, st>>>(A, reinterpret_cast<int32_t*>(x->ws + x->off_err));
+    LAUNCHED("k_accum_insert_tma");
+    return SSGD_OK;
+}
+
+int launch_accum_tma(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_accum_tma_t, x, A, st)
+}
+
+template <int R, bool POW2>
 int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
-    const int64_t groups = (A.d + 3) / 4;
+    const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     // a few blocks per SM: each block pays one histogram flush
     const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * 8);
     k_unsketch<R, POW2><<<grid, K3_THREADS, 0, st>>>(A);
@@ -596,7 +642,7 @@ int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* ca
     if (e) return e;
     if (timed && (e = mark(x, 2, st))) return e;
     if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st))) return e;
-    k_emit_candidates<<<(int)x->nchunk_c, SEL_THREADS, 0, st>>>(est, x->d, sb, cand_idx, cand_est);
+    k_emit_candidates<<<(int)x->nchunk_c, SEL_THREADS, 0, st>>>(est, x->d, sb, cand_idx, cand_est, (uint32_t)ncand);
     LAUNCHED("k_emit_candidates");
     return SSGD_OK;
 }
@@ -612,7 +658,7 @@ int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t*
     LAUNCHED("k_gather");
     int e = launch_select(x, xs, ncand, sb, nch, st);
     if (e) return e;
-    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand, out_idx, out_val);
+    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand, out_idx, out_val, (uint32_t)x->k);
     LAUNCHED("k_emit_final");
     k_zero<<<grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, st>>>(out_idx, x->k, x->u, x->v,
                                                                                             x->ld, x->W, x->d);
@@ -625,7 +671,7 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     const bool fits = table_bytes <= (size_t)200 * 1024 && (int64_t)table_bytes <= x->max_smem_optin;
     if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
     if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
-    return INS_MERGED_GLOBAL;
+    return INS_MERGED_TMA;
 }
 
 }  // namespace
@@ -648,7 +694,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->pow2 = (c & (c - 1)) == 0;
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
-    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0;
+    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
     x->timing = false; x->ev = nullptr; x->ev_steps = 0;
     *out = x;
     return SSGD_OK;
@@ -686,7 +732,7 @@ int ssgd_set_hash_params(ssgd_ctx* x, const uint32_t* in4r) {
 }
 
 int ssgd_set_insert_mode(ssgd_ctx* x, int32_t mode) {
-    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_SMEM) return SSGD_EINVAL;
+    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_TMA) return SSGD_EINVAL;
     x->insert_mode = mode;
     return SSGD_OK;
 }
@@ -788,7 +834,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
     if ((e = mark(x, 0, st))) return e;
-    if ((e = launch_accum(x, A, mode, st))) return e;
+    if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st) : launch_accum(x, A, mode, st))) return e;
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);
@@ -894,7 +940,7 @@ const char* ssgd_strerror(int code) {
         case SSGD_ENOTBOUND: return "no state/workspace bound (call ssgd_bind)";
         case SSGD_EWORKSPACE: return "workspace too small for this ncand";
         case SSGD_ECUDA: return "CUDA runtime error (see ssgd_last_error)";
-        case SSGD_EDEVICE: return "a kernel reported an out-of-range index";
+        case SSGD_EDEVICE: return "a kernel reported an error (index out of range, or a bounded wait gave up)";
         case SSGD_ENOMEM: return "out of host memory";
         default: return "unknown error";
     }

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssgd.so")
 
 OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM = 0, -1, -2, -3, -4, -5, -6, -7
-INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM = 0, 1, 2
+INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 MAX_R = 15
 
 # name -> argument types, exactly the declarations of include/ssgd.h
