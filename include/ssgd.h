@@ -55,6 +55,7 @@ extern "C" {
 #define SSGD_ECUDA      -5  /* a CUDA runtime call failed; ssgd_last_error gives its text              */
 #define SSGD_EDEVICE    -6  /* a kernel recorded an error: bad index in a caller's list, or a wait gave up */
 #define SSGD_ENOMEM     -7  /* host allocation failed                                                  */
+#define SSGD_ETOOBIG    -8  /* size beyond the fixed capacity of ssgd_exact_topk_static                */
 
 #define SSGD_MAX_R 15
 
@@ -132,6 +133,38 @@ int ssgd_step_buffers(const ssgd_ctx* ctx, const float** merged, const float** e
  * The same device functions the step uses (Algorithm 4 lines 2, 6, 11); for bit-exactness checks. */
 int ssgd_hashes(ssgd_ctx* ctx, const int32_t* idx, int64_t n, int32_t* h_out, int32_t* s_out,
                 void* stream);
+
+/* Second round and final top-k WITHOUT a workspace.  (The paper has no counterpart: this exists for
+ * the way the library gets embedded, not for the method.)
+ *
+ * Who needs it: code that is handed gradient and state buffers but may not allocate device memory
+ * itself -- a compression hook called from inside a trainer whose caching allocator owns the whole
+ * GPU (a raw cudaMalloc there can fail, and it stalls every stream of the device while it runs), or a
+ * caller on a latency-critical path that must not trigger allocation at all.  Such a caller cannot
+ * provide the workspace that ssgd_bind asks for, so this entry point keeps its scratch (second-round
+ * sums, radix histograms, chunk counters) in a fixed array of SSGD_STATIC_SCRATCH_BYTES (1.06 MiB)
+ * that is part of the library image: every GPU that loads the library holds that much until the
+ * process exits.  The call itself allocates nothing, on the host or on the device.
+ *
+ * What it computes: Algorithm 3 lines 10-11 exactly as ssgd_exact_topk does -- xs[m] = sum over
+ * w = 0..W-1 of v[w][cand_idx[m]] (fp64, that order), then the k entries with the largest |xs|, ties
+ * to the earlier position -- written to out_idx/out_val ([k], device) in cand_idx order.  It does NOT
+ * zero any state (line 13 stays with the caller) and needs no context: v ([W][ld] fp32, device),
+ * cand_idx ([ncand] int32, device, distinct, in [0, d); out-of-range entries count as zero) and the
+ * sizes are passed directly.  k <= ncand <= min(d, SSGD_STATIC_MAX_NCAND); a larger ncand is refused
+ * with SSGD_ETOOBIG before anything is launched.
+ *
+ * Sharing: all calls on one GPU use the same array, and it still holds the previous call's data.
+ * Each call first clears the parts that must start at zero, in stream order.  Two calls whose work
+ * can overlap on the GPU (different streams without an ordering between them, or different host
+ * threads doing so) race on the array and give wrong results: keep calls on one device ordered.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with that
+ * device current); make that first call before starting any stream capture.  Asynchronous on
+ * `stream` like the other stage calls. */
+#define SSGD_STATIC_MAX_NCAND     262144
+#define SSGD_STATIC_SCRATCH_BYTES 1114112
+int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, const int32_t* cand_idx,
+                           int64_t ncand, int64_t k, int32_t* out_idx, float* out_val, void* stream);
 
 /* Optional per-stage timing of ssgd_step with CUDA events recorded on the caller's stream (up to 256
  * steps between collections).  Stages: 0 = the accumulate+insert kernel, 1 = the unsketch kernel,

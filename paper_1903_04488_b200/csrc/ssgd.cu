@@ -18,6 +18,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 
@@ -932,6 +933,87 @@ int ssgd_status(ssgd_ctx* x, void* stream) {
     return SSGD_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Second round + final top-k for callers that cannot hand over a workspace (see include/ssgd.h).
+// The scratch lives in a fixed device array inside this library; its device address is looked up
+// once per device with cudaGetSymbolAddress (in host code the symbol's name is only a stand-in).
+// ------------------------------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+constexpr int64_t STATIC_MAX_NCAND = SSGD_STATIC_MAX_NCAND;
+constexpr size_t ST_OFF_HIST = 0;                                              // histograms (zeroed per call)
+constexpr size_t ST_OFF_STATE = ST_OFF_HIST + SEL_HIST_WORDS * 4;             // selection state (zeroed per call)
+constexpr size_t ST_ZERO_BYTES = ST_OFF_STATE + 256;
+constexpr size_t ST_OFF_ERR = ST_ZERO_BYTES;                                   // skipped-entry flag
+constexpr size_t ST_OFF_CHUNK = ST_OFF_ERR + 256;                              // 2 x nchunks counters
+constexpr size_t ST_NCHUNK_MAX = (STATIC_MAX_NCAND + SEL_CHUNK - 1) / SEL_CHUNK;
+constexpr size_t ST_OFF_XS = (ST_OFF_CHUNK + 2 * ST_NCHUNK_MAX * 4 + 255) / 256 * 256;   // second-round sums
+constexpr size_t ST_BYTES = ST_OFF_XS + (size_t)STATIC_MAX_NCAND * 4;
+static_assert(sizeof(SelState) <= 256, "selection state must fit its slot");
+static_assert(ST_BYTES <= SSGD_STATIC_SCRATCH_BYTES, "static scratch is smaller than its layout");
+
+static __device__ __align__(256) unsigned char g_static_scratch[SSGD_STATIC_SCRATCH_BYTES];
+
+constexpr int ST_MAX_DEVICES = 64;
+struct StaticDevice { unsigned char* scratch; int sm_count; };
+StaticDevice g_static_dev[ST_MAX_DEVICES] = {};
+std::mutex g_static_mutex;
+
+// Device address of the scratch array on the current device (looked up on the first call per device).
+int static_setup(StaticDevice** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= ST_MAX_DEVICES) return SSGD_ECUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice& sd = g_static_dev[dev];
+    if (!sd.scratch) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return SSGD_ECUDA;
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SSGD_ECUDA;
+        sd.sm_count = sms;
+        sd.scratch = static_cast<unsigned char*>(p);
+    }
+    *out = &sd;
+    return SSGD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, const int32_t* cand_idx,
+                           int64_t ncand, int64_t k, int32_t* out_idx, float* out_val, void* stream) {
+    if (!v || !cand_idx || !out_idx || !out_val) return SSGD_EINVAL;
+    if (d < 1 || d >= (int64_t)P31 || ld < d || W < 1 || k < 1 || k > ncand || ncand > d) return SSGD_EINVAL;
+    if (ncand > STATIC_MAX_NCAND) return SSGD_ETOOBIG;
+    StaticDevice* sd = nullptr;
+    int e = static_setup(&sd);
+    if (e) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = sd->scratch;
+    // the array keeps whatever the previous call left: histograms and selection state start from zero
+    if (cudaMemsetAsync(base, 0, ST_ZERO_BYTES, st) != cudaSuccess) return SSGD_ECUDA;
+    const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
+    SelBuffers sb;
+    uint32_t* h = reinterpret_cast<uint32_t*>(base + ST_OFF_HIST);
+    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
+    sb.state = reinterpret_cast<SelState*>(base + ST_OFF_STATE);
+    sb.chunk_gt = reinterpret_cast<uint32_t*>(base + ST_OFF_CHUNK);
+    sb.chunk_eq = sb.chunk_gt + nch;
+    float* xs = reinterpret_cast<float*>(base + ST_OFF_XS);
+    int32_t* err = reinterpret_cast<int32_t*>(base + ST_OFF_ERR);
+    k_gather<<<grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, st>>>(cand_idx, ncand, v, ld, W, d, xs, sb, (uint32_t)k, err);
+    const int grid = grid_for(ncand, SEL_THREADS * 8, (int64_t)sd->sm_count * 8);
+    k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
+    k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
+    k_sel_count<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb);
+    k_sel_scan<<<1, 1024, 0, st>>>(sb, nch);
+    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k);
+    return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ECUDA;
+}
+
 const char* ssgd_strerror(int code) {
     switch (code) {
         case SSGD_OK: return "ok";
@@ -942,6 +1024,7 @@ const char* ssgd_strerror(int code) {
         case SSGD_ECUDA: return "CUDA runtime error (see ssgd_last_error)";
         case SSGD_EDEVICE: return "a kernel reported an error (index out of range, or a bounded wait gave up)";
         case SSGD_ENOMEM: return "out of host memory";
+        case SSGD_ETOOBIG: return "size exceeds the fixed capacity of the built-in scratch";
         default: return "unknown error";
     }
 }

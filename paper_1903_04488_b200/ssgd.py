@@ -14,7 +14,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssgd.so")
 
-OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM = 0, -1, -2, -3, -4, -5, -6, -7
+OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7, -8
+STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 MAX_R = 15
 
@@ -36,6 +37,7 @@ SIGNATURES = {
     "ssgd_step_host": [_vp, _vp, _i64, _f32, _i64, _vp, _vp, _vp, _vp],
     "ssgd_step_buffers": [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp)],
     "ssgd_hashes": [_vp, _vp, _i64, _vp, _vp, _vp],
+    "ssgd_exact_topk_static": [_vp, _i64, _i32, _i64, _vp, _i64, _i64, _vp, _vp, _vp],
     "ssgd_set_timing": [_vp, _i32],
     "ssgd_get_stage_times": [_vp, _vp, C.POINTER(C.c_double), C.POINTER(_i64)],
     "ssgd_launch_count": [_vp, C.POINTER(_i64)],
@@ -81,6 +83,19 @@ def _dev_ptr(t: torch.Tensor | None, dtype, name: str):
 
 def _stream():
     return torch.cuda.current_stream().cuda_stream
+
+
+def exact_topk_static(v: torch.Tensor, d: int, cand_idx: torch.Tensor, k: int, out_idx: torch.Tensor,
+                      out_val: torch.Tensor) -> None:
+    """Second round + final top-k on the library's built-in scratch: no workspace, no context, no allocation
+    (for callers that may not allocate device memory; at most STATIC_MAX_NCAND candidates).  Does not zero
+    any state.  Calls on one GPU must not overlap: they share that scratch."""
+    code = lib().ssgd_exact_topk_static(_dev_ptr(v, torch.float32, "v"), v.shape[1], v.shape[0], d,
+                                        _dev_ptr(cand_idx, torch.int32, "cand_idx"), cand_idx.numel(), k,
+                                        _dev_ptr(out_idx, torch.int32, "out_idx"),
+                                        _dev_ptr(out_val, torch.float32, "out_val"), _stream())
+    if code:
+        raise SsgdError(code, "ssgd_exact_topk_static")
 
 
 class Ssgd:
