@@ -672,7 +672,10 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     const bool fits = table_bytes <= (size_t)200 * 1024 && (int64_t)table_bytes <= x->max_smem_optin;
     if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
     if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
-    return INS_MERGED_TMA;
+    if (x->insert_mode == SSGD_INSERT_TMA) return INS_MERGED_TMA;
+    // measured on B200: the bulk-copy pipeline wins once a tile's walk over the workers is long
+    // (W = 128: 5.73 vs 5.43 TB/s), plain loads win for short walks (W = 16: 4.93 vs 4.83 TB/s)
+    return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
 }  // namespace

@@ -40,7 +40,32 @@ def bucket_tau(orc, M, idx=None, chunk=1 << 20):
     return tau
 
 
-def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=None):
+def oracle_intermediates(orc, g_h, rho, u_o, v_o, ncand, by_linearity):
+    """T, M (fp64 [r][c]), est (fp32 [d]), cand (best first) of the oracle for this step; u_o, v_o are
+    advanced by the momentum/error accumulation (not zeroed).
+
+    by_linearity=False: the oracle's own step (every worker sketched on its own, then summed).
+    by_linearity=True: for sizes where W separate sketches take minutes -- the oracle's accumulate, then
+    ONE oracle sketch of the fp64 sum over workers (sum_w S(v_w) = S(sum_w v_w), a pinned property of the
+    oracle) and one of sum_w |v_w| for the bucket masses, then the oracle's estimate and selection."""
+    if not by_linearity:
+        o = orc.step(g_h, rho, u_o, v_o, ncand, zero_state=False, full=True)
+        return o["T"], o["M"], o["est"], o["cand"], o["out_idx"]
+    orc.accumulate(g_h, rho, u_o, v_o)
+    d = orc.d
+    x64 = np.zeros(d)
+    a64 = np.zeros(d)
+    for w in range(orc.W):                      # worker order, fp64
+        x64 += v_o[w, :d]
+        a64 += np.abs(v_o[w, :d])
+    T = orc.sketch(x64)
+    M = orc.sketch(a64, with_mass=True)[1]
+    est = orc.estimate(T.astype(np.float32))
+    cand = oracle_select(est, ncand)
+    return T, M, est, cand, None
+
+
+def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=None, by_linearity=False):
     """Runs eng.step on g_dev and the oracle on the same g; asserts the protocol; adopts.
 
     orc: oracle.Oracle; eng: bound Ssgd; u_o, v_o: the oracle's numpy state, bit-identical to the
@@ -58,26 +83,21 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
 
     # oracle, without its own zero-out
     g_h = g_dev.cpu().numpy()
-    o = orc.step(g_h, rho, u_o, v_o, ncand, zero_state=False, full=True)
+    T, M, est_o, cand_o, out_idx_o = oracle_intermediates(orc, g_h, rho, u_o, v_o, ncand, by_linearity)
+    del g_h
 
-    # 5 + 1: chosen coordinates are +0.0f everywhere, everything else equals the oracle bit for bit
+    # 5 + 1: the k chosen coordinates are distinct, ascending, in range (the bit-exact comparison of u and
+    # v -- zeros exactly there, the oracle's accumulation everywhere else -- follows the adoption below)
     assert len(np.unique(out_idx_g)) == k and out_idx_g.min() >= 0 and out_idx_g.max() < d
     assert (np.diff(out_idx_g) > 0).all(), "out_idx must be ascending"
-    chosen = np.zeros(u_o.shape[1], bool)
-    chosen[out_idx_g] = True
-    for name, got, want in (("u", u_g_h, u_o), ("v", v_g_h, v_o)):
-        assert (got[:, chosen].view(np.uint32) == 0).all(), f"{name}: chosen coordinates must be +0.0f"
-        assert (got[:, ~chosen].view(np.uint32) == want[:, ~chosen].view(np.uint32)).all(), \
-            f"{name}: momentum/error accumulation is not bit-exact"
 
     # 2: table and estimates
-    T, M = o["T"], o["M"]
     err = np.abs(merged_g.astype(np.float64) - T)
     assert (err <= TABLE_RTOL * M).all(), f"table: worst error/mass {np.max(err / np.maximum(M, 1e-300)):.3e}"
     tau = None
     if check_est:
         tau = bucket_tau(orc, M)
-        e_err = np.abs(est_g.astype(np.float64) - o["est"].astype(np.float64))
+        e_err = np.abs(est_g.astype(np.float64) - est_o.astype(np.float64))
         assert (e_err <= tau).all(), "estimates outside tolerance"
 
     # 3: candidates -- exact given the GPU's own estimates, admissible against the oracle's
@@ -85,7 +105,7 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
     want_c = np.sort(oracle_select(est_g, ncand))
     assert (cand_g == want_c).all(), "candidates are not the top-ncand of the GPU's estimates"
     if check_est and ncand < d:
-        a = np.abs(o["est"].astype(np.float64))
+        a = np.abs(est_o.astype(np.float64))
         hi = np.partition(a + tau, d - ncand)[d - ncand]   # ncand-th largest upper bound
         lo = np.partition(a - tau, d - ncand)[d - ncand]   # ncand-th largest lower bound
         inc = np.zeros(d, bool)
@@ -93,7 +113,7 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
         assert inc[(a - tau) > hi].all(), "a coordinate surely above the threshold is missing"
         assert not inc[(a + tau) < lo].any(), "a coordinate surely below the threshold was selected"
     if report is not None:
-        report.append(dict(cand_sym_diff=int(np.setxor1d(cand_g, o["cand"]).size)))
+        report.append(dict(cand_sym_diff=int(np.setxor1d(cand_g, cand_o).size)))
 
     # 4: final top-k -- the oracle's second round and top-k on the GPU's candidates
     xs = orc.second_round(v_o, cand_g)
@@ -102,10 +122,14 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
     order = np.argsort(want_idx)
     assert (out_idx_g == want_idx[order]).all(), "final k-set differs from the oracle's on the same candidates"
     assert (out_val_g.view(np.uint32) == want_val[order].view(np.uint32)).all(), "out_val differs"
-    if report is not None:
-        report[-1]["final_sym_diff_vs_unadopted"] = int(np.setxor1d(out_idx_g, o["out_idx"]).size)
+    if report is not None and out_idx_o is not None:
+        report[-1]["final_sym_diff_vs_unadopted"] = int(np.setxor1d(out_idx_g, out_idx_o).size)
 
-    # 6: adopt the GPU's selection
+    # 5 + 6: adopt the GPU's selection (the oracle zeroes u, v there, every worker); then the whole state
+    # must agree bit for bit: +0.0f at the chosen coordinates, the oracle's accumulation everywhere else
     orc.zero(u_o, v_o, out_idx_g)
-    assert (u_g_h.view(np.uint32) == u_o.view(np.uint32)).all() and (v_g_h.view(np.uint32) == v_o.view(np.uint32)).all()
+    for name, got, want in (("u", u_g_h, u_o), ("v", v_g_h, v_o)):
+        for w in range(W):
+            assert (got[w].view(np.uint32) == want[w].view(np.uint32)).all(), \
+                f"{name}[{w}]: state differs from the oracle's (accumulation or zero-out mask)"
     return out_idx_g, out_val_g

@@ -258,6 +258,51 @@ def test_step_host_matches_step(cuda_device):
 
 
 # ------------------------------------------------------------------------------------------------
+# the BASELINE configurations at full size, in the launch configuration bench.py times
+# ------------------------------------------------------------------------------------------------
+def run_full(cfg, dev, steps, by_linearity):
+    eng, orc, u, v = make(cfg, dev)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, dev)
+    report = []
+    g = None
+    for t in range(steps):
+        g = wl.gradients(st, t, out=g)
+        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report,
+                   by_linearity=by_linearity[t] if isinstance(by_linearity, (list, tuple)) else by_linearity)
+    return report
+
+
+def test_full_size_C1(cuda_device):
+    run_full(wl.C1, cuda_device, 1, False)
+
+
+def test_full_size_C2_bench_configuration(cuda_device):
+    # step 0: every worker sketched separately by the oracle; steps 1-2 (non-zero state, zeroed
+    # coordinates from the step before): the oracle's sketch of the fp64 sum
+    rep = run_full(wl.C2, cuda_device, 3, [False, True, True])
+    assert len(rep) == 3
+
+
+def test_full_size_C3(cuda_device):
+    run_full(wl.C3, cuda_device, 2, True)
+
+
+def test_full_size_C4_table_larger_than_half_of_l2(cuda_device):
+    run_full(wl.C4, cuda_device, 1, True)
+
+
+@pytest.mark.parametrize("W", [8, 256])
+def test_full_size_C5_worker_sweep(cuda_device, W):
+    cfg = wl.CONFIGS[f"C5_W{W}"]
+    free, _ = torch.cuda.mem_get_info()
+    need = 3 * cfg.W * cfg.ld * 4 + (1 << 30)
+    if free < need:
+        pytest.skip(f"needs {need >> 30} GiB of device memory")
+    run_full(cfg, cuda_device, 1, True)
+
+
+# ------------------------------------------------------------------------------------------------
 # argument checking (host side; nothing is launched)
 # ------------------------------------------------------------------------------------------------
 def test_argument_errors(cuda_device):
