@@ -113,11 +113,13 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
     const int64_t d_main = A.d & ~(int64_t)3;                      // bulk copies cover whole float4 groups
     const int64_t ntiles = (d_main + KT_TC - 1) / KT_TC;
 
+    pdl_trigger();
     if (tid == 0) {
         for (int s = 0; s < KT_STAGES; ++s) { mbar_init(&S.full[s], 1); mbar_init(&S.empty[s], KT_CONSUMER_WARPS); }
         S.abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    pdl_wait();
     __syncthreads();
 
     if (warp == KT_CONSUMER_WARPS) {

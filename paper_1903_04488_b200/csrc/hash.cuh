@@ -43,6 +43,13 @@ inline Bucketizer make_bucketizer(uint64_t c) {
 
 #ifdef __CUDACC__
 
+// Programmatic dependent launch: every kernel of the step lets its successor's blocks become resident
+// early (trigger) and waits for its predecessor to finish and flush before it touches global memory
+// (wait).  Both are no-ops when the launch does not carry the attribute.  Every block must reach
+// pdl_wait() before it exits, so that "kernel N finished" always implies "kernel N-1 finished".
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // x mod (2^31-1) for x < 2^62 + 2^31.
 __device__ __forceinline__ uint32_t mod_p31(uint64_t x) {
     const uint32_t lo = (uint32_t)x & P31;

@@ -123,8 +123,10 @@ __device__ __forceinline__ void flush_hist(const uint32_t* s_hist, uint32_t* __r
 __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ SelShared sh;
-    const uint32_t d1 = sb.state->d1;
+    pdl_trigger();
     for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    pdl_wait();
+    const uint32_t d1 = sb.state->d1;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
     for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
@@ -144,9 +146,11 @@ k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
 __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ SelShared sh;
+    pdl_trigger();
+    for (int b = threadIdx.x; b < H3_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    pdl_wait();
     const uint32_t d1 = sb.state->d1, d2 = sb.state->d2;
     const uint32_t prefix = (d1 << H2_BITS) | d2;
-    for (int b = threadIdx.x; b < H3_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
     for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
@@ -198,6 +202,8 @@ __device__ __forceinline__ void chunk_ballots(const float* __restrict__ val, int
 __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ uint32_t s_cnt[2 * SEL_WARPS];
+    pdl_trigger();
+    pdl_wait();
     const uint32_t T = sb.state->thr_key;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
@@ -218,7 +224,9 @@ k_sel_scan(SelBuffers sb, int64_t nchunks) {
     __shared__ uint32_t s_g[32], s_e[32];
     __shared__ uint32_t carry_g, carry_e;
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    pdl_trigger();
     if (t == 0) { carry_g = 0; carry_e = 0; }
+    pdl_wait();
     __syncthreads();
     for (int64_t base = 0; base < nchunks; base += 1024) {
         const int64_t i = base + t;
@@ -260,6 +268,8 @@ template <typename Sink>
 __device__ __forceinline__ void sel_emit_chunk(const float* __restrict__ val, int64_t n, const SelBuffers& sb,
                                                Sink sink) {
     __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
+    pdl_trigger();
+    pdl_wait();
     const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t warp_base = (int64_t)blockIdx.x * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS);

@@ -17,6 +17,7 @@
 
 #include <cstdint>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -50,6 +51,8 @@ __global__ void __launch_bounds__(K1_THREADS, SSGD_K1_MINBLOCKS)
 k_accum_insert(const AccumArgs A) {
     extern __shared__ float s_table[];  // MODE == INS_MERGED_SMEM: [R][c]
     const int64_t rc = (int64_t)R * A.c;
+    pdl_trigger();
+    pdl_wait();
     if (MODE == INS_MERGED_SMEM) {
         for (int64_t t = threadIdx.x; t < rc; t += K1_THREADS) s_table[t] = 0.0f;
         __syncthreads();
@@ -251,7 +254,9 @@ __global__ void __launch_bounds__(K3_THREADS)
 k_unsketch(const UnsketchArgs A) {
     __shared__ SelShared sh;
     uint32_t* s_hist = sh.hist;
+    pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += K3_THREADS) s_hist[b] = 0;
+    pdl_wait();
     __syncthreads();
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     const int64_t stride = (int64_t)gridDim.x * K3_THREADS;
@@ -310,7 +315,9 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
          int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag) {
     __shared__ SelShared sh;
     uint32_t* s_hist = sh.hist;
+    pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += 256) s_hist[b] = 0;
+    pdl_wait();
     __syncthreads();
     const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
     if (m < ncand) {
@@ -356,6 +363,8 @@ k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const i
 __global__ void __launch_bounds__(256)
 k_zero(const int32_t* __restrict__ out_idx, int64_t k, float* __restrict__ u, float* __restrict__ v,
        int64_t ld, int32_t W, int64_t d) {
+    pdl_trigger();
+    pdl_wait();
     const int64_t total = k * (int64_t)W;
     const int64_t stride = (int64_t)gridDim.x * 256;
     for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < total; t += stride) {
@@ -506,6 +515,28 @@ int ensure_device(ssgd_ctx* x) {
     return SSGD_OK;
 }
 
+// Launch with programmatic stream serialization: the kernel may become resident while its predecessor
+// drains; it orders itself with pdl_wait().  SSGD_NO_PDL=1 in the environment turns the attribute off.
+bool pdl_enabled() {
+    static const bool on = [] { const char* e = std::getenv("SSGD_NO_PDL"); return !(e && e[0] == '1'); }();
+    return on;
+}
+
+template <typename... P, typename... A>
+cudaError_t launch_pdl(cudaStream_t st, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, P(args)...);
+}
+
 inline int grid_for(int64_t items, int threads, int64_t cap) {
     int64_t b = (items + threads - 1) / threads;
     if (b < 1) b = 1;
@@ -525,7 +556,7 @@ int launch_accum_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
         k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, smem, st>>>(A);
     } else {
         const int grid = grid_for(groups, K1_THREADS, (int64_t)1 << 30);
-        k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, 0, st>>>(A);
+        CU(launch_pdl(st, k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
     }
     LAUNCHED("k_accum_insert");
     return SSGD_OK;
@@ -575,7 +606,8 @@ int launch_accum_tma_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
     }
     const int64_t ntiles = ((A.d & ~(int64_t)3) + KT_TC - 1) / KT_TC;
     const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->kt_blocks_per_sm);
-    kern<<<grid, KT_THREADS, smem, st>>>(A, reinterpret_cast<int32_t*>(x->ws + x->off_err));
+    CU(launch_pdl(st, kern, grid, KT_THREADS, smem, A, reinterpret_cast<int32_t*>(x->ws + x->off_err)),
+       "launch k_accum_insert_tma");
     LAUNCHED("k_accum_insert_tma");
     return SSGD_OK;
 }
@@ -589,7 +621,7 @@ int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     // a few blocks per SM: each block pays one histogram flush
     const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * 8);
-    k_unsketch<R, POW2><<<grid, K3_THREADS, 0, st>>>(A);
+    CU(launch_pdl(st, k_unsketch<R, POW2>, grid, K3_THREADS, 0, A), "launch k_unsketch");
     LAUNCHED("k_unsketch");
     return SSGD_OK;
 }
@@ -603,13 +635,13 @@ int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
 int launch_select(ssgd_ctx* x, const float* val, int64_t n, const SelBuffers& sb, int64_t nchunks,
                   cudaStream_t st) {
     const int grid = grid_for(n, SEL_THREADS * 8, (int64_t)x->sm_count * 8);
-    k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(val, n, sb);
+    CU(launch_pdl(st, k_sel_pass2, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass2");
     LAUNCHED("k_sel_pass2");
-    k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(val, n, sb);
+    CU(launch_pdl(st, k_sel_pass3, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass3");
     LAUNCHED("k_sel_pass3");
-    k_sel_count<<<(int)nchunks, SEL_THREADS, 0, st>>>(val, n, sb);
+    CU(launch_pdl(st, k_sel_count, (int)nchunks, SEL_THREADS, 0, val, n, sb), "launch k_sel_count");
     LAUNCHED("k_sel_count");
-    k_sel_scan<<<1, 1024, 0, st>>>(sb, nchunks);
+    CU(launch_pdl(st, k_sel_scan, 1, 1024, 0, sb, nchunks), "launch k_sel_scan");
     LAUNCHED("k_sel_scan");
     return SSGD_OK;
 }
@@ -643,7 +675,8 @@ int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* ca
     if (e) return e;
     if (timed && (e = mark(x, 2, st))) return e;
     if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st))) return e;
-    k_emit_candidates<<<(int)x->nchunk_c, SEL_THREADS, 0, st>>>(est, x->d, sb, cand_idx, cand_est, (uint32_t)ncand);
+    CU(launch_pdl(st, k_emit_candidates, (int)x->nchunk_c, SEL_THREADS, 0, (const float*)est, x->d, sb, cand_idx, cand_est,
+                  (uint32_t)ncand), "launch k_emit_candidates");
     LAUNCHED("k_emit_candidates");
     return SSGD_OK;
 }
@@ -654,15 +687,16 @@ int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t*
     int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
     SelBuffers sb = sel_buffers(x, true);
     const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
-    k_gather<<<grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, st>>>(cand, ncand, x->v, x->ld, x->W, x->d, xs,
-                                                                      sb, (uint32_t)x->k, err);
+    CU(launch_pdl(st, k_gather, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, (const float*)x->v, x->ld, x->W,
+                  x->d, xs, sb, (uint32_t)x->k, err), "launch k_gather");
     LAUNCHED("k_gather");
     int e = launch_select(x, xs, ncand, sb, nch, st);
     if (e) return e;
-    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand, out_idx, out_val, (uint32_t)x->k);
+    CU(launch_pdl(st, k_emit_final, (int)nch, SEL_THREADS, 0, (const float*)xs, ncand, sb, cand, out_idx, out_val,
+                  (uint32_t)x->k), "launch k_emit_final");
     LAUNCHED("k_emit_final");
-    k_zero<<<grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, st>>>(out_idx, x->k, x->u, x->v,
-                                                                                            x->ld, x->W, x->d);
+    CU(launch_pdl(st, k_zero, grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, (const int32_t*)out_idx,
+                  x->k, x->u, x->v, x->ld, x->W, x->d), "launch k_zero");
     LAUNCHED("k_zero");
     return SSGD_OK;
 }
