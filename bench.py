@@ -178,28 +178,22 @@ def workload_config(cfg, args):
 
 def run_ours(args, cfg):
     import torch
-    import torch.distributed as dist
     from paper_1903_04488_b200 import ssgd as S
     from paper_1903_04488_b200 import workloads as wl
+    from paper_1903_04488_b200.replicas import Replicas
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    rep = Replicas("nccl", dev)
+    rank, world, barrier = rep.rank, rep.world, rep.barrier
     if world != args.gpus:
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-
     # replicas differ only in their seeds
-    rcfg = cfg.scaled(base_seed=cfg.base_seed + 100 * rank)
+    rcfg = cfg.scaled(base_seed=cfg.base_seed + rep.replica_seed_offset())
     st = wl.Structure(rcfg, dev)
     n_sets = args.sets or cfg.steps
     g_sets = [wl.gradients(st, t) for t in range(n_sets)]
@@ -233,12 +227,7 @@ def run_ours(args, cfg):
     stage_ms, stage_n = eng.get_stage_times()
     eng.set_timing(False)
     assert eng.status() == S.OK
-    if world > 1:
-        tmax = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_total = float(tmax.item())
-    ms_step = ms_total / args.steps
-    value = world * cfg.W * cfg.d / (ms_step * 1e-3)
+    value, ms_step = rep.whole_job_value(cfg.W * cfg.d, ms_total / args.steps)
 
     # ---- end to end: host gradients in, host results out, through ssgd_step_host ------------------
     e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
@@ -258,10 +247,7 @@ def run_ours(args, cfg):
     e1.record()
     torch.cuda.synchronize(); barrier()
     e2e_ms = e0.elapsed_time(e1)
-    if world > 1:
-        tmax = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = rep.max_over_ranks(e2e_ms)
     e2e_value = world * cfg.W * cfg.d / (e2e_ms / e2e_steps * 1e-3) if e2e_steps else None
 
     # ---- roofline of the dominant kernel and of the whole step -----------------------------------
@@ -303,8 +289,7 @@ def run_ours(args, cfg):
                                 "sample": what, "seconds": sec}
     if rank == 0:
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    rep.close()
 
 
 def main():
