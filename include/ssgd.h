@@ -65,6 +65,14 @@ extern "C" {
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
 
+/* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  With pruning, coordinates that
+ * provably cannot be among the ncand largest |estimate| stop reading sketch rows early (a median of r
+ * values reaches a magnitude only if (r+1)/2 of them do); the candidates are identical either way.
+ * AUTO prunes when r >= 3, d >= 2^22 and ncand <= d/8 (below that the fixed costs outweigh the saving). */
+#define SSGD_PRUNE_AUTO 0
+#define SSGD_PRUNE_OFF  1
+#define SSGD_PRUNE_ON   2
+
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
 
 /* Algorithm 4 init(r, c) plus the shape of Algorithm 3: d coordinates, r rows (odd, 1..15), c columns,
@@ -77,6 +85,11 @@ int ssgd_get_hash_params(const ssgd_ctx* ctx, uint32_t* out4r);
 /* Replace them (for tests): a, a' in [1, p-1], b, b' in [0, p-1]. */
 int ssgd_set_hash_params(ssgd_ctx* ctx, const uint32_t* in4r);
 int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
+int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
+/* Diagnostics of the last ssgd_step's pruned path (waits for the stream): out[0] = 1 if the dense path had
+ * to take over (too few survivors, list overflow, too many ties), out[1] = number of coordinates that
+ * survived the early exit, out[2] = the prune threshold as a histogram-bin index (0: nothing pruned). */
+int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out3);
 
 /* Bytes of device scratch needed to run steps with up to ncand_max candidates (host only). */
 int ssgd_workspace_bytes(const ssgd_ctx* ctx, int64_t ncand_max, size_t* out_bytes);
@@ -125,7 +138,8 @@ int ssgd_step_host(ssgd_ctx* ctx, const float* g_host, int64_t ld_g, float rho, 
                    float* g_stage, int32_t* out_idx_host, float* out_val_host, void* stream);
 
 /* Device pointers into the workspace holding, after ssgd_step, the merged [r][c] table, est[d] and
- * the candidate list [ncand] (for tests and diagnostics).  Any of the outputs may be NULL. */
+ * the candidate list [ncand] (for tests and diagnostics).  Any of the outputs may be NULL.  est[d] is
+ * only filled when the step ran without pruning (or fell back to the dense path). */
 int ssgd_step_buffers(const ssgd_ctx* ctx, const float** merged, const float** est,
                       const int32_t** cand_idx, const float** cand_xs);
 

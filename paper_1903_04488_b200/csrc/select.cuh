@@ -8,8 +8,8 @@
 //   producer kernel   histogram H1 of key bits 30..19          (fused into the kernel that makes the values)
 //   k_sel_pass2       histogram H2 of bits 18..8 among items whose top digit is the threshold digit
 //   k_sel_pass3       histogram H3 of bits 7..0 among items matching the 23-bit threshold prefix
-//   k_sel_count       threshold key T and tie quota Q are now known: per-chunk counts of key > T, key == T
-//   k_sel_scan        exclusive scan of the chunk counts (one block)
+//   k_sel_count       threshold key T and tie quota Q are now known: per-chunk counts of key > T, key == T;
+//                     its last block turns the counts into exclusive offsets
 //   emit kernel       item i is selected iff key > T or (key == T and #equal before i < Q); its output
 //                     slot is #greater before i + min(#equal before i, Q): outputs come out in position
 //                     order, with no atomics and no dependence on scheduling.
@@ -38,8 +38,8 @@ struct SelState {
     uint32_t d2, rem2;   // same for H2
     uint32_t thr_key;    // T: the full 31-bit threshold key
     uint32_t quota_eq;   // Q >= 1: how many items with key == T are selected
-    uint32_t ticket[3];  // finished-block counters of the three histogram kernels
-    uint32_t pad[7];
+    uint32_t ticket[4];  // finished-block counters of the three histogram kernels and of the count kernel
+    uint32_t pad[6];
 };
 
 struct SelBuffers {
@@ -49,11 +49,16 @@ struct SelBuffers {
     SelState* state;
     uint32_t* chunk_gt;  // [nchunks] counts, then exclusive offsets
     uint32_t* chunk_eq;  // [nchunks]
+    const uint32_t* gate;  // if not NULL: the kernels of this selection run only when *gate != 0
 };
 
 #ifdef __CUDACC__
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// A gated selection is the dense fall-back of the sparse candidate path: its kernels are always
+// enqueued and leave at once unless the sparse path raised the flag (read after pdl_wait()).
+__device__ __forceinline__ bool gate_closed(const uint32_t* gate) { return gate != nullptr && __ldcg(gate) == 0; }
 
 struct SelShared {
     uint32_t hist[H1_BINS];
@@ -126,6 +131,7 @@ k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
+    if (gate_closed(sb.gate)) return;
     const uint32_t d1 = sb.state->d1;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
@@ -149,6 +155,7 @@ k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H3_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
+    if (gate_closed(sb.gate)) return;
     const uint32_t d1 = sb.state->d1, d2 = sb.state->d2;
     const uint32_t prefix = (d1 << H2_BITS) | d2;
     __syncthreads();
@@ -198,39 +205,18 @@ __device__ __forceinline__ void chunk_ballots(const float* __restrict__ val, int
     }
 }
 
-// ---- count: per-chunk numbers of key > T and key == T ---------------------------------------------
-__global__ void __launch_bounds__(SEL_THREADS)
-k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb) {
-    __shared__ uint32_t s_cnt[2 * SEL_WARPS];
-    pdl_trigger();
-    pdl_wait();
-    const uint32_t T = sb.state->thr_key;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
-    chunk_ballots(val, n, (int64_t)blockIdx.x * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS), T, bg, be, ngt, neq);
-    if (lane == 0) { s_cnt[warp] = ngt; s_cnt[SEL_WARPS + warp] = neq; }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t a = 0, b = 0;
-        for (int w = 0; w < SEL_WARPS; ++w) { a += s_cnt[w]; b += s_cnt[SEL_WARPS + w]; }
-        sb.chunk_gt[blockIdx.x] = a;
-        sb.chunk_eq[blockIdx.x] = b;
-    }
-}
-
-// ---- scan: chunk counts -> exclusive offsets (single block of 1024 threads) ------------------------
-__global__ void __launch_bounds__(1024)
-k_sel_scan(SelBuffers sb, int64_t nchunks) {
-    __shared__ uint32_t s_g[32], s_e[32];
-    __shared__ uint32_t carry_g, carry_e;
+// ---- count: per-chunk numbers of key > T and key == T; the last block turns them into offsets ------
+// Exclusive scan of the chunk counts in place, by one block of SEL_THREADS threads.
+__device__ __forceinline__ void block_scan_chunks(const SelBuffers& sb, int64_t nchunks, SelShared& sh) {
+    uint32_t* s_g = sh.hist;                 // [SEL_WARPS + 1] warp totals, then exclusive + tile total
+    uint32_t* s_e = sh.hist + 32;
+    uint32_t* carry = sh.hist + 64;          // [2]
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    pdl_trigger();
-    if (t == 0) { carry_g = 0; carry_e = 0; }
-    pdl_wait();
+    if (t == 0) { carry[0] = 0; carry[1] = 0; }
     __syncthreads();
-    for (int64_t base = 0; base < nchunks; base += 1024) {
+    for (int64_t base = 0; base < nchunks; base += SEL_THREADS) {
         const int64_t i = base + t;
-        const uint32_t g = i < nchunks ? sb.chunk_gt[i] : 0, e = i < nchunks ? sb.chunk_eq[i] : 0;
+        const uint32_t g = i < nchunks ? __ldcg(sb.chunk_gt + i) : 0, e = i < nchunks ? __ldcg(sb.chunk_eq + i) : 0;
         uint32_t ig = g, ie = e;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -239,45 +225,69 @@ k_sel_scan(SelBuffers sb, int64_t nchunks) {
         }
         if (lane == 31) { s_g[warp] = ig; s_e[warp] = ie; }
         __syncthreads();
-        if (warp == 0) {
-            uint32_t wg = s_g[lane], we = s_e[lane];
-            uint32_t xg = wg, xe = we;
-#pragma unroll
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t og = __shfl_up_sync(0xFFFFFFFFu, xg, off), oe = __shfl_up_sync(0xFFFFFFFFu, xe, off);
-                if (lane >= off) { xg += og; xe += oe; }
+        if (t == 0) {
+            uint32_t ag = 0, ae = 0;
+            for (int w = 0; w < SEL_WARPS; ++w) {
+                const uint32_t tg = s_g[w], te = s_e[w];
+                s_g[w] = ag; s_e[w] = ae;
+                ag += tg; ae += te;
             }
-            s_g[lane] = xg - wg;  // exclusive over warps
-            s_e[lane] = xe - we;
+            s_g[SEL_WARPS] = ag; s_e[SEL_WARPS] = ae;   // tile totals
         }
         __syncthreads();
-        const uint32_t cg = carry_g, ce = carry_e;
         if (i < nchunks) {
-            sb.chunk_gt[i] = cg + s_g[warp] + ig - g;
-            sb.chunk_eq[i] = ce + s_e[warp] + ie - e;
+            sb.chunk_gt[i] = carry[0] + s_g[warp] + ig - g;
+            sb.chunk_eq[i] = carry[1] + s_e[warp] + ie - e;
         }
         __syncthreads();
-        if (t == 1023) { carry_g = cg + s_g[warp] + ig; carry_e = ce + s_e[warp] + ie; }
+        if (t == 0) { carry[0] += s_g[SEL_WARPS]; carry[1] += s_e[SEL_WARPS]; }
         __syncthreads();
     }
+}
+
+__global__ void __launch_bounds__(SEL_THREADS)
+k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nchunks) {
+    __shared__ SelShared sh;
+    pdl_trigger();
+    pdl_wait();
+    if (gate_closed(sb.gate)) return;
+    const uint32_t T = sb.state->thr_key;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+        uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
+        chunk_ballots(val, n, chunk * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS), T, bg, be, ngt, neq);
+        if (lane == 0) { sh.hist[warp] = ngt; sh.hist[SEL_WARPS + warp] = neq; }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t a = 0, b = 0;
+            for (int w = 0; w < SEL_WARPS; ++w) { a += sh.hist[w]; b += sh.hist[SEL_WARPS + w]; }
+            sb.chunk_gt[chunk] = a;
+            sb.chunk_eq[chunk] = b;
+        }
+        __syncthreads();
+    }
+    if (block_is_last(&sb.state->ticket[3], sh)) block_scan_chunks(sb, nchunks, sh);
 }
 
 // ---- emit: ordered compaction of the selected items -----------------------------------------------
 // `sink(slot, i)` is called once for every selected item i with its output slot (0 .. m-1).
 template <typename Sink>
-__device__ __forceinline__ void sel_emit_chunk(const float* __restrict__ val, int64_t n, const SelBuffers& sb,
-                                               Sink sink) {
+__device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, int64_t n, const SelBuffers& sb,
+                                                int64_t nchunks, Sink sink) {
     __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
     pdl_trigger();
     pdl_wait();
+    if (gate_closed(sb.gate)) return;
     const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t warp_base = (int64_t)blockIdx.x * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS);
+  for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
+    const int64_t warp_base = chunk * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS);
     uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
     chunk_ballots(val, n, warp_base, T, bg, be, ngt, neq);
+    __syncthreads();                       // the previous chunk's readers are done with s_wg, s_we
     if (lane == 0) { s_wg[warp] = ngt; s_we[warp] = neq; }
     __syncthreads();
-    uint32_t gt_before = sb.chunk_gt[blockIdx.x], eq_before = sb.chunk_eq[blockIdx.x];
+    uint32_t gt_before = sb.chunk_gt[chunk], eq_before = sb.chunk_eq[chunk];
     for (int w = 0; w < warp; ++w) { gt_before += s_wg[w]; eq_before += s_we[w]; }
     const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
@@ -289,6 +299,7 @@ __device__ __forceinline__ void sel_emit_chunk(const float* __restrict__ val, in
         gt_before += __popc(bg[it]);
         eq_before += __popc(be[it]);
     }
+  }
 }
 
 #endif  // __CUDACC__

@@ -18,6 +18,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <mutex>
 #include <new>
@@ -27,6 +28,8 @@
 #include "hash.cuh"
 #include "select.cuh"
 #include "accum_tma.cuh"
+#include "estimate.cuh"
+#include "sparse_select.cuh"
 
 namespace ssgd {
 
@@ -38,13 +41,19 @@ namespace ssgd {
 enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
 
 #ifndef SSGD_K1_UNROLL
-#define SSGD_K1_UNROLL 4
+#define SSGD_K1_UNROLL 16
 #endif
 #ifndef SSGD_K1_MINBLOCKS
 #define SSGD_K1_MINBLOCKS 1
 #endif
-constexpr int K1_THREADS = 256;
+// Measured on B200 (C2, W = 16): 256 threads x 4 workers in flight 4.93 TB/s; 128 x 8 5.38; 128 x 16 5.58;
+// 64 x 16 5.56; forcing more resident blocks (fewer registers) or 32 workers in flight is slower.
+#ifndef SSGD_K1_THREADS
+#define SSGD_K1_THREADS 128
+#endif
+constexpr int K1_THREADS = SSGD_K1_THREADS;
 constexpr int K1_UNROLL = SSGD_K1_UNROLL;  // workers in flight per thread: 3 x 16 B loads each
+constexpr int K1_UNROLL_PW = 4;            // same, for the per-worker-table mode (it also holds 4r hashes)
 
 template <int R, bool POW2, int MODE>
 __global__ void __launch_bounds__(K1_THREADS, SSGD_K1_MINBLOCKS)
@@ -68,10 +77,11 @@ k_accum_insert(const AccumArgs A) {
         }
         float x[4] = {0.f, 0.f, 0.f, 0.f};  // sum over workers of the new v (worker order)
         if (i0 + 3 < A.d) {
-            for (int w0 = 0; w0 < A.W; w0 += K1_UNROLL) {
-                float4 gg[K1_UNROLL], uu[K1_UNROLL], vv[K1_UNROLL];
+            constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : K1_UNROLL;
+            for (int w0 = 0; w0 < A.W; w0 += U) {
+                float4 gg[U], uu[U], vv[U];
 #pragma unroll
-                for (int s = 0; s < K1_UNROLL; ++s) {
+                for (int s = 0; s < U; ++s) {
                     if (w0 + s < A.W) {
                         const int64_t w = w0 + s;
                         gg[s] = __ldcs(reinterpret_cast<const float4*>(A.g + w * A.ld_g + i0));
@@ -80,7 +90,7 @@ k_accum_insert(const AccumArgs A) {
                     }
                 }
 #pragma unroll
-                for (int s = 0; s < K1_UNROLL; ++s) {
+                for (int s = 0; s < U; ++s) {
                     if (w0 + s < A.W) {
                         const int64_t w = w0 + s;
                         float4 un, vn;
@@ -138,11 +148,7 @@ k_accum_insert(const AccumArgs A) {
                     if (i0 + e < A.d && x[e] != 0.0f) {
                         const float sx = apply_sign(x[e], h1[e]);
                         if (MODE == INS_MERGED_SMEM) atomicAdd(&s_table[(int64_t)j * A.c + (h1[e] & P31)], sx);
-#ifndef SSGD_EXP_NOATOMICS
                         else red_add(A.table + (int64_t)j * A.c + (h1[e] & P31), sx);
-#else
-                        else if (sx == 1.2345e-30f) A.table[0] = sx;
-#endif
                     }
                 }
             }
@@ -194,34 +200,6 @@ k_merge(const float* __restrict__ tables, float* __restrict__ merged, int64_t rc
 // ------------------------------------------------------------------------------------------------
 // K3: estimate of every coordinate (median of r signed buckets) + first histogram of |estimate|
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void cswap(float& a, float& b) {
-    const float lo = fminf(a, b), hi = fmaxf(a, b);
-    a = lo; b = hi;
-}
-
-template <int R>
-__device__ __forceinline__ float median_of(float (&a)[R]) {
-    if constexpr (R == 1) {
-        return a[0];
-    } else if constexpr (R == 3) {
-        return fmaxf(fminf(a[0], a[1]), fminf(fmaxf(a[0], a[1]), a[2]));
-    } else if constexpr (R == 5) {
-        // sort two pairs; the smaller of the two minima and the larger of the two maxima cannot be
-        // the median; the median of the remaining three is the median of five
-        cswap(a[0], a[1]); cswap(a[3], a[4]);
-        const float lo = fmaxf(a[0], a[3]);   // larger of the pair minima
-        const float hi = fminf(a[1], a[4]);   // smaller of the pair maxima
-        return fmaxf(fminf(lo, hi), fminf(fmaxf(lo, hi), a[2]));
-    } else {
-        // general odd R: odd-even transposition sort in registers, then the middle element
-#pragma unroll
-        for (int round = 0; round < R; ++round)
-#pragma unroll
-            for (int p = round & 1; p + 1 < R; p += 2) cswap(a[p], a[p + 1]);
-        return a[R / 2];
-    }
-}
-
 struct UnsketchArgs {
     const float* table; int64_t c; int64_t d;
     HashParams hp; Bucketizer bk;
@@ -230,24 +208,8 @@ struct UnsketchArgs {
     uint32_t want;       // ncand
 };
 
-#ifndef SSGD_K3_NC
-#define SSGD_K3_NC 4
-#endif
-#ifndef SSGD_K3_LOAD
-#define SSGD_K3_LOAD 0
-#endif
 constexpr int K3_THREADS = 256;
-constexpr int K3_NC = SSGD_K3_NC;  // consecutive coordinates per thread (multiple of 4)
-
-__device__ __forceinline__ float table_load(const float* p) {
-#if SSGD_K3_LOAD == 0
-    return __ldg(p);
-#elif SSGD_K3_LOAD == 1
-    return __ldcg(p);
-#else
-    return *p;
-#endif
-}
+constexpr int K3_NC = 4;  // consecutive coordinates per thread
 
 template <int R, bool POW2>
 __global__ void __launch_bounds__(K3_THREADS)
@@ -257,6 +219,7 @@ k_unsketch(const UnsketchArgs A) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += K3_THREADS) s_hist[b] = 0;
     pdl_wait();
+    if (gate_closed(A.sb.gate)) return;
     __syncthreads();
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     const int64_t stride = (int64_t)gridDim.x * K3_THREADS;
@@ -278,10 +241,8 @@ k_unsketch(const UnsketchArgs A) {
 #pragma unroll
             for (int e = 0; e < K3_NC; e += 4)
                 *reinterpret_cast<float4*>(A.est + i0 + e) = make_float4(m[e], m[e + 1], m[e + 2], m[e + 3]);
-#ifndef SSGD_EXP_NOHIST
 #pragma unroll
             for (int e = 0; e < K3_NC; ++e) atomicAdd(&s_hist[key_of(m[e]) >> H1_SHIFT], 1u);
-#endif
         } else {
             for (int e = 0; e < K3_NC && i0 + e < A.d; ++e) {
                 A.est[i0 + e] = m[e];
@@ -299,8 +260,8 @@ k_unsketch(const UnsketchArgs A) {
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32_t* __restrict__ cand_idx,
-                  float* __restrict__ cand_est, uint32_t cap) {
-    sel_emit_chunk(est, d, sb, [&](uint32_t slot, int64_t i) {
+                  float* __restrict__ cand_est, uint32_t cap, int64_t nchunks) {
+    sel_emit_chunks(est, d, sb, nchunks, [&](uint32_t slot, int64_t i) {
         if (slot >= cap) return;  // cannot happen with consistent histograms; never write past the list
         cand_idx[slot] = (int32_t)i;
         if (cand_est) cand_est[slot] = est[i];
@@ -352,8 +313,8 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const int32_t* __restrict__ cand,
-             int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap) {
-    sel_emit_chunk(xs, ncand, sb, [&](uint32_t slot, int64_t m) {
+             int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap, int64_t nchunks) {
+    sel_emit_chunks(xs, ncand, sb, nchunks, [&](uint32_t slot, int64_t m) {
         if (slot >= cap) return;
         out_idx[slot] = cand[m];
         out_val[slot] = xs[m];
@@ -415,6 +376,9 @@ struct ssgd_ctx {
     char* ws; size_t ws_bytes; int64_t ncand_max;
     // workspace layout (byte offsets)
     size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
+    size_t off_sp_hist, off_sp_state, off_bitmap, off_list_idx, off_list_est;   // sparse candidate path
+    int64_t list_cap;
+    int32_t prune_mode;
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;
     // device facts
@@ -460,6 +424,9 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_state_c = o; o += up(sizeof(SelState));
     x->off_hist_f = o;  o += up(SEL_HIST_WORDS * 4);
     x->off_state_f = o; o += up(sizeof(SelState));
+    x->off_sp_hist = o; o += up(2 * H1_BINS * 4);
+    x->off_sp_state = o; o += up(sizeof(SparseState));
+    x->off_bitmap = o;  o += up((size_t)((x->d + 31) / 32) * 4);
     x->off_err = o;     o += up(16);
     x->zero_bytes = o;
     x->nchunk_c = (x->d + SEL_CHUNK - 1) / SEL_CHUNK;
@@ -469,13 +436,17 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_chunk_f = o; o += up((size_t)x->nchunk_f * 8);
     x->off_cand = o;    o += up((size_t)ncand_max * 4);
     x->off_xs = o;      o += up((size_t)ncand_max * 4);
+    x->list_cap = 4 * ncand_max > 65536 ? 4 * ncand_max : 65536;
+    if (x->list_cap > x->d) x->list_cap = x->d;
+    x->off_list_idx = o; o += up((size_t)x->list_cap * 4);
+    x->off_list_est = o; o += up((size_t)x->list_cap * 4);
     x->off_oidx = o;    o += up((size_t)x->k * 4);
     x->off_oval = o;    o += up((size_t)x->k * 4);
     x->total_bytes = o;
 }
 
 SelBuffers sel_buffers(ssgd_ctx* x, bool final_stage) {
-    SelBuffers sb;
+    SelBuffers sb{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_hist_f : x->off_hist_c));
     sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
     sb.state = reinterpret_cast<SelState*>(x->ws + (final_stage ? x->off_state_f : x->off_state_c));
@@ -639,10 +610,9 @@ int launch_select(ssgd_ctx* x, const float* val, int64_t n, const SelBuffers& sb
     LAUNCHED("k_sel_pass2");
     CU(launch_pdl(st, k_sel_pass3, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass3");
     LAUNCHED("k_sel_pass3");
-    CU(launch_pdl(st, k_sel_count, (int)nchunks, SEL_THREADS, 0, val, n, sb), "launch k_sel_count");
+    CU(launch_pdl(st, k_sel_count, grid_for(nchunks, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, val, n, sb, nchunks),
+       "launch k_sel_count");
     LAUNCHED("k_sel_count");
-    CU(launch_pdl(st, k_sel_scan, 1, 1024, 0, sb, nchunks), "launch k_sel_scan");
-    LAUNCHED("k_sel_scan");
     return SSGD_OK;
 }
 
@@ -666,19 +636,92 @@ int mark(ssgd_ctx* x, int which, cudaStream_t st) {
 }
 
 int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, float* cand_est,
-                    float* est, cudaStream_t st, bool timed = false) {
+                    float* est, cudaStream_t st, bool timed = false, const uint32_t* gate = nullptr) {
     UnsketchArgs A;
     A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk; A.est = est;
     SelBuffers sb = sel_buffers(x, false);
+    sb.gate = gate;
     A.sb = sb; A.want = (uint32_t)ncand;
     int e = launch_unsketch(x, A, st);
     if (e) return e;
     if (timed && (e = mark(x, 2, st))) return e;
     if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st))) return e;
-    CU(launch_pdl(st, k_emit_candidates, (int)x->nchunk_c, SEL_THREADS, 0, (const float*)est, x->d, sb, cand_idx, cand_est,
-                  (uint32_t)ncand), "launch k_emit_candidates");
+    CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)est,
+                  x->d, sb, cand_idx, cand_est, (uint32_t)ncand, x->nchunk_c), "launch k_emit_candidates");
     LAUNCHED("k_emit_candidates");
     return SSGD_OK;
+}
+
+SparseBuffers sparse_buffers(ssgd_ctx* x) {
+    SparseBuffers sp{};
+    uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + x->off_sp_hist);
+    sp.h1_sample = h; sp.h1 = h + H1_BINS;
+    sp.state = reinterpret_cast<SparseState*>(x->ws + x->off_sp_state);
+    sp.list_idx = reinterpret_cast<int32_t*>(x->ws + x->off_list_idx);
+    sp.list_est = reinterpret_cast<float*>(x->ws + x->off_list_est);
+    sp.cap = (uint32_t)x->list_cap;
+    sp.bitmap = reinterpret_cast<uint32_t*>(x->ws + x->off_bitmap);
+    return sp;
+}
+
+// Whether ssgd_step takes the early-exit unsketch + sparse selection (sparse_select.cuh).
+bool use_sparse(const ssgd_ctx* x, int64_t ncand) {
+    if (x->prune_mode == SSGD_PRUNE_OFF) return false;
+    if (x->prune_mode == SSGD_PRUNE_ON) return true;
+    return x->r >= 3 && x->d >= (1 << 22) && ncand * 8 <= x->d;
+}
+
+template <int R, bool POW2>
+int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
+    CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count), SEL_THREADS, 0, A),
+       "launch k_unsketch_sample");
+    LAUNCHED("k_unsketch_sample");
+    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, grid_for(groups, SEL_THREADS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, A),
+       "launch k_unsketch_pruned");
+    LAUNCHED("k_unsketch_pruned");
+    return SSGD_OK;
+}
+
+int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_sparse_t, x, A, st)
+}
+
+int launch_select_sparse(ssgd_ctx* x, const SparseBuffers& sp, int64_t ncand, int32_t* cand_idx, cudaStream_t st) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(SPARSE_CLUSTER);
+    cfg.blockDim = dim3(SPARSE_THREADS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = SPARSE_CLUSTER; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    CU(cudaLaunchKernelEx(&cfg, k_select_sparse, sp, x->d, (uint32_t)ncand, cand_idx), "launch k_select_sparse");
+    LAUNCHED("k_select_sparse");
+    return SSGD_OK;
+}
+
+// Line 9 with early exit: sample -> pruned unsketch -> cluster selection; the dense path follows, gated.
+int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, float* est,
+                           cudaStream_t st) {
+    SparseArgs A;
+    A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk;
+    A.sp = sparse_buffers(x);
+    A.ncand = (uint32_t)ncand;
+    const int64_t groups = (x->d + 3) / 4;
+    const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
+    const double mean = (double)ncand * (double)(windows * 4) / (double)x->d;
+    A.want_sample = (uint32_t)(mean + 6.0 * std::sqrt(mean) + 16.0 + 1.0);
+    int e = launch_sparse(x, A, st);
+    if (e) return e;
+    if ((e = mark(x, 2, st))) return e;
+    if ((e = launch_select_sparse(x, A.sp, ncand, cand_idx, st))) return e;
+    return unsketch_select(x, merged, ncand, cand_idx, nullptr, est, st, false, &A.sp.state->fallback);
 }
 
 int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
@@ -692,8 +735,8 @@ int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t*
     LAUNCHED("k_gather");
     int e = launch_select(x, xs, ncand, sb, nch, st);
     if (e) return e;
-    CU(launch_pdl(st, k_emit_final, (int)nch, SEL_THREADS, 0, (const float*)xs, ncand, sb, cand, out_idx, out_val,
-                  (uint32_t)x->k), "launch k_emit_final");
+    CU(launch_pdl(st, k_emit_final, grid_for(nch, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)xs, ncand, sb,
+                  cand, out_idx, out_val, (uint32_t)x->k, nch), "launch k_emit_final");
     LAUNCHED("k_emit_final");
     CU(launch_pdl(st, k_zero, grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, (const int32_t*)out_idx,
                   x->k, x->u, x->v, x->ld, x->W, x->d), "launch k_zero");
@@ -733,7 +776,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0;
     *out = x;
     return SSGD_OK;
 }
@@ -766,6 +809,23 @@ int ssgd_set_hash_params(ssgd_ctx* x, const uint32_t* in4r) {
         x->hp.row[j].a = in4r[4 * j]; x->hp.row[j].b = in4r[4 * j + 1];
         x->hp.row[j].a2 = in4r[4 * j + 2]; x->hp.row[j].b2 = in4r[4 * j + 3];
     }
+    return SSGD_OK;
+}
+
+int ssgd_set_prune_mode(ssgd_ctx* x, int32_t mode) {
+    if (!x || mode < SSGD_PRUNE_AUTO || mode > SSGD_PRUNE_ON) return SSGD_EINVAL;
+    x->prune_mode = mode;
+    return SSGD_OK;
+}
+
+int ssgd_step_used_fallback(ssgd_ctx* x, void* stream, int32_t* out) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!out) return SSGD_EINVAL;
+    CU(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)), "stream synchronize");
+    SparseState s;
+    CU(cudaMemcpy(&s, x->ws + x->off_sp_state, sizeof(s), cudaMemcpyDeviceToHost), "read sparse state");
+    out[0] = (int32_t)s.fallback; out[1] = (int32_t)s.n_surv; out[2] = (int32_t)s.bin_lo;
     return SSGD_OK;
 }
 
@@ -876,7 +936,11 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);
-    if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
+    if (use_sparse(x, ncand)) {
+        if ((e = unsketch_select_sparse(x, merged, ncand, cand, est, st))) return e;
+    } else {
+        if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
+    }
     if ((e = mark(x, 3, st))) return e;
     if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st))) return e;
     if ((e = mark(x, 4, st))) return e;
@@ -1033,7 +1097,7 @@ int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, con
     // the array keeps whatever the previous call left: histograms and selection state start from zero
     if (cudaMemsetAsync(base, 0, ST_ZERO_BYTES, st) != cudaSuccess) return SSGD_ECUDA;
     const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
-    SelBuffers sb;
+    SelBuffers sb{};
     uint32_t* h = reinterpret_cast<uint32_t*>(base + ST_OFF_HIST);
     sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
     sb.state = reinterpret_cast<SelState*>(base + ST_OFF_STATE);
@@ -1045,9 +1109,8 @@ int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, con
     const int grid = grid_for(ncand, SEL_THREADS * 8, (int64_t)sd->sm_count * 8);
     k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
     k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
-    k_sel_count<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb);
-    k_sel_scan<<<1, 1024, 0, st>>>(sb, nch);
-    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k);
+    k_sel_count<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, nch);
+    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k, nch);
     return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ECUDA;
 }
 

@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libssgd.so")
 OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
+PRUNE_AUTO, PRUNE_OFF, PRUNE_ON = 0, 1, 2
 MAX_R = 15
 
 # name -> argument types, exactly the declarations of include/ssgd.h
@@ -27,6 +28,8 @@ SIGNATURES = {
     "ssgd_get_hash_params": [_vp, _vp],
     "ssgd_set_hash_params": [_vp, _vp],
     "ssgd_set_insert_mode": [_vp, _i32],
+    "ssgd_set_prune_mode": [_vp, _i32],
+    "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
     "ssgd_sketch_accumulate": [_vp, _vp, _i64, _f32, _vp, _vp],
@@ -133,6 +136,15 @@ class Ssgd:
 
     def set_insert_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_insert_mode(self._h, mode), "ssgd_set_insert_mode")
+
+    def set_prune_mode(self, mode: int) -> None:
+        self._chk(self._lib.ssgd_set_prune_mode(self._h, mode), "ssgd_set_prune_mode")
+
+    def step_used_fallback(self):
+        """(fell back to the dense path?, survivors of the early exit, prune threshold bin) of the last step."""
+        out = (_i32 * 3)()
+        self._chk(self._lib.ssgd_step_used_fallback(self._h, _stream(), out), "ssgd_step_used_fallback")
+        return bool(out[0]), int(out[1]), int(out[2])
 
     def workspace_bytes(self, ncand_max: int) -> int:
         out = _sz()

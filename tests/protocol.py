@@ -77,7 +77,15 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
     eng.step(g_dev, rho, ncand, out_idx, out_val)
     assert eng.status() == 0
     u_g, v_g, _ = eng._keep
-    merged_g, est_g, cand_g, xs_g = [t.cpu().numpy() for t in eng.step_buffers(ncand)]
+    merged_t, _, cand_t, xs_t = eng.step_buffers(ncand)
+    merged_g, cand_g, xs_g = merged_t.cpu().numpy(), cand_t.cpu().numpy(), xs_t.cpu().numpy()
+    # the step may have skipped estimates that provably cannot matter (early exit); the dense stage call
+    # on the step's own table gives the estimate of EVERY coordinate, and must pick the same candidates
+    est_t = torch.empty(d + 4, dtype=torch.float32, device=dev)[:d]
+    cand_dense = torch.empty(ncand, dtype=torch.int32, device=dev)
+    eng.unsketch_candidates(merged_t, ncand, cand_dense, None, est_t)
+    est_g = est_t.cpu().numpy()
+    assert (cand_dense.cpu().numpy() == cand_g).all(), "step and dense stage call disagree on the candidates"
     out_idx_g, out_val_g = out_idx.cpu().numpy(), out_val.cpu().numpy()
     u_g_h, v_g_h = u_g.cpu().numpy(), v_g.cpu().numpy()
 

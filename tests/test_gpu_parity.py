@@ -153,11 +153,15 @@ STEP_CASES = [
 
 @pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
 @pytest.mark.parametrize("mode", [S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
-def test_step_lockstep(cuda_device, cfg, steps, mode):
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
     if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
         pytest.skip("table does not fit the shared-memory variant")
+    if prune == S.PRUNE_ON and mode != S.INSERT_GLOBAL:
+        pytest.skip("the candidate path does not depend on the insert variant: one combination suffices")
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_insert_mode(mode)
+    eng.set_prune_mode(prune)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     st = wl.Structure(cfg, cuda_device)
     report = []
@@ -168,19 +172,26 @@ def test_step_lockstep(cuda_device, cfg, steps, mode):
         assert all(r["final_sym_diff_vs_unadopted"] == 0 for r in report)
 
 
-def test_all_zero_gradient_ties_break_by_index(cuda_device):
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     cfg = wl.C2.scaled(d=10_001, W=3, c=256, ncand=700, k=300)
     eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(prune)
     g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     assert idx.tolist() == list(range(cfg.k)) and (val == 0).all()
+    if prune == S.PRUNE_ON:
+        fell_back, survivors, bin_lo = eng.step_used_fallback()
+        assert fell_back and bin_lo == 0 and survivors == cfg.d     # d equal magnitudes: the dense path ranks them
 
 
-def test_heavy_ties_at_the_threshold(cuda_device):
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
     cfg = wl.C2.scaled(d=40_000, W=2, r=1, c=40_000, ncand=1000, k=400)
     eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(prune)
     ident = [[1, 0, 1, 0]]
     eng.set_hash_params(ident)
     orc.set_params(ident)          # table = signed copy of the summed vector: estimates are exact
@@ -191,6 +202,21 @@ def test_heavy_ties_at_the_threshold(cuda_device):
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     big = set(range(11, 500, 13))
     assert big <= set(idx.tolist())
+
+
+def test_pruned_path_is_taken_and_prunes(cuda_device):
+    """On a gradient-shaped input the early-exit path must do its job: no fall-back, a non-trivial
+    threshold, at least ncand survivors and far fewer than d; a few ties at the threshold are ranked by index."""
+    cfg = wl.C2.scaled(d=600_001, W=4, c=16_384, ncand=6000, k=3000)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    for t in range(2):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
+        fell_back, survivors, bin_lo = eng.step_used_fallback()
+        assert not fell_back and bin_lo > 0
+        assert cfg.ncand <= survivors <= cfg.d // 10
 
 
 def test_planted_heavy_coordinates_recovered(cuda_device):
