@@ -86,6 +86,11 @@ int ssgd_get_hash_params(const ssgd_ctx* ctx, uint32_t* out4r);
 int ssgd_set_hash_params(ssgd_ctx* ctx, const uint32_t* in4r);
 int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
 int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
+/* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
+ * (cudaLimitPersistingL2CacheSize of this process's CUDA context is raised to the table size, capped by the
+ * device; the launches then carry an access-policy window over the table).  Off by default because the limit
+ * is shared with everything else the process runs on that device.  enable = 0 stops attaching the window. */
+int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
 /* Diagnostics of the last ssgd_step's pruned path (waits for the stream): out[0] = 1 if the dense path had
  * to take over (too few survivors, list overflow, too many ties), out[1] = number of coordinates that
  * survived the early exit, out[2] = the prune threshold as a histogram-bin index (0: nothing pruned). */

@@ -123,6 +123,9 @@ k_unsketch_sample(const SparseArgs A) {
 #ifndef SSGD_PRUNED_MINBLOCKS
 #define SSGD_PRUNED_MINBLOCKS 1
 #endif
+#ifndef SSGD_PRUNED_NC
+#define SSGD_PRUNED_NC 4
+#endif
 template <int R, bool POW2>
 __global__ void __launch_bounds__(SEL_THREADS, SSGD_PRUNED_MINBLOCKS)
 k_unsketch_pruned(const SparseArgs A) {
@@ -134,39 +137,43 @@ k_unsketch_pruned(const SparseArgs A) {
     const uint32_t bin_lo = A.sp.state->bin_lo;
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    const int64_t groups = (A.d + 3) >> 2;
+    constexpr int NC = SSGD_PRUNED_NC;                     // consecutive coordinates per thread
+    const int64_t groups = (A.d + NC - 1) / NC;
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
     // warp-uniform trip count: the append below uses warp-wide shuffles
     for (int64_t base = (int64_t)blockIdx.x * SEL_THREADS + (threadIdx.x & ~31); base < groups; base += stride) {
         const int64_t q = base + lane;
-        const int64_t i0 = q << 2;
-        float rowv[4][R];
-        int cnt[4] = {0, 0, 0, 0};
-        bool alive[4];
+        const int64_t i0 = q * NC;
+        float rowv[NC][R];
+        int cnt[NC];
+        bool alive[NC];
+        bool any = false;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) alive[e] = q < groups && i0 + e < A.d;
-        const bool any0 = alive[0];
-        if (any0) {
+        for (int e = 0; e < NC; ++e) { cnt[e] = 0; alive[e] = q < groups && i0 + e < A.d; any = any || alive[e]; }
+        if (any) {
 #pragma unroll
             for (int j = 0; j < NEED; ++j) {
-                uint32_t hb[4];
-                row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+                uint32_t hb[NC];
+                row_hashes<POW2, NC>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
 #pragma unroll
-                for (int e = 0; e < 4; ++e) {
+                for (int e = 0; e < NC; ++e) {
                     const float val = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
                     rowv[e][j] = val;
                     cnt[e] += (key_of(val) >> H1_SHIFT) >= bin_lo ? 1 : 0;
                 }
             }
 #pragma unroll
-            for (int e = 0; e < 4; ++e) alive[e] = alive[e] && cnt[e] + (R - NEED) >= NEED;
+            for (int e = 0; e < NC; ++e) alive[e] = alive[e] && cnt[e] + (R - NEED) >= NEED;
 #pragma unroll
             for (int j = NEED; j < R; ++j) {
-                if (alive[0] || alive[1] || alive[2] || alive[3]) {
-                    uint32_t hb[4];
-                    row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+                any = false;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
+                for (int e = 0; e < NC; ++e) any = any || alive[e];
+                if (any) {
+                    uint32_t hb[NC];
+                    row_hashes<POW2, NC>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+#pragma unroll
+                    for (int e = 0; e < NC; ++e) {
                         if (alive[e]) {
                             const float val = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
                             rowv[e][j] = val;
@@ -177,10 +184,10 @@ k_unsketch_pruned(const SparseArgs A) {
                 }
             }
         }
-        float m[4];
+        float m[NC];
         int ns = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < NC; ++e) {
             m[e] = 0.f;
             if (alive[e]) {
                 m[e] = median_of<R>(rowv[e]);
@@ -201,7 +208,7 @@ k_unsketch_pruned(const SparseArgs A) {
             wbase = __shfl_sync(0xFFFFFFFFu, wbase, 0);
             uint32_t pos = wbase + (uint32_t)(incl - ns);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
+            for (int e = 0; e < NC; ++e) {
                 if (alive[e]) {
                     if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)(i0 + e); A.sp.list_est[pos] = m[e]; }
                     ++pos;

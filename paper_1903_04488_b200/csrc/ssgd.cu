@@ -30,6 +30,15 @@
 #include "accum_tma.cuh"
 #include "estimate.cuh"
 #include "sparse_select.cuh"
+// Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
+// takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
+// second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
+#ifndef SSGD_PRUNED_GRID
+#define SSGD_PRUNED_GRID 4
+#endif
+#ifndef SSGD_K3_GRID
+#define SSGD_K3_GRID 4
+#endif
 
 namespace ssgd {
 
@@ -379,6 +388,7 @@ struct ssgd_ctx {
     size_t off_sp_hist, off_sp_state, off_bitmap, off_list_idx, off_list_est;   // sparse candidate path
     int64_t list_cap;
     int32_t prune_mode;
+    size_t persist_bytes;   // > 0: launches that touch the table carry an L2 access-policy window of this size
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;
     // device facts
@@ -493,19 +503,41 @@ bool pdl_enabled() {
     return on;
 }
 
+// An L2 access-policy window for one launch: accesses inside [base, base+bytes) are kept (persisting),
+// everything else the kernel touches is treated as streaming.
+struct L2Window { const void* base; size_t bytes; };
+
 template <typename... P, typename... A>
-cudaError_t launch_pdl(cudaStream_t st, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
+cudaError_t launch_pdl_w(cudaStream_t st, L2Window win, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3((unsigned)block);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute at[1];
-    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute at[2];
+    int n = 0;
+    if (pdl_enabled()) {
+        at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        at[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    if (win.base && win.bytes) {
+        at[n].id = cudaLaunchAttributeAccessPolicyWindow;
+        at[n].val.accessPolicyWindow.base_ptr = const_cast<void*>(win.base);
+        at[n].val.accessPolicyWindow.num_bytes = win.bytes;
+        at[n].val.accessPolicyWindow.hitRatio = 1.0f;
+        at[n].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
+        at[n].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
+        ++n;
+    }
     cfg.attrs = at;
-    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, kern, P(args)...);
+}
+
+template <typename... P, typename... A>
+cudaError_t launch_pdl(cudaStream_t st, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
+    return launch_pdl_w(st, L2Window{nullptr, 0}, kern, grid, block, smem, args...);
 }
 
 inline int grid_for(int64_t items, int threads, int64_t cap) {
@@ -527,7 +559,8 @@ int launch_accum_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
         k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, smem, st>>>(A);
     } else {
         const int grid = grid_for(groups, K1_THREADS, (int64_t)1 << 30);
-        CU(launch_pdl(st, k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
+        CU(launch_pdl_w(st, L2Window{MODE == INS_MERGED_GLOBAL ? A.table : nullptr, x->persist_bytes},
+                        k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
     }
     LAUNCHED("k_accum_insert");
     return SSGD_OK;
@@ -577,8 +610,8 @@ int launch_accum_tma_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
     }
     const int64_t ntiles = ((A.d & ~(int64_t)3) + KT_TC - 1) / KT_TC;
     const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->kt_blocks_per_sm);
-    CU(launch_pdl(st, kern, grid, KT_THREADS, smem, A, reinterpret_cast<int32_t*>(x->ws + x->off_err)),
-       "launch k_accum_insert_tma");
+    CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, kern, grid, KT_THREADS, smem, A,
+                    reinterpret_cast<int32_t*>(x->ws + x->off_err)), "launch k_accum_insert_tma");
     LAUNCHED("k_accum_insert_tma");
     return SSGD_OK;
 }
@@ -591,7 +624,7 @@ template <int R, bool POW2>
 int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     // a few blocks per SM: each block pays one histogram flush
-    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * 8);
+    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * SSGD_K3_GRID);
     CU(launch_pdl(st, k_unsketch<R, POW2>, grid, K3_THREADS, 0, A), "launch k_unsketch");
     LAUNCHED("k_unsketch");
     return SSGD_OK;
@@ -678,7 +711,8 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
     CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count), SEL_THREADS, 0, A),
        "launch k_unsketch_sample");
     LAUNCHED("k_unsketch_sample");
-    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, grid_for(groups, SEL_THREADS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, A),
+    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>,
+                  grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID), SEL_THREADS, 0, A),
        "launch k_unsketch_pruned");
     LAUNCHED("k_unsketch_pruned");
     return SSGD_OK;
@@ -776,7 +810,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->persist_bytes = 0;
     *out = x;
     return SSGD_OK;
 }
@@ -809,6 +843,24 @@ int ssgd_set_hash_params(ssgd_ctx* x, const uint32_t* in4r) {
         x->hp.row[j].a = in4r[4 * j]; x->hp.row[j].b = in4r[4 * j + 1];
         x->hp.row[j].a2 = in4r[4 * j + 2]; x->hp.row[j].b2 = in4r[4 * j + 3];
     }
+    return SSGD_OK;
+}
+
+int ssgd_set_table_persistence(ssgd_ctx* x, int32_t enable) {
+    if (!x) return SSGD_EINVAL;
+    x->persist_bytes = 0;
+    if (!enable) return SSGD_OK;
+    int e = ensure_device(x);
+    if (e) return e;
+    int max_persist = 0, max_window = 0;
+    CU(cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, x->device), "persisting L2 size");
+    CU(cudaDeviceGetAttribute(&max_window, cudaDevAttrMaxAccessPolicyWindowSize, x->device), "access window size");
+    size_t want = (size_t)x->r * x->c * 4;
+    if (want > (size_t)max_window) want = (size_t)max_window;
+    size_t carve = want < (size_t)max_persist ? want : (size_t)max_persist;
+    if (carve == 0) return SSGD_OK;
+    CU(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve), "set persisting L2 size");
+    x->persist_bytes = want;
     return SSGD_OK;
 }
 

@@ -29,6 +29,7 @@ SIGNATURES = {
     "ssgd_set_hash_params": [_vp, _vp],
     "ssgd_set_insert_mode": [_vp, _i32],
     "ssgd_set_prune_mode": [_vp, _i32],
+    "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
@@ -139,6 +140,9 @@ class Ssgd:
 
     def set_prune_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_prune_mode(self._h, mode), "ssgd_set_prune_mode")
+
+    def set_table_persistence(self, enable: bool) -> None:
+        self._chk(self._lib.ssgd_set_table_persistence(self._h, 1 if enable else 0), "ssgd_set_table_persistence")
 
     def step_used_fallback(self):
         """(fell back to the dense path?, survivors of the early exit, prune threshold bin) of the last step."""
