@@ -68,7 +68,8 @@ def test_workspace_bytes(lib):
     eng = S.Ssgd(d, r, c, k, W, 0)
     n = eng.workspace_bytes(100_000)
     floor = 4 * r * c + 4 * d + 8 * 100_000          # table + estimates + candidates and their sums
-    assert floor <= n <= floor + (1 << 20)
+    extra = d // 8 + 32 * 100_000                    # coordinate bitmap + survivor list of the early-exit path
+    assert floor + extra <= n <= floor + extra + (1 << 20)
     assert n % 256 == 0
     assert eng.workspace_bytes(200_000) > n
     for bad in (k - 1, d + 1):
@@ -93,11 +94,11 @@ def test_unbound_context_refuses_to_run(lib):
 
 def test_error_strings(lib):
     seen = set()
-    for code in range(0, -8, -1):
+    for code in range(0, -9, -1):
         s = lib.ssgd_strerror(code).decode()
         assert s and s != "unknown error"
         seen.add(s)
-    assert len(seen) == 8
+    assert len(seen) == 9
     assert lib.ssgd_strerror(-99).decode() == "unknown error"
 
 
