@@ -186,6 +186,24 @@ def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
         assert fell_back and bin_lo == 0 and survivors == cfg.d     # d equal magnitudes: the dense path ranks them
 
 
+def test_survivor_list_overflow_falls_back_to_the_dense_path(cuda_device):
+    """All estimates equal (zero): nothing can be pruned, the survivors (all d) do not fit the list, and the
+    gated dense path must produce the candidates; ties go to the smallest indices.  A normal gradient right
+    after it takes the pruned path again."""
+    cfg = wl.C2.scaled(d=300_001, W=2, c=1024, ncand=1000, k=500)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
+    fell_back, survivors, bin_lo = eng.step_used_fallback()
+    assert fell_back and survivors == cfg.d and bin_lo == 0
+    assert idx.tolist() == list(range(cfg.k))
+    st = wl.Structure(cfg, cuda_device)
+    check_step(orc, eng, wl.gradients(st, 0), cfg.rho, cfg.ncand, u_o, v_o)
+    assert not eng.step_used_fallback()[0]
+
+
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
 def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
