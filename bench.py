@@ -167,8 +167,19 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def communication(cfg):
+    """What one worker sends and receives per step, in values (Section 5.1: P*k + |S| + k), and the
+    compression factor 2d / (|S| + P*k + k) of Section 5.3 -- a property of the configuration, printed as context."""
+    sketch = cfg.r * cfg.c
+    per_worker = sketch + cfg.ncand + cfg.k
+    return {"sketch_values": sketch, "second_round_values": cfg.ncand, "update_values": cfg.k,
+            "per_worker_values": per_worker, "compression_vs_dense": 2.0 * cfg.d / per_worker}
+
+
 def workload_config(cfg, args):
     return {
+        "mode": getattr(args, "mode", "fused"),
+        "communication": communication(cfg),
         "workload": f"{cfg.name}: d={cfg.d}, W={cfg.W}, r={cfg.r}, c={cfg.c}, ncand={cfg.ncand}, k={cfg.k}, "
                     f"rho={cfg.rho}, {cfg.steps} resident gradient sets in rotation",
         "l2": "inputs larger than L2: every step streams 20*W*d bytes of g, u, v",
@@ -203,8 +214,23 @@ def run_ours(args, cfg):
     out_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
     out_val = torch.empty(cfg.k, dtype=torch.float32, device=dev)
 
+    if args.mode == "faithful":
+        # what the paper transmits: every worker's own sketch is materialised, then merged (Algorithm 3 lines 7-8)
+        tables = torch.empty((cfg.W, cfg.r, cfg.c), dtype=torch.float32, device=dev)
+        merged = torch.empty((cfg.r, cfg.c), dtype=torch.float32, device=dev)
+        cand = torch.empty(cfg.ncand, dtype=torch.int32, device=dev)
+
+        def one_step(g):
+            eng.sketch_accumulate(g, cfg.rho, tables)
+            eng.sketch_merge(tables, merged)
+            eng.unsketch_candidates(merged, cfg.ncand, cand)
+            eng.exact_topk(cand, out_idx, out_val)
+    else:
+        def one_step(g):
+            eng.step(g, cfg.rho, cfg.ncand, out_idx, out_val)
+
     for t in range(max(3, args.warmup)):
-        eng.step(g_sets[t % n_sets], cfg.rho, cfg.ncand, out_idx, out_val)
+        one_step(g_sets[t % n_sets])
     assert eng.status() == S.OK
     u.zero_(); v.zero_()
     torch.cuda.synchronize()
@@ -218,7 +244,7 @@ def run_ours(args, cfg):
     sampler.start()
     ev0.record()
     for t in range(args.steps):
-        eng.step(g_sets[t % n_sets], cfg.rho, cfg.ncand, out_idx, out_val)
+        one_step(g_sets[t % n_sets])
     ev1.record()
     torch.cuda.synchronize(); barrier()
     clocks = sampler.stop()
@@ -230,7 +256,7 @@ def run_ours(args, cfg):
     value, ms_step = rep.whole_job_value(cfg.W * cfg.d, ms_total / args.steps)
 
     # ---- end to end: host gradients in, host results out, through ssgd_step_host ------------------
-    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 20))
+    e2e_steps = 0 if (args.no_e2e or args.mode != "fused") else max(1, min(args.steps, 20))
     g_host = [g_sets[i % n_sets].cpu().pin_memory() for i in range(2 if e2e_steps else 0)]
     g_stage = torch.empty_like(g_sets[0])
     oi_h = torch.empty(cfg.k, dtype=torch.int32).pin_memory()
@@ -252,18 +278,19 @@ def run_ours(args, cfg):
 
     # ---- roofline of the dominant kernel and of the whole step -----------------------------------
     peak, peak_kind = peaks()
-    k1_ms = stage_ms[0] / max(1, stage_n)
+    split = stage_n > 0         # stage calls are not instrumented: no per-kernel split in faithful mode
+    k1_ms = stage_ms[0] / stage_n if split else None
     k1_bytes = 20.0 * cfg.W * cfg.d                       # g read; u, v read and written
-    k1_gbs = k1_bytes / (k1_ms * 1e-3) / 1e9
+    k1_gbs = k1_bytes / (k1_ms * 1e-3) / 1e9 if split else None
     step_bytes = (20.0 * cfg.W * cfg.d + 8.0 * cfg.r * cfg.c + 8.0 * cfg.d + 4.0 * cfg.W * cfg.ncand
                   + 8.0 * cfg.W * cfg.k + 8.0 * cfg.k)
     step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "k_accum_insert", "achieved": k1_gbs, "peak": peak, "unit": "GB/s",
-        "frac": k1_gbs / peak, "peak_source": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
+        "frac": k1_gbs / peak if split else None, "peak_source": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(cfg.name),
         "algorithmic_bytes_per_launch": k1_bytes, "ms_per_launch": k1_ms, "launches_timed": stage_n,
     }
-    breakdown = {n: (ms / max(1, stage_n)) for n, ms in
+    breakdown = {n: (ms / stage_n if split else None) for n, ms in
                  zip(("accumulate_insert_ms", "unsketch_ms", "select_candidates_ms", "second_round_topk_zero_ms"), stage_ms)}
 
     line = {
@@ -299,6 +326,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default="C2")
+    ap.add_argument("--mode", choices=["fused", "faithful"], default="fused",
+                    help="fused: ssgd_step; faithful: per-worker sketches materialised and merged (stage calls)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--d", type=int, default=0, help="override the number of coordinates (small profiling cases)")

@@ -68,7 +68,7 @@ extern "C" {
 /* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  With pruning, coordinates that
  * provably cannot be among the ncand largest |estimate| stop reading sketch rows early (a median of r
  * values reaches a magnitude only if (r+1)/2 of them do); the candidates are identical either way.
- * AUTO prunes when r >= 3, d >= 2^22 and ncand <= d/8 (below that the fixed costs outweigh the saving). */
+ * AUTO prunes when 5 <= r <= 9, d >= 2^22 and ncand <= d/8 (elsewhere the fixed costs outweigh the saving). */
 #define SSGD_PRUNE_AUTO 0
 #define SSGD_PRUNE_OFF  1
 #define SSGD_PRUNE_ON   2

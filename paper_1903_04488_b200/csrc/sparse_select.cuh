@@ -7,9 +7,9 @@
 //   * |median of r values| >= t  implies  at least (r+1)/2 of the r values have magnitude >= t.
 //     So once a coordinate cannot reach (r+1)/2 "big" row estimates any more, its remaining rows need
 //     not be read: it is certainly below t.
-//   * A safe t comes from a sample: k_unsketch_sample computes exact estimates for 1/32 of the
+//   * A safe t comes from a sample: k_unsketch_sample computes exact estimates for 1/64 of the
 //     float4 groups (pseudo-randomly placed), histograms them, and takes the histogram-bin edge `bin_lo`
-//     below which fewer than  ncand/32 + 6*sqrt(ncand/32) + 16  sampled estimates remain ... i.e. a
+//     below which fewer than  ncand/64 + 6*sqrt(ncand/64) + 16  sampled estimates remain ... i.e. a
 //     threshold the full vector exceeds at least ncand times except with negligible probability.
 //   * k_unsketch_pruned evaluates every coordinate with that early exit and appends the survivors
 //     (exact estimate in a bin >= bin_lo) to a compact list.  The survivor set does not depend on how the
@@ -31,7 +31,11 @@
 
 namespace ssgd {
 
-constexpr int SPARSE_SAMPLE_SHIFT = 5;            // one float4 group in 32 is sampled
+// measured at C2/C3/C4: 1/32 0.210/0.345/1.524 ms (sample + early-exit kernel), 1/64 0.207, 1/128 0.205, 1/256 0.208/0.338/1.467
+#ifndef SSGD_SAMPLE_SHIFT
+#define SSGD_SAMPLE_SHIFT 6
+#endif
+constexpr int SPARSE_SAMPLE_SHIFT = SSGD_SAMPLE_SHIFT;   // one float4 group in 2^shift is sampled
 constexpr int SPARSE_CLUSTER = 8;                 // CTAs in the selection cluster (portable maximum)
 constexpr int SPARSE_THREADS = 1024;
 constexpr int SPARSE_MAX_TIES = 2048;             // ties at the threshold handled in shared memory

@@ -54,7 +54,14 @@ C3 = Workload("C3", "block_laplace", 3, 20_000_000, 32, 5, 1_048_576, 200_000, 1
 C4 = Workload("C4", "embedding_mix", 4, 90_000_000, 16, 5, 4_194_304, 200_000, 100_000, 0.9, 5)
 C5 = tuple(C2.scaled(name=f"C5_W{w}", base_seed=5, W=w, steps=3) for w in (8, 32, 128, 256))
 
-CONFIGS = {w.name: w for w in (C1, C2, C3, C4) + C5}
+# The paper's own sketch shapes (Table 1 footnotes; 4 workers, k = 100,000), on the block-structured
+# Gaussian gradient model: 40x transformer run (15 x 180,000, P = 16), 20x transformer run (5 x 1,000,000,
+# P = 36) and the LSTM run (~73M parameters, 5 x 180,000, P = 26).
+P1 = Workload("P1", "block_gauss", 11, 90_000_000, 4, 15, 180_000, 1_600_000, 100_000, 0.9, 3)
+P2 = Workload("P2", "block_gauss", 12, 90_000_000, 4, 5, 1_000_000, 3_600_000, 100_000, 0.9, 3)
+P3 = Workload("P3", "block_gauss", 13, 73_000_000, 4, 5, 180_000, 2_600_000, 100_000, 0.9, 3)
+
+CONFIGS = {w.name: w for w in (C1, C2, C3, C4) + C5 + (P1, P2, P3)}
 
 
 def structure_seed(cfg: Workload) -> int:
