@@ -3,4 +3,4 @@
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
 It shares no code with the CUDA library and never imports it.
 """
-from .ssgd_oracle import Oracle, build, derive_params, select  # noqa: F401
+from .ssgd_oracle import Oracle, build, derive_params, fill_priority, select  # noqa: F401

@@ -303,4 +303,92 @@ int ssgd_oracle_step(const ssgd_oracle_ctx* ctx, const float* g, int64_t ld_g, f
     return 0;
 }
 
+// ---- Algorithm 1 (HEAVYMIX) ---------------------------------------------------------------------------
+
+int ssgd_oracle_fill_priority(uint64_t seed, int64_t n, const int64_t* idx, uint32_t* out) {
+    if (n < 0 || (n > 0 && (!idx || !out))) return -1;
+    for (int64_t t = 0; t < n; ++t) {
+        uint64_t z = seed + ((uint64_t)idx[t] + 1ULL) * 0x9E3779B97F4A7C15ULL;
+        z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
+        z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
+        z ^= z >> 31;
+        out[t] = (uint32_t)(z >> 32);
+    }
+    return 0;
+}
+
+int ssgd_oracle_l2_estimate(const ssgd_oracle_ctx* ctx, const float* Tf, double* l2_out) {
+    const Ctx* x = C(ctx);
+    if (!x || !Tf || !l2_out) return -1;
+    double rows[SSGD_ORACLE_MAX_R];
+    for (int j = 0; j < x->r; ++j) {
+        double s = 0.0;
+        for (int64_t b = 0; b < x->c; ++b) {
+            const double t = (double)Tf[(int64_t)j * x->c + b];
+            s += t * t;
+        }
+        rows[j] = s;
+    }
+    // median over the rows (r is odd): insertion sort, middle element
+    for (int p = 1; p < x->r; ++p) {
+        const double key = rows[p];
+        int q = p - 1;
+        while (q >= 0 && rows[q] > key) { rows[q + 1] = rows[q]; --q; }
+        rows[q + 1] = key;
+    }
+    *l2_out = rows[x->r / 2];
+    return 0;
+}
+
+int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const float* v, int64_t ld,
+                         uint64_t fill_seed, int32_t* out_idx, float* out_val, double* l2_out,
+                         int64_t* nheavy_out) {
+    const Ctx* x = C(ctx);
+    if (!x || !Tf || !v || !out_idx || !out_val || ld < x->d) return -1;
+    int e;
+    // line 1
+    double l2 = 0.0;
+    if ((e = ssgd_oracle_l2_estimate(ctx, Tf, &l2))) return e;
+    if (l2_out) *l2_out = l2;
+    // line 2
+    std::vector<float> est((size_t)x->d);
+    if ((e = ssgd_oracle_estimate(ctx, Tf, est.data()))) return e;
+    // line 3
+    const double thr = l2 / (double)x->k;
+    std::vector<int32_t> H, NH;
+    for (int64_t i = 0; i < x->d; ++i) {
+        const double g2 = (double)est[(size_t)i] * (double)est[(size_t)i];
+        (g2 >= thr ? H : NH).push_back((int32_t)i);
+    }
+    if (nheavy_out) *nheavy_out = (int64_t)H.size();
+    // line 4
+    std::vector<int32_t> top;
+    if ((int64_t)H.size() <= x->k) {
+        top = H;
+        const int64_t l = x->k - (int64_t)H.size();
+        std::vector<int64_t> nh64(NH.begin(), NH.end());
+        std::vector<uint32_t> prio(NH.size());
+        if ((e = ssgd_oracle_fill_priority(fill_seed, (int64_t)NH.size(), nh64.data(), prio.data()))) return e;
+        std::vector<int64_t> order(NH.size());
+        for (size_t t = 0; t < NH.size(); ++t) order[t] = (int64_t)t;
+        std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+            if (prio[(size_t)a] != prio[(size_t)b]) return prio[(size_t)a] > prio[(size_t)b];
+            return NH[(size_t)a] < NH[(size_t)b];
+        });
+        for (int64_t t = 0; t < l; ++t) top.push_back(NH[(size_t)order[(size_t)t]]);
+    } else {
+        std::vector<float> hv(H.size());
+        for (size_t t = 0; t < H.size(); ++t) hv[t] = est[(size_t)H[t]];
+        std::vector<int32_t> best((size_t)x->k);
+        if ((e = ssgd_oracle_select((int64_t)H.size(), hv.data(), H.data(), x->k, best.data()))) return e;
+        for (int64_t t = 0; t < x->k; ++t) top.push_back(H[(size_t)best[(size_t)t]]);
+    }
+    std::sort(top.begin(), top.end());
+    // line 5
+    std::vector<double> xs((size_t)x->k);
+    if ((e = ssgd_oracle_second_round(ctx, v, ld, top.data(), x->k, xs.data()))) return e;
+    for (int64_t t = 0; t < x->k; ++t) { out_idx[t] = top[(size_t)t]; out_val[t] = (float)xs[(size_t)t]; }
+    return 0;
+}
+
 }  // extern "C"

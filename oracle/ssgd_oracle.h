@@ -1,7 +1,7 @@
 /*
  * ssgd_oracle.h -- plain, slow, single-threaded CPU statement of one Sketched-SGD
  * compression step (Algorithm 3 "Empirical Training", lines 5-13, with the Count
- * Sketch of Algorithm 4).
+ * Sketch of Algorithm 4), and of the HEAVYMIX selection rule (Algorithm 1).
  *
  * THIS IS TEST INFRASTRUCTURE.  It exists so that the CUDA library can be checked
  * against something written directly from the paper.  It shares no code with the
@@ -105,6 +105,30 @@ int ssgd_oracle_step(const ssgd_oracle_ctx* ctx, const float* g, int64_t ld_g, f
                      int32_t* out_idx, float* out_val,
                      double* T_out, double* M_out, float* est_out,
                      int32_t* cand_out, double* xs_out, int32_t zero_state);
+
+/* ---- Algorithm 1 (HEAVYMIX): the selection rule the paper's theory covers ---------------------------
+ *
+ * Per-coordinate priority of the random fill: a 64-bit mix of (seed, i),
+ *   z = seed + (i+1)*0x9E3779B97F4A7C15;  z = (z^(z>>30))*0xBF58476D1CE4E5B9;
+ *   z = (z^(z>>27))*0x94D049BB133111EB;   z ^= z>>31;   priority = upper 32 bits of z.
+ * The l coordinates of NH with the largest priority (ties: smaller index) are a uniformly random
+ * l-subset of NH for a random seed: that is the reading of "rand_l(NH)" taken here. */
+int ssgd_oracle_fill_priority(uint64_t seed, int64_t n, const int64_t* idx, uint32_t* out);
+
+/* Line 1: the squared-norm estimate of the sketched vector, median over rows j of sum_b Tf[j][b]^2
+ * (each row is an AMS-type estimator, Appendix B), accumulated in fp64 in bucket order. */
+int ssgd_oracle_l2_estimate(const ssgd_oracle_ctx* ctx, const float* Tf, double* l2_out);
+
+/* Lines 1-5 on an fp32 [r][c] table Tf:
+ *   l2 = ssgd_oracle_l2_estimate;  est = ssgd_oracle_estimate;
+ *   H  = { i : (double)est_i^2 >= l2/k }           (line 3, read with the square its proof uses)
+ *   if |H| <= k:  Top = H  +  the k-|H| coordinates of NH with the largest fill priority
+ *   else:         Top = the k coordinates of H with the largest |est| (ties: smaller index)
+ *   out_val[t] = (float) sum over w = 0..W-1 of v_w[out_idx[t]]   (line 5, fp64 in worker order)
+ * out_idx is ascending.  nheavy_out receives |H|.  The state is not modified. */
+int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const float* v, int64_t ld,
+                         uint64_t fill_seed, int32_t* out_idx, float* out_val, double* l2_out,
+                         int64_t* nheavy_out);
 
 #ifdef __cplusplus
 }

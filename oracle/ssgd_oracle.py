@@ -55,6 +55,9 @@ def _load():
                 "ssgd_oracle_second_round": [vp, vp, i64, vp, i64, vp],
                 "ssgd_oracle_zero": [vp, vp, vp, i64, vp, i64],
                 "ssgd_oracle_step": [vp, vp, i64, f32, vp, vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, i32],
+                "ssgd_oracle_fill_priority": [u64, i64, vp, vp],
+                "ssgd_oracle_l2_estimate": [vp, vp, vp],
+                "ssgd_oracle_heavymix": [vp, vp, vp, i64, u64, vp, vp, vp, vp],
             }
             for name, args in sig.items():
                 fn = getattr(lib, name)
@@ -95,6 +98,14 @@ def select(val: np.ndarray, m: int, ids: np.ndarray | None = None) -> np.ndarray
         ids = _chk(np.ascontiguousarray(ids, np.int32), np.int32, "ids")
     out = np.zeros(m, np.int32)
     _ok(_load().ssgd_oracle_select(val.size, _ptr(val), _ptr(ids), m, _ptr(out)), "select")
+    return out
+
+
+def fill_priority(seed: int, idx) -> np.ndarray:
+    """Random-fill priorities of HEAVYMIX (Algorithm 1 line 4) for the listed coordinates."""
+    idx = np.ascontiguousarray(idx, np.int64)
+    out = np.zeros(idx.size, np.uint32)
+    _ok(_load().ssgd_oracle_fill_priority(seed, idx.size, _ptr(idx), _ptr(out)), "fill_priority")
     return out
 
 
@@ -220,3 +231,23 @@ class Oracle:
                                        ncand, _ptr(out_idx), _ptr(out_val), _ptr(T), _ptr(M), _ptr(est),
                                        _ptr(cand), _ptr(xs), 1 if zero_state else 0), "step")
         return dict(out_idx=out_idx, out_val=out_val, T=T, M=M, est=est, cand=cand, xs=xs)
+
+    # ---- Algorithm 1 (HEAVYMIX) --------------------------------------------------------------------
+    def l2_estimate(self, Tf) -> float:
+        """Line 1: median over rows of the row's sum of squares."""
+        Tf = _chk(np.ascontiguousarray(Tf, np.float32), np.float32, "Tf")
+        out = C.c_double()
+        _ok(self._lib.ssgd_oracle_l2_estimate(self._h, _ptr(Tf), C.byref(out)), "l2_estimate")
+        return out.value
+
+    def heavymix(self, Tf, v, fill_seed):
+        """Lines 1-5: dict(out_idx ascending, out_val, l2, nheavy)."""
+        Tf = _chk(np.ascontiguousarray(Tf, np.float32), np.float32, "Tf")
+        self._state(v, "v")
+        out_idx = np.zeros(self.k, np.int32)
+        out_val = np.zeros(self.k, np.float32)
+        l2 = C.c_double()
+        nh = C.c_int64()
+        _ok(self._lib.ssgd_oracle_heavymix(self._h, _ptr(Tf), _ptr(v), v.shape[1], fill_seed, _ptr(out_idx),
+                                           _ptr(out_val), C.byref(l2), C.byref(nh)), "heavymix")
+        return dict(out_idx=out_idx, out_val=out_val, l2=l2.value, nheavy=nh.value)
