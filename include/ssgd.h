@@ -136,6 +136,21 @@ int ssgd_exact_topk(ssgd_ctx* ctx, const int32_t* cand_idx, int64_t ncand, int32
 int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t ncand,
               int32_t* out_idx, float* out_val, void* stream);
 
+/* Algorithm 1 (HEAVYMIX), the selection rule of the paper's analysis, on a merged [r][c] table (device):
+ *   line 1  l2 = median over rows of the row's sum of squared counters (fp64)
+ *   line 3  H = { i : est_i^2 >= l2 / k }, est the median-of-r estimate, compared in fp64
+ *   line 4  Top_k = H plus a uniformly random (k - |H|)-subset of the other coordinates: every coordinate has
+ *           a 30-bit priority mixed from (fill_seed, i) -- z = fill_seed + (i+1)*0x9E3779B97F4A7C15,
+ *           z = (z^(z>>30))*0xBF58476D1CE4E5B9, z = (z^(z>>27))*0x94D049BB133111EB, z ^= z>>31, priority = z>>34
+ *           -- and the non-heavy coordinates with the largest priorities are taken (ties: smaller index).
+ *           Should more than k coordinates be heavy (outside the paper's guarantee), the k with the largest
+ *           |est| (compared without the last mantissa bit) are kept.
+ *   line 5  out_val[t] = sum over the workers of the bound v at out_idx[t] (fp64, worker order).
+ * out_idx / out_val: [k] device outputs, ascending coordinate order.  l2_out (device double) and nheavy_out
+ * (device int32) are optional.  The bound state is read, not modified.  Asynchronous on `stream`. */
+int ssgd_heavymix(ssgd_ctx* ctx, const float* merged, uint64_t fill_seed, int32_t* out_idx, float* out_val,
+                  double* l2_out, int32_t* nheavy_out, void* stream);
+
 /* The same step for a caller whose gradients and results live in HOST memory: copies g_host
  * ([W][ld_g] fp32; pinned memory makes the copy asynchronous) into g_stage (device, [W][ld_g]),
  * runs ssgd_step, copies the k results back to out_idx_host/out_val_host and waits for the stream. */

@@ -312,7 +312,7 @@ int ssgd_oracle_fill_priority(uint64_t seed, int64_t n, const int64_t* idx, uint
         z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ULL;
         z = (z ^ (z >> 27)) * 0x94D049BB133111EBULL;
         z ^= z >> 31;
-        out[t] = (uint32_t)(z >> 32);
+        out[t] = (uint32_t)(z >> 34);  // upper 30 bits
     }
     return 0;
 }
@@ -361,28 +361,26 @@ int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const floa
         (g2 >= thr ? H : NH).push_back((int32_t)i);
     }
     if (nheavy_out) *nheavy_out = (int64_t)H.size();
-    // line 4
-    std::vector<int32_t> top;
-    if ((int64_t)H.size() <= x->k) {
-        top = H;
-        const int64_t l = x->k - (int64_t)H.size();
-        std::vector<int64_t> nh64(NH.begin(), NH.end());
-        std::vector<uint32_t> prio(NH.size());
-        if ((e = ssgd_oracle_fill_priority(fill_seed, (int64_t)NH.size(), nh64.data(), prio.data()))) return e;
-        std::vector<int64_t> order(NH.size());
-        for (size_t t = 0; t < NH.size(); ++t) order[t] = (int64_t)t;
-        std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
-            if (prio[(size_t)a] != prio[(size_t)b]) return prio[(size_t)a] > prio[(size_t)b];
-            return NH[(size_t)a] < NH[(size_t)b];
-        });
-        for (int64_t t = 0; t < l; ++t) top.push_back(NH[(size_t)order[(size_t)t]]);
-    } else {
-        std::vector<float> hv(H.size());
-        for (size_t t = 0; t < H.size(); ++t) hv[t] = est[(size_t)H[t]];
-        std::vector<int32_t> best((size_t)x->k);
-        if ((e = ssgd_oracle_select((int64_t)H.size(), hv.data(), H.data(), x->k, best.data()))) return e;
-        for (int64_t t = 0; t < x->k; ++t) top.push_back(H[(size_t)best[(size_t)t]]);
+    // line 4: Top_k = H + rand_l(NH).  One ordering expresses it: heavy coordinates come first (among
+    // themselves by magnitude), the others in the order of their fill priority; the k first are taken.
+    std::vector<uint32_t> key((size_t)x->d);
+    {
+        std::vector<int64_t> all((size_t)x->d);
+        for (int64_t i = 0; i < x->d; ++i) all[(size_t)i] = i;
+        std::vector<uint32_t> prio((size_t)x->d);
+        if ((e = ssgd_oracle_fill_priority(fill_seed, x->d, all.data(), prio.data()))) return e;
+        for (int64_t i = 0; i < x->d; ++i) {
+            const double g2 = (double)est[(size_t)i] * (double)est[(size_t)i];
+            key[(size_t)i] = g2 >= thr ? (0x40000000u | (abs_bits(est[(size_t)i]) >> 1)) : prio[(size_t)i];
+        }
     }
+    std::vector<int32_t> order((size_t)x->d);
+    for (int64_t i = 0; i < x->d; ++i) order[(size_t)i] = (int32_t)i;
+    std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+        if (key[(size_t)a] != key[(size_t)b]) return key[(size_t)a] > key[(size_t)b];
+        return a < b;
+    });
+    std::vector<int32_t> top(order.begin(), order.begin() + x->k);
     std::sort(top.begin(), top.end());
     // line 5
     std::vector<double> xs((size_t)x->k);

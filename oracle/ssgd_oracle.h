@@ -110,7 +110,7 @@ int ssgd_oracle_step(const ssgd_oracle_ctx* ctx, const float* g, int64_t ld_g, f
  *
  * Per-coordinate priority of the random fill: a 64-bit mix of (seed, i),
  *   z = seed + (i+1)*0x9E3779B97F4A7C15;  z = (z^(z>>30))*0xBF58476D1CE4E5B9;
- *   z = (z^(z>>27))*0x94D049BB133111EB;   z ^= z>>31;   priority = upper 32 bits of z.
+ *   z = (z^(z>>27))*0x94D049BB133111EB;   z ^= z>>31;   priority = upper 30 bits of z.
  * The l coordinates of NH with the largest priority (ties: smaller index) are a uniformly random
  * l-subset of NH for a random seed: that is the reading of "rand_l(NH)" taken here. */
 int ssgd_oracle_fill_priority(uint64_t seed, int64_t n, const int64_t* idx, uint32_t* out);
@@ -122,8 +122,12 @@ int ssgd_oracle_l2_estimate(const ssgd_oracle_ctx* ctx, const float* Tf, double*
 /* Lines 1-5 on an fp32 [r][c] table Tf:
  *   l2 = ssgd_oracle_l2_estimate;  est = ssgd_oracle_estimate;
  *   H  = { i : (double)est_i^2 >= l2/k }           (line 3, read with the square its proof uses)
- *   if |H| <= k:  Top = H  +  the k-|H| coordinates of NH with the largest fill priority
- *   else:         Top = the k coordinates of H with the largest |est| (ties: smaller index)
+ *   Top = the k first coordinates when heavy ones are put first and the others follow by fill priority:
+ *         key(i) = 2^30 + floor(bits(|est_i|) / 2)  if i is in H,  else  priority(i)  (< 2^30);
+ *         larger key first, ties to the smaller index.
+ *         For |H| <= k that is H plus a random (k-|H|)-subset of NH (line 4).  |H| > k lies outside the
+ *         paper's guarantee and its line 4; the same ordering then keeps the k heavy coordinates with
+ *         the largest estimates (magnitudes compared without their last mantissa bit).
  *   out_val[t] = (float) sum over w = 0..W-1 of v_w[out_idx[t]]   (line 5, fp64 in worker order)
  * out_idx is ascending.  nheavy_out receives |H|.  The state is not modified. */
 int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const float* v, int64_t ld,

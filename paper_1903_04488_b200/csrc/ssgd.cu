@@ -30,6 +30,7 @@
 #include "accum_tma.cuh"
 #include "estimate.cuh"
 #include "sparse_select.cuh"
+#include "heavymix.cuh"
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
@@ -387,6 +388,7 @@ struct ssgd_ctx {
     size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
     size_t off_sp_hist, off_sp_state, off_bitmap, off_list_idx, off_list_est;   // sparse candidate path
     int64_t list_cap;
+    size_t off_hm;
     int32_t prune_mode;
     size_t persist_bytes;   // > 0: launches that touch the table carry an L2 access-policy window of this size
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
@@ -437,6 +439,7 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_sp_hist = o; o += up(2 * H1_BINS * 4);
     x->off_sp_state = o; o += up(sizeof(SparseState));
     x->off_bitmap = o;  o += up((size_t)((x->d + 31) / 32) * 4);
+    x->off_hm = o;      o += up(sizeof(HeavymixState));
     x->off_err = o;     o += up(16);
     x->zero_bytes = o;
     x->nchunk_c = (x->d + SEL_CHUNK - 1) / SEL_CHUNK;
@@ -791,6 +794,18 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
+template <int R, bool POW2>
+int launch_heavymix_keys_t(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    k_heavymix_keys<R, POW2><<<grid_for(groups, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, st>>>(A);
+    LAUNCHED("k_heavymix_keys");
+    return SSGD_OK;
+}
+
+int launch_heavymix_keys(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_heavymix_keys_t, x, A, st)
+}
+
 }  // namespace
 
 extern "C" {
@@ -1026,6 +1041,48 @@ int ssgd_get_stage_times(ssgd_ctx* x, void* stream, double* ms_out, int64_t* ste
         }
     *steps_out = x->ev_steps;
     x->ev_steps = 0;
+    return SSGD_OK;
+}
+
+int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t* out_idx, float* out_val,
+                  double* l2_out, int32_t* nheavy_out, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!merged || !out_idx || !out_val) return SSGD_EINVAL;
+    if ((e = ensure_device(x))) return e;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // histograms + state of the candidate selection, and the HEAVYMIX state
+    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->off_hist_f - x->off_hist_c, st), "memset hist");
+    CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_sp_hist - x->off_hist_f, st), "memset hist");
+    CU(cudaMemsetAsync(x->ws + x->off_hm, 0, sizeof(HeavymixState), st), "memset heavymix state");
+    x->launches += 3;
+    HeavymixArgs A;
+    A.table = merged; A.c = x->c; A.d = x->d; A.r = x->r; A.hp = x->hp; A.bk = x->bk;
+    A.hm = reinterpret_cast<HeavymixState*>(x->ws + x->off_hm);
+    A.keys = reinterpret_cast<float*>(x->ws + x->off_est);
+    A.sb = sel_buffers(x, false);
+    A.k = (uint32_t)x->k;
+    A.fill_seed = fill_seed;
+    dim3 grid((unsigned)grid_for(x->c, 256, x->sm_count * 2), (unsigned)x->r);
+    k_row_sumsq<<<grid, 256, 0, st>>>(merged, x->c, A.hm);
+    LAUNCHED("k_row_sumsq");
+    if ((e = launch_heavymix_keys(x, A, st))) return e;
+    if ((e = launch_select(x, A.keys, x->d, A.sb, x->nchunk_c, st))) return e;
+    CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)A.keys,
+                  x->d, A.sb, out_idx, (float*)nullptr, (uint32_t)x->k, x->nchunk_c), "launch k_emit_candidates");
+    LAUNCHED("k_emit_candidates");
+    // line 5: exact values of the chosen coordinates, summed over the workers
+    SelBuffers sf = sel_buffers(x, true);
+    CU(launch_pdl(st, k_gather, grid_for(x->k, 256, (int64_t)1 << 30), 256, 0, (const int32_t*)out_idx, x->k, (const float*)x->v,
+                  x->ld, x->W, x->d, out_val, sf, (uint32_t)1, reinterpret_cast<int32_t*>(x->ws + x->off_err)),
+       "launch k_gather");
+    LAUNCHED("k_gather");
+    if (l2_out || nheavy_out) {
+        // l2 = median of the row sums: computed on the host side of the copy-out by the caller would need a
+        // sync; instead one thread writes both results
+        k_heavymix_report<<<1, 32, 0, st>>>(A.hm, x->r, l2_out, nheavy_out);
+        LAUNCHED("k_heavymix_report");
+    }
     return SSGD_OK;
 }
 

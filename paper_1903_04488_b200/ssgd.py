@@ -39,6 +39,7 @@ SIGNATURES = {
     "ssgd_exact_topk": [_vp, _vp, _i64, _vp, _vp, _vp],
     "ssgd_step": [_vp, _vp, _i64, _f32, _i64, _vp, _vp, _vp],
     "ssgd_step_host": [_vp, _vp, _i64, _f32, _i64, _vp, _vp, _vp, _vp],
+    "ssgd_heavymix": [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _vp],
     "ssgd_step_buffers": [_vp, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp)],
     "ssgd_hashes": [_vp, _vp, _i64, _vp, _vp, _vp],
     "ssgd_exact_topk_static": [_vp, _i64, _i32, _i64, _vp, _i64, _i64, _vp, _vp, _vp],
@@ -211,6 +212,15 @@ class Ssgd:
         self._chk(self._lib.ssgd_step(self._h, _dev_ptr(g, torch.float32, "g"), g.shape[1], rho, ncand,
                                       _dev_ptr(out_idx, torch.int32, "out_idx"),
                                       _dev_ptr(out_val, torch.float32, "out_val"), _stream()), "ssgd_step")
+
+    def heavymix(self, merged: torch.Tensor, fill_seed: int, out_idx: torch.Tensor, out_val: torch.Tensor,
+                 l2_out: torch.Tensor | None = None, nheavy_out: torch.Tensor | None = None) -> None:
+        """Algorithm 1 on a merged table: k coordinates (heavy ones + seeded random fill) and their exact sums."""
+        self._chk(self._lib.ssgd_heavymix(self._h, _dev_ptr(merged, torch.float32, "merged"), fill_seed,
+                                          _dev_ptr(out_idx, torch.int32, "out_idx"),
+                                          _dev_ptr(out_val, torch.float32, "out_val"),
+                                          _dev_ptr(l2_out, torch.float64, "l2_out"),
+                                          _dev_ptr(nheavy_out, torch.int32, "nheavy_out"), _stream()), "ssgd_heavymix")
 
     def step_host(self, g_host: torch.Tensor, rho: float, ncand: int, g_stage: torch.Tensor,
                   out_idx_host: torch.Tensor, out_val_host: torch.Tensor) -> None:

@@ -14,7 +14,7 @@ def py_priority(seed, i):
     z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & M64
     z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & M64
     z ^= z >> 31
-    return z >> 32
+    return z >> 34
 
 
 def test_fill_priority_matches_big_integers():
