@@ -3,4 +3,5 @@
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
 It shares no code with the CUDA library and never imports it.
 """
-from .ssgd_oracle import Oracle, build, derive_params, fill_priority, select  # noqa: F401
+from .ssgd_oracle import (FMT_BF16, FMT_F16, Oracle, build, derive_params, fill_priority, merge16,  # noqa: F401
+                          quantize16, select)

@@ -389,4 +389,69 @@ int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const floa
     return 0;
 }
 
+// ---- 16-bit sketches ------------------------------------------------------------------------------------
+
+namespace {
+inline uint32_t f32_bits(float f) { uint32_t u; std::memcpy(&u, &f, 4); return u; }
+inline float bits_f32(uint32_t u) { float f; std::memcpy(&f, &u, 4); return f; }
+
+// fp32 -> bfloat16, round to nearest, ties to even (finite input)
+inline uint16_t to_bf16(float f) {
+    const uint32_t u = f32_bits(f);
+    const uint32_t lsb = (u >> 16) & 1u;
+    return (uint16_t)((u + 0x7FFFu + lsb) >> 16);
+}
+inline float from_bf16(uint16_t h) { return bits_f32((uint32_t)h << 16); }
+
+// fp32 -> binary16, round to nearest even, saturating at the largest finite value
+inline uint16_t to_f16(float f) {
+    const uint32_t u = f32_bits(f);
+    const uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    const float a = std::fabs(f);
+    if (a >= 65520.0f) return (uint16_t)(sign | 0x7BFFu);          // would round to infinity: saturate to 65504
+    if (a < 5.9604644775390625e-8f * 0.5f) return sign;            // below half the smallest subnormal: zero
+    // scale into the binary16 grid and round with the fp32 adder (exact: a * 2^k is exact, + magic rounds RNE)
+    int e;
+    std::frexp(a, &e);                                              // a = m * 2^e, m in [0.5, 1)
+    const int exp16 = e - 1;                                        // unbiased exponent of a
+    const int q = exp16 < -14 ? -24 : exp16 - 10;                   // quantum 2^q (subnormals share 2^-24)
+    const double scaled = std::ldexp((double)a, -q);                // a / 2^q, exact in fp64
+    const double r = std::nearbyint(scaled);                        // ties to even (default rounding mode)
+    const double back = std::ldexp(r, q);                           // the binary16 value
+    // encode
+    int e2;
+    const double m2 = std::frexp(back, &e2);                        // back = m2 * 2^e2
+    (void)m2;
+    const int ex = e2 - 1;
+    if (back == 0.0) return sign;
+    if (ex < -14) return (uint16_t)(sign | (uint16_t)std::ldexp(back, 24));                  // subnormal
+    const uint32_t mant = (uint32_t)std::ldexp(back, 10 - ex) - 1024u;
+    return (uint16_t)(sign | ((uint32_t)(ex + 15) << 10) | mant);
+}
+inline float from_f16(uint16_t h) {
+    const int sign = (h >> 15) & 1, ex = (h >> 10) & 31, mant = h & 1023;
+    double v = ex == 0 ? std::ldexp((double)mant, -24) : std::ldexp((double)(1024 + mant), ex - 25);
+    return (float)(sign ? -v : v);
+}
+}  // namespace
+
+int ssgd_oracle_quantize16(int64_t n, const float* x, int32_t fmt, uint16_t* q16) {
+    if (n < 0 || (n > 0 && (!x || !q16)) || (fmt != 0 && fmt != 1)) return -1;
+    for (int64_t t = 0; t < n; ++t) q16[t] = fmt == 0 ? to_f16(x[t]) : to_bf16(x[t]);
+    return 0;
+}
+
+int ssgd_oracle_merge16(int32_t W, int64_t n, const uint16_t* q16, int32_t fmt, float* out) {
+    if (W < 1 || n < 0 || (n > 0 && (!q16 || !out)) || (fmt != 0 && fmt != 1)) return -1;
+    for (int64_t t = 0; t < n; ++t) {
+        float acc = 0.0f;
+        for (int w = 0; w < W; ++w) {
+            const uint16_t h = q16[(int64_t)w * n + t];
+            acc = acc + (fmt == 0 ? from_f16(h) : from_bf16(h));
+        }
+        out[t] = acc;
+    }
+    return 0;
+}
+
 }  // extern "C"

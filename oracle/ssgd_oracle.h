@@ -134,6 +134,15 @@ int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const floa
                          uint64_t fill_seed, int32_t* out_idx, float* out_val, double* l2_out,
                          int64_t* nheavy_out);
 
+/* ---- 16-bit sketches (Section 6: "quantizing sketches to 16 bits") ------------------------------------
+ * What a worker would transmit: its fp32 sketch rounded to a 16-bit format, round-to-nearest-even.
+ * fmt 0: IEEE binary16 (values beyond +-65504 saturate to +-65504); fmt 1: bfloat16 (upper 16 bits of fp32).
+ * q16 receives the n encodings.  Inputs must be finite. */
+int ssgd_oracle_quantize16(int64_t n, const float* x, int32_t fmt, uint16_t* q16);
+/* The server's merge of W quantised sketches: out[t] = sum over w = 0..W-1, in that order, in fp32, of the
+ * decoded q16[w][t]; q16 is [W][n]. */
+int ssgd_oracle_merge16(int32_t W, int64_t n, const uint16_t* q16, int32_t fmt, float* out);
+
 #ifdef __cplusplus
 }
 #endif

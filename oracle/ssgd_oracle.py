@@ -58,6 +58,8 @@ def _load():
                 "ssgd_oracle_fill_priority": [u64, i64, vp, vp],
                 "ssgd_oracle_l2_estimate": [vp, vp, vp],
                 "ssgd_oracle_heavymix": [vp, vp, vp, i64, u64, vp, vp, vp, vp],
+                "ssgd_oracle_quantize16": [i64, vp, i32, vp],
+                "ssgd_oracle_merge16": [i32, i64, vp, i32, vp],
             }
             for name, args in sig.items():
                 fn = getattr(lib, name)
@@ -106,6 +108,26 @@ def fill_priority(seed: int, idx) -> np.ndarray:
     idx = np.ascontiguousarray(idx, np.int64)
     out = np.zeros(idx.size, np.uint32)
     _ok(_load().ssgd_oracle_fill_priority(seed, idx.size, _ptr(idx), _ptr(out)), "fill_priority")
+    return out
+
+
+FMT_F16, FMT_BF16 = 0, 1
+
+
+def quantize16(x, fmt: int) -> np.ndarray:
+    """fp32 -> 16-bit encodings (uint16), round to nearest even; fmt 0 = binary16 (saturating), 1 = bfloat16."""
+    x = np.ascontiguousarray(x, np.float32)
+    q = np.zeros(x.shape, np.uint16)
+    _ok(_load().ssgd_oracle_quantize16(x.size, _ptr(x), fmt, _ptr(q)), "quantize16")
+    return q
+
+
+def merge16(q16, fmt: int) -> np.ndarray:
+    """[W][...] uint16 encodings -> fp32 sum over the first axis, in worker order."""
+    q16 = np.ascontiguousarray(q16, np.uint16)
+    W = q16.shape[0]
+    out = np.zeros(q16.shape[1:], np.float32)
+    _ok(_load().ssgd_oracle_merge16(W, out.size, _ptr(q16), fmt, _ptr(out)), "merge16")
     return out
 
 
