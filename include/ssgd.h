@@ -115,6 +115,16 @@ int ssgd_sketch_accumulate(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rh
  * of tables[w][j][b].  merged is [r][c] fp32, device. */
 int ssgd_sketch_merge(ssgd_ctx* ctx, const float* tables, float* merged, void* stream);
 
+/* 16-bit sketches (Section 6: quantising sketches to 16 bits).  ssgd_sketch_quantize16 rounds the W per-worker
+ * tables ([W][r][c] fp32, device) to a 16-bit format, round-to-nearest-even -- SSGD_FMT_F16: IEEE binary16,
+ * magnitudes beyond 65504 saturate; SSGD_FMT_BF16: bfloat16 -- into q16 ([W][r][c] uint16, device): what each
+ * worker would transmit.  ssgd_sketch_merge16 is the server side: merged[j][b] = sum over w = 0..W-1, in that
+ * order, in fp32, of the decoded q16[w][j][b].  The rest of the pipeline runs on `merged` unchanged. */
+#define SSGD_FMT_F16  0
+#define SSGD_FMT_BF16 1
+int ssgd_sketch_quantize16(ssgd_ctx* ctx, const float* tables, int32_t fmt, uint16_t* q16, void* stream);
+int ssgd_sketch_merge16(ssgd_ctx* ctx, const uint16_t* q16, int32_t fmt, float* merged, void* stream);
+
 /* Algorithm 3 line 9 (Algorithm 4 estimate for every coordinate, Section 5.2): computes est[i] for
  * all i < d from merged ([r][c] fp32, device) and writes the ncand coordinates with the largest
  * |est| to cand_idx ([ncand] int32, device), in ASCENDING coordinate order.  cand_est ([ncand] fp32)

@@ -13,6 +13,8 @@
 //   k_zero              line 13: u = v = 0 at the chosen coordinates.
 // HBM-bound work is the first kernel (20 bytes per worker-coordinate); nothing here is a dense
 // contraction, so there are no tensor-core instructions.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -204,6 +206,37 @@ k_merge(const float* __restrict__ tables, float* __restrict__ merged, int64_t rc
             for (int w = 0; w < W; ++w) acc = __fadd_rn(acc, tables[(int64_t)w * rc + t]);
             merged[t] = acc;
         }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// 16-bit sketches (Section 6): what a worker would send is its table rounded to binary16 or bfloat16
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint16_t quant16(float x, int fmt) {
+    if (fmt == 0) {
+        x = fminf(fmaxf(x, -65504.0f), 65504.0f);          // saturate instead of rounding to infinity
+        return __half_as_ushort(__float2half_rn(x));
+    }
+    return __bfloat16_as_ushort(__float2bfloat16_rn(x));
+}
+__device__ __forceinline__ float dequant16(uint16_t h, int fmt) {
+    return fmt == 0 ? __half2float(__ushort_as_half(h)) : __bfloat162float(__ushort_as_bfloat16(h));
+}
+
+__global__ void __launch_bounds__(256)
+k_quantize16(const float* __restrict__ x, uint16_t* __restrict__ q, int64_t n, int fmt) {
+    const int64_t stride = (int64_t)gridDim.x * 256;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < n; t += stride) q[t] = quant16(__ldcs(x + t), fmt);
+}
+
+// merged[t] = sum over w = 0..W-1 (that order, fp32) of the decoded q[w][t]
+__global__ void __launch_bounds__(256)
+k_merge16(const uint16_t* __restrict__ q, float* __restrict__ merged, int64_t n, int32_t W, int fmt) {
+    const int64_t stride = (int64_t)gridDim.x * 256;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < n; t += stride) {
+        float acc = 0.f;
+        for (int w = 0; w < W; ++w) acc = __fadd_rn(acc, dequant16(q[(int64_t)w * n + t], fmt));
+        merged[t] = acc;
     }
 }
 
@@ -952,6 +985,26 @@ int ssgd_sketch_merge(ssgd_ctx* x, const float* tables, float* merged, void* str
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     k_merge<<<grid_for((rc + 3) / 4, 256, (int64_t)x->sm_count * 16), 256, 0, st>>>(tables, merged, rc, x->W);
     LAUNCHED("k_merge");
+    return SSGD_OK;
+}
+
+int ssgd_sketch_quantize16(ssgd_ctx* x, const float* tables, int32_t fmt, uint16_t* q16, void* stream) {
+    if (!x || !tables || !q16 || (fmt != SSGD_FMT_F16 && fmt != SSGD_FMT_BF16)) return SSGD_EINVAL;
+    int e = ensure_device(x);
+    if (e) return e;
+    const int64_t n = (int64_t)x->W * x->r * x->c;
+    k_quantize16<<<grid_for(n, 256, (int64_t)x->sm_count * 16), 256, 0, static_cast<cudaStream_t>(stream)>>>(tables, q16, n, fmt);
+    LAUNCHED("k_quantize16");
+    return SSGD_OK;
+}
+
+int ssgd_sketch_merge16(ssgd_ctx* x, const uint16_t* q16, int32_t fmt, float* merged, void* stream) {
+    if (!x || !q16 || !merged || (fmt != SSGD_FMT_F16 && fmt != SSGD_FMT_BF16)) return SSGD_EINVAL;
+    int e = ensure_device(x);
+    if (e) return e;
+    const int64_t n = (int64_t)x->r * x->c;
+    k_merge16<<<grid_for(n, 256, (int64_t)x->sm_count * 16), 256, 0, static_cast<cudaStream_t>(stream)>>>(q16, merged, n, x->W, fmt);
+    LAUNCHED("k_merge16");
     return SSGD_OK;
 }
 

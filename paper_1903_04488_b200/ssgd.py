@@ -18,6 +18,7 @@ OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, 
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 PRUNE_AUTO, PRUNE_OFF, PRUNE_ON = 0, 1, 2
+FMT_F16, FMT_BF16 = 0, 1
 MAX_R = 15
 
 # name -> argument types, exactly the declarations of include/ssgd.h
@@ -35,6 +36,8 @@ SIGNATURES = {
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
     "ssgd_sketch_accumulate": [_vp, _vp, _i64, _f32, _vp, _vp],
     "ssgd_sketch_merge": [_vp, _vp, _vp, _vp],
+    "ssgd_sketch_quantize16": [_vp, _vp, _i32, _vp, _vp],
+    "ssgd_sketch_merge16": [_vp, _vp, _i32, _vp, _vp],
     "ssgd_unsketch_candidates": [_vp, _vp, _i64, _vp, _vp, _vp, _vp],
     "ssgd_exact_topk": [_vp, _vp, _i64, _vp, _vp, _vp],
     "ssgd_step": [_vp, _vp, _i64, _f32, _i64, _vp, _vp, _vp],
@@ -195,6 +198,15 @@ class Ssgd:
         self._chk(self._lib.ssgd_sketch_merge(self._h, _dev_ptr(tables, torch.float32, "tables"),
                                               _dev_ptr(merged, torch.float32, "merged"), _stream()),
                   "ssgd_sketch_merge")
+
+    def sketch_quantize16(self, tables: torch.Tensor, fmt: int, q16: torch.Tensor) -> None:
+        """tables [W][r][c] fp32 -> q16 [W][r][c] int16 (the 16-bit encodings), round to nearest even."""
+        self._chk(self._lib.ssgd_sketch_quantize16(self._h, _dev_ptr(tables, torch.float32, "tables"), fmt,
+                                                   _dev_ptr(q16, torch.int16, "q16"), _stream()), "ssgd_sketch_quantize16")
+
+    def sketch_merge16(self, q16: torch.Tensor, fmt: int, merged: torch.Tensor) -> None:
+        self._chk(self._lib.ssgd_sketch_merge16(self._h, _dev_ptr(q16, torch.int16, "q16"), fmt,
+                                                _dev_ptr(merged, torch.float32, "merged"), _stream()), "ssgd_sketch_merge16")
 
     def unsketch_candidates(self, merged, ncand, cand_idx, cand_est=None, est_all=None) -> None:
         self._chk(self._lib.ssgd_unsketch_candidates(
