@@ -64,6 +64,7 @@ extern "C" {
 #define SSGD_INSERT_GLOBAL 1  /* plain 128-bit loads; reductions straight into the L2-resident table    */
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
+#define SSGD_INSERT_WS     4  /* the same pipeline, warp-specialised: separate stream and sketch warps   */
 
 /* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  With pruning, coordinates that
  * provably cannot be among the ncand largest |estimate| stop reading sketch rows early (a median of r

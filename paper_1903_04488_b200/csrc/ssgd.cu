@@ -30,6 +30,7 @@
 #include "hash.cuh"
 #include "select.cuh"
 #include "accum_tma.cuh"
+#include "accum_ws.cuh"
 #include "estimate.cuh"
 #include "sparse_select.cuh"
 #include "heavymix.cuh"
@@ -50,7 +51,7 @@ namespace ssgd {
 // pipeline of accum_tma.cuh; this form serves the per-worker tables of ssgd_sketch_accumulate and the
 // shared-memory table variant.
 // ------------------------------------------------------------------------------------------------
-enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
+enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3, INS_MERGED_WS = 4 };
 
 #ifndef SSGD_K1_UNROLL
 #define SSGD_K1_UNROLL 16
@@ -429,6 +430,7 @@ struct ssgd_ctx {
     // device facts
     int device; int sm_count; int max_smem_optin;
     int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
+    int ws_blocks_per_sm;   // same for the warp-specialised kernel
     int64_t launches;
     // optional per-stage timing of ssgd_step (CUDA events on the caller's stream)
     bool timing;
@@ -657,6 +659,28 @@ int launch_accum_tma(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
 }
 
 template <int R, bool POW2>
+int launch_accum_ws_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
+    auto kern = k_accum_insert_ws<R, POW2>;
+    const size_t smem = sizeof(WsShared);
+    if (x->ws_blocks_per_sm == 0) {
+        CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "smem attribute");
+        int nb = 0;
+        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, WS_THREADS, smem), "occupancy query");
+        x->ws_blocks_per_sm = nb < 1 ? 1 : nb;
+    }
+    const int64_t ntiles = ((A.d & ~(int64_t)3) + WS_TC - 1) / WS_TC;
+    const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->ws_blocks_per_sm);
+    CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, kern, grid, WS_THREADS, smem, A,
+                    reinterpret_cast<int32_t*>(x->ws + x->off_err)), "launch k_accum_insert_ws");
+    LAUNCHED("k_accum_insert_ws");
+    return SSGD_OK;
+}
+
+int launch_accum_ws(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_accum_ws_t, x, A, st)
+}
+
+template <int R, bool POW2>
 int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     // a few blocks per SM: each block pays one histogram flush
@@ -822,6 +846,7 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
     if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
     if (x->insert_mode == SSGD_INSERT_TMA) return INS_MERGED_TMA;
+    if (x->insert_mode == SSGD_INSERT_WS) return INS_MERGED_WS;
     // measured on B200: the bulk-copy pipeline wins once a tile's walk over the workers is long
     // (W = 128: 5.73 vs 5.43 TB/s), plain loads win for short walks (W = 16: 4.93 vs 4.83 TB/s)
     return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
@@ -859,7 +884,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->pow2 = (c & (c - 1)) == 0;
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
-    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
+    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
     x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->persist_bytes = 0;
     *out = x;
     return SSGD_OK;
@@ -932,7 +957,7 @@ int ssgd_step_used_fallback(ssgd_ctx* x, void* stream, int32_t* out) {
 }
 
 int ssgd_set_insert_mode(ssgd_ctx* x, int32_t mode) {
-    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_TMA) return SSGD_EINVAL;
+    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_WS) return SSGD_EINVAL;
     x->insert_mode = mode;
     return SSGD_OK;
 }
@@ -1054,7 +1079,8 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
     if ((e = mark(x, 0, st))) return e;
-    if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st) : launch_accum(x, A, mode, st))) return e;
+    if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st)
+             : mode == INS_MERGED_WS ? launch_accum_ws(x, A, st) : launch_accum(x, A, mode, st))) return e;
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);

@@ -155,7 +155,7 @@ STEP_CASES = [
 
 
 @pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
-@pytest.mark.parametrize("mode", [S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
+@pytest.mark.parametrize("mode", [S.INSERT_WS, S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
 def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
     if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
