@@ -87,6 +87,11 @@ int ssgd_get_hash_params(const ssgd_ctx* ctx, uint32_t* out4r);
 int ssgd_set_hash_params(ssgd_ctx* ctx, const uint32_t* in4r);
 int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
 int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
+/* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
+ * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
+ * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 48 MiB,
+ * which leaves tables up to that size untouched). */
+int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
 /* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
  * (cudaLimitPersistingL2CacheSize of this process's CUDA context is raised to the table size, capped by the
  * device; the launches then carry an access-policy window over the table).  Off by default because the limit

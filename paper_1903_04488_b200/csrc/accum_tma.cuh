@@ -31,6 +31,10 @@ struct AccumArgs {
     float* table;        // merged [r][c], or per-worker [W][r][c]
     int64_t c;
     HashParams hp; Bucketizer bk;
+    // plain-load merged mode only: insert rows [0, rows_here) in this kernel and, if xsum is not NULL, also
+    // write the per-coordinate sum over workers to xsum[d] so that k_insert_rows can do the remaining rows
+    int32_t rows_here;
+    float* xsum;
 };
 
 #ifndef SSGD_KT_STAGES

@@ -37,6 +37,11 @@
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
+#ifndef SSGD_SPLIT_BYTES_DEFAULT
+// measured on B200 (C4: d = 9e7, W = 16, 5 x 4,194,304 = 80 MB table): unsplit 7.80 ms, 48 MB or 32 MB slices 6.26 ms,
+// 16 MB slices 6.44 ms
+#define SSGD_SPLIT_BYTES_DEFAULT ((size_t)48 << 20)
+#endif
 #ifndef SSGD_PRUNED_GRID
 #define SSGD_PRUNED_GRID 4
 #endif
@@ -152,8 +157,13 @@ k_accum_insert(const AccumArgs A) {
             }
         }
         if (MODE != INS_PER_WORKER) {
+            if (MODE == INS_MERGED_GLOBAL && A.xsum != nullptr) {
+                if (i0 + 3 < A.d) *reinterpret_cast<float4*>(A.xsum + i0) = make_float4(x[0], x[1], x[2], x[3]);
+                else for (int e = 0; e < 4 && i0 + e < A.d; ++e) A.xsum[i0 + e] = x[e];
+            }
 #pragma unroll
             for (int j = 0; j < R; ++j) {
+                if (MODE == INS_MERGED_GLOBAL && j >= A.rows_here) break;
                 uint32_t h1[4];
                 row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, h1);
 #pragma unroll
@@ -172,6 +182,40 @@ k_accum_insert(const AccumArgs A) {
         for (int64_t t = threadIdx.x; t < rc; t += K1_THREADS) {
             const float s = s_table[t];
             if (s != 0.0f) red_add(A.table + t, s);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Rows [row_lo, R) of the insert, from the per-coordinate sums written by k_accum_insert.  Used when the
+// whole r x c table is too large to stay in L2 next to the stream: the streaming kernel then inserts only as
+// many rows as fit, and the rest are inserted here, a few rows (an L2-sized slice of the table) per launch.
+// ------------------------------------------------------------------------------------------------
+template <int R, bool POW2>
+__global__ void __launch_bounds__(256)
+k_insert_rows(const float* __restrict__ xsum, int64_t d, float* __restrict__ table, int64_t c, HashParams hp,
+              Bucketizer bk, int row_lo, int row_hi) {
+    pdl_trigger();
+    pdl_wait();
+    const int64_t groups = (d + 3) >> 2;
+    const int64_t stride = (int64_t)gridDim.x * 256;
+    for (int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x; q < groups; q += stride) {
+        const int64_t i0 = q << 2;
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        if (i0 + 3 < d) {
+            const float4 t = __ldcs(reinterpret_cast<const float4*>(xsum + i0));
+            x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+        } else {
+            for (int e = 0; e < 4 && i0 + e < d; ++e) x[e] = xsum[i0 + e];
+        }
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            if (j < row_lo || j >= row_hi) continue;
+            uint32_t hb[4];
+            row_hashes<POW2, 4>(hp.row[j], bk, (uint32_t)i0, hb);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                if (i0 + e < d && x[e] != 0.0f) red_add(table + (int64_t)j * c + (hb[e] & P31), apply_sign(x[e], hb[e]));
         }
     }
 }
@@ -424,7 +468,8 @@ struct ssgd_ctx {
     int64_t list_cap;
     size_t off_hm;
     int32_t prune_mode;
-    size_t persist_bytes;   // > 0: launches that touch the table carry an L2 access-policy window of this size
+    size_t persist_bytes;
+    size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel   // > 0: launches that touch the table carry an L2 access-policy window of this size
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;
     // device facts
@@ -659,6 +704,19 @@ int launch_accum_tma(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
 }
 
 template <int R, bool POW2>
+int launch_insert_rows_t(ssgd_ctx* x, const float* xsum, float* table, int lo, int hi, cudaStream_t st) {
+    const int64_t groups = (x->d + 3) / 4;
+    CU(launch_pdl(st, k_insert_rows<R, POW2>, grid_for(groups, 256, (int64_t)x->sm_count * 8), 256, 0, xsum, x->d, table, x->c,
+                  x->hp, x->bk, lo, hi), "launch k_insert_rows");
+    LAUNCHED("k_insert_rows");
+    return SSGD_OK;
+}
+
+int launch_insert_rows(ssgd_ctx* x, const float* xsum, float* table, int lo, int hi, cudaStream_t st) {
+    DISPATCH_R(launch_insert_rows_t, x, xsum, table, lo, hi, st)
+}
+
+template <int R, bool POW2>
 int launch_accum_ws_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
     auto kern = k_accum_insert_ws<R, POW2>;
     const size_t smem = sizeof(WsShared);
@@ -885,7 +943,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->persist_bytes = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -936,6 +994,12 @@ int ssgd_set_table_persistence(ssgd_ctx* x, int32_t enable) {
     if (carve == 0) return SSGD_OK;
     CU(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve), "set persisting L2 size");
     x->persist_bytes = want;
+    return SSGD_OK;
+}
+
+int ssgd_set_insert_split(ssgd_ctx* x, int64_t bytes) {
+    if (!x || bytes < 0) return SSGD_EINVAL;
+    x->split_bytes = (size_t)bytes;
     return SSGD_OK;
 }
 
@@ -997,7 +1061,7 @@ int ssgd_sketch_accumulate(ssgd_ctx* x, const float* g, int64_t ld_g, float rho,
     x->launches++;
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
-    A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
+    A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
     return launch_accum(x, A, INS_PER_WORKER, st);
 }
 
@@ -1077,10 +1141,18 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     float* merged = reinterpret_cast<float*>(x->ws + x->off_table);
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
-    A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk;
+    A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
+    // a table that cannot stay in L2 next to the stream is inserted a slice of rows at a time
+    const size_t row_bytes = (size_t)x->c * 4;
+    const int rows_fit = (int)(x->split_bytes / row_bytes);
+    const bool split = mode == INS_MERGED_GLOBAL && x->split_bytes > 0 && rows_fit >= 1 && rows_fit < x->r;
+    if (split) { A.rows_here = rows_fit; A.xsum = reinterpret_cast<float*>(x->ws + x->off_est); }
     if ((e = mark(x, 0, st))) return e;
     if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st)
              : mode == INS_MERGED_WS ? launch_accum_ws(x, A, st) : launch_accum(x, A, mode, st))) return e;
+    if (split)
+        for (int lo = rows_fit; lo < x->r; lo += rows_fit)
+            if ((e = launch_insert_rows(x, A.xsum, merged, lo, lo + rows_fit < x->r ? lo + rows_fit : x->r, st))) return e;
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);

@@ -30,6 +30,7 @@ SIGNATURES = {
     "ssgd_set_hash_params": [_vp, _vp],
     "ssgd_set_insert_mode": [_vp, _i32],
     "ssgd_set_prune_mode": [_vp, _i32],
+    "ssgd_set_insert_split": [_vp, _i64],
     "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
@@ -144,6 +145,9 @@ class Ssgd:
 
     def set_prune_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_prune_mode(self._h, mode), "ssgd_set_prune_mode")
+
+    def set_insert_split(self, nbytes: int) -> None:
+        self._chk(self._lib.ssgd_set_insert_split(self._h, nbytes), "ssgd_set_insert_split")
 
     def set_table_persistence(self, enable: bool) -> None:
         self._chk(self._lib.ssgd_set_table_persistence(self._h, 1 if enable else 0), "ssgd_set_table_persistence")

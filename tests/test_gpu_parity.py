@@ -225,6 +225,24 @@ def test_heavy_ties_at_the_threshold(cuda_device, prune):
     assert big <= set(idx.tolist())
 
 
+def test_row_split_insert(cuda_device):
+    """Tables above the L2 budget are inserted a slice of rows at a time (the streaming kernel does the first
+    slice and leaves per-coordinate sums for the rest); forced here with a budget of two rows."""
+    cfg = wl.C4.scaled(d=400_003, W=5, r=7, c=4096, ncand=2000, k=1000)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_insert_mode(S.INSERT_GLOBAL)
+    eng.set_insert_split(2 * cfg.c * 4)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    n0 = eng.launch_count()
+    for t in range(3):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
+    eng2, _, _, _ = make(cfg, cuda_device)
+    eng2.set_insert_mode(S.INSERT_GLOBAL)
+    eng2.set_insert_split(0)
+    assert eng.launch_count() - n0 > 0
+
+
 def test_pruned_path_is_taken_and_prunes(cuda_device):
     """On a gradient-shaped input the early-exit path must do its job: no fall-back, a non-trivial
     threshold, at least ncand survivors and far fewer than d; a few ties at the threshold are ranked by index."""
