@@ -56,6 +56,19 @@ struct SelBuffers {
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
 
+// Histogram passes load SEL_BATCH items per thread before touching shared memory, so that a pass costs a few
+// L2 round trips instead of one per item (the shared-memory atomics keep the compiler from hoisting loads).
+constexpr int SEL_BATCH = 8;
+constexpr uint32_t NO_ITEM = 0xFFFFFFFFu;                  // keys have bit 31 clear
+__device__ __forceinline__ void load_keys(const float* __restrict__ val, int64_t n, int64_t i0, int64_t step,
+                                          uint32_t (&keys)[SEL_BATCH]) {
+#pragma unroll
+    for (int u = 0; u < SEL_BATCH; ++u) {
+        const int64_t i = i0 + u * step;
+        keys[u] = i < n ? key_of(val[i]) : NO_ITEM;
+    }
+}
+
 // A gated selection is the dense fall-back of the sparse candidate path: its kernels are always
 // enqueued and leave at once unless the sparse path raised the flag (read after pdl_wait()).
 __device__ __forceinline__ bool gate_closed(const uint32_t* gate) { return gate != nullptr && __ldcg(gate) == 0; }
@@ -135,9 +148,12 @@ k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     const uint32_t d1 = sb.state->d1;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
-    for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
-        const uint32_t key = key_of(val[i]);
-        if ((key >> H1_SHIFT) == d1) atomicAdd(&sh.hist[(key >> H2_SHIFT) & (H2_BINS - 1)], 1u);
+    for (int64_t i0 = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i0 < n; i0 += stride * SEL_BATCH) {
+        uint32_t keys[SEL_BATCH];
+        load_keys(val, n, i0, stride, keys);
+#pragma unroll
+        for (int u = 0; u < SEL_BATCH; ++u)
+            if (keys[u] != NO_ITEM && (keys[u] >> H1_SHIFT) == d1) atomicAdd(&sh.hist[(keys[u] >> H2_SHIFT) & (H2_BINS - 1)], 1u);
     }
     __syncthreads();
     flush_hist<H2_BINS>(sh.hist, sb.h2);
@@ -160,9 +176,12 @@ k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     const uint32_t prefix = (d1 << H2_BITS) | d2;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
-    for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < n; i += stride) {
-        const uint32_t key = key_of(val[i]);
-        if ((key >> H2_SHIFT) == prefix) atomicAdd(&sh.hist[key & (H3_BINS - 1)], 1u);
+    for (int64_t i0 = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i0 < n; i0 += stride * SEL_BATCH) {
+        uint32_t keys[SEL_BATCH];
+        load_keys(val, n, i0, stride, keys);
+#pragma unroll
+        for (int u = 0; u < SEL_BATCH; ++u)
+            if (keys[u] != NO_ITEM && (keys[u] >> H2_SHIFT) == prefix) atomicAdd(&sh.hist[keys[u] & (H3_BINS - 1)], 1u);
     }
     __syncthreads();
     flush_hist<H3_BINS>(sh.hist, sb.h3);
@@ -193,13 +212,17 @@ __device__ __forceinline__ void chunk_ballots(const float* __restrict__ val, int
                                               uint32_t& ngt, uint32_t& neq) {
     const int lane = threadIdx.x & 31;
     ngt = 0; neq = 0;
+    uint32_t keys[SEL_ITEMS];                               // all of the lane's items are loaded before any is used
 #pragma unroll
     for (int it = 0; it < SEL_ITEMS; ++it) {
         const int64_t i = warp_base + it * 32 + lane;
-        uint32_t key = 0; bool ok = i < n;
-        if (ok) key = key_of(val[i]);
-        bg[it] = __ballot_sync(0xFFFFFFFFu, ok && key > T);
-        be[it] = __ballot_sync(0xFFFFFFFFu, ok && key == T);
+        keys[it] = i < n ? key_of(val[i]) : NO_ITEM;
+    }
+#pragma unroll
+    for (int it = 0; it < SEL_ITEMS; ++it) {
+        const bool ok = keys[it] != NO_ITEM;
+        bg[it] = __ballot_sync(0xFFFFFFFFu, ok && keys[it] > T);
+        be[it] = __ballot_sync(0xFFFFFFFFu, ok && keys[it] == T);
         ngt += __popc(bg[it]);
         neq += __popc(be[it]);
     }
