@@ -359,6 +359,11 @@ k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32
 // ------------------------------------------------------------------------------------------------
 // K5: second round -- xs[m] = sum_w v_w[cand[m]] (fp64, w = 0..W-1), rounded once to fp32
 // ------------------------------------------------------------------------------------------------
+#ifndef SSGD_GATHER_UNROLL
+#define SSGD_GATHER_UNROLL 8
+#endif
+constexpr int GATHER_UNROLL = SSGD_GATHER_UNROLL;   // scattered loads in flight per thread
+
 __global__ void __launch_bounds__(256)
 k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ v, int64_t ld, int32_t W,
          int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag) {
@@ -378,12 +383,12 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
             double acc = 0.0;
             const float* p = v + i;
             int w = 0;
-            for (; w + 8 <= W; w += 8) {
-                float t[8];
+            for (; w + GATHER_UNROLL <= W; w += GATHER_UNROLL) {
+                float t[GATHER_UNROLL];
 #pragma unroll
-                for (int s = 0; s < 8; ++s) t[s] = __ldg(p + (int64_t)(w + s) * ld);
+                for (int s = 0; s < GATHER_UNROLL; ++s) t[s] = __ldg(p + (int64_t)(w + s) * ld);
 #pragma unroll
-                for (int s = 0; s < 8; ++s) acc = __dadd_rn(acc, (double)t[s]);
+                for (int s = 0; s < GATHER_UNROLL; ++s) acc = __dadd_rn(acc, (double)t[s]);
             }
             for (; w < W; ++w) acc = __dadd_rn(acc, (double)__ldg(p + (int64_t)w * ld));
             out = (float)acc;

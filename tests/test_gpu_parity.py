@@ -367,6 +367,40 @@ def test_full_size_C5_worker_sweep(cuda_device, W):
     run_full(cfg, cuda_device, 1, True)
 
 
+def test_step_can_be_captured_in_a_cuda_graph(cuda_device):
+    """ssgd_step only enqueues work (no host synchronisation, no allocation), so once the context is warm a
+    step can be captured and replayed; a replay from zero state selects what an eager step selects (up to
+    near-ties: the order of the reductions into the table differs from run to run)."""
+    dev = cuda_device
+    cfg = wl.C2.scaled(d=5_000_002, W=4, c=65_536, ncand=20_000, k=10_000)     # early-exit path included
+    g = wl.gradients(wl.Structure(cfg, dev), 0)
+    eng, _, u, v = make(cfg, dev)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    ov = torch.empty(cfg.k, device=dev)
+    eng.step(g, cfg.rho, cfg.ncand, oi, ov)                # warm-up: device queries, function attributes
+    assert eng.status() == S.OK
+    eager_idx, eager_val = oi.clone(), ov.clone()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    u.zero_(); v.zero_()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            eng.step(g, cfg.rho, cfg.ncand, oi, ov)
+    for _ in range(2):
+        u.zero_(); v.zero_(); oi.zero_(); ov.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert eng.status() == S.OK
+        a, b = eager_idx.cpu().numpy(), oi.cpu().numpy()
+        assert (np.diff(b) > 0).all()
+        common, ia, ib = np.intersect1d(a, b, return_indices=True)
+        assert common.size >= 0.995 * cfg.k
+        assert (eager_val.cpu().numpy()[ia] == ov.cpu().numpy()[ib]).all()
+        assert int((v[0, :cfg.d] == 0).sum().item()) >= cfg.k
+
+
 # ------------------------------------------------------------------------------------------------
 # argument checking (host side; nothing is launched)
 # ------------------------------------------------------------------------------------------------
