@@ -367,6 +367,45 @@ def test_full_size_C5_worker_sweep(cuda_device, W):
     run_full(cfg, cuda_device, 1, True)
 
 
+def test_stored_small_case_is_reproduced_exactly(cuda_device):
+    """Integer gradients and rho = 1/2 make every operation exact, reductions included, so the library must
+    reproduce the stored case (written by the oracle alone) bit for bit: table, candidates, k-set, values."""
+    import hashlib
+    import importlib.util
+    import json
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    spec = importlib.util.spec_from_file_location("make_golden", os.path.join(here, "golden", "make_golden.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    want = json.load(open(os.path.join(here, "golden", "oracle_small_case.json")))
+    sh = want["shape"]
+    dev = cuda_device
+    for mode in (S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_SMEM):
+        eng = S.Ssgd(sh["d"], sh["r"], sh["c"], sh["k"], sh["W"], sh["seed"])
+        assert eng.get_hash_params().tolist() == want["hash_params"]
+        ld = (sh["d"] + 3) // 4 * 4
+        u = torch.zeros((sh["W"], ld), device=dev)
+        v = torch.zeros_like(u)
+        eng.bind(u, v, want["ncand"])
+        eng.set_insert_mode(mode)
+        oi = torch.empty(sh["k"], dtype=torch.int32, device=dev)
+        ov = torch.empty(sh["k"], device=dev)
+        for t, step in enumerate(want["steps"]):
+            g = torch.zeros((sh["W"], ld), device=dev)
+            g[:, :sh["d"]] = torch.tensor(mod.gradients(t), device=dev)
+            eng.step(g, want["rho"], want["ncand"], oi, ov)
+            assert eng.status() == S.OK
+            merged, _, cand, _ = eng.step_buffers(want["ncand"])
+            table64 = merged.cpu().numpy().astype(np.float64)
+            assert hashlib.sha256(np.ascontiguousarray(table64).tobytes()).hexdigest() == step["table_sha256"]
+            assert cand.cpu().tolist() == step["cand"]
+            assert oi.cpu().tolist() == step["out_idx"]
+            assert ov.cpu().tolist() == step["out_val"]
+        state = u.cpu().numpy()[:, :sh["d"]].tobytes() + v.cpu().numpy()[:, :sh["d"]].tobytes()
+        assert hashlib.sha256(state).hexdigest() == want["state_sha256"]
+
+
 def test_step_can_be_captured_in_a_cuda_graph(cuda_device):
     """ssgd_step only enqueues work (no host synchronisation, no allocation), so once the context is warm a
     step can be captured and replayed; a replay from zero state selects what an eager step selects (up to
