@@ -97,10 +97,14 @@ int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
  * device; the launches then carry an access-policy window over the table).  Off by default because the limit
  * is shared with everything else the process runs on that device.  enable = 0 stops attaching the window. */
 int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
-/* Diagnostics of the last ssgd_step's pruned path (waits for the stream): out[0] = 1 if the dense path had
- * to take over (too few survivors, list overflow, too many ties), out[1] = number of coordinates that
- * survived the early exit, out[2] = the prune threshold as a histogram-bin index (0: nothing pruned). */
+/* Diagnostics of the last ssgd_step's pruned path (waits for the stream): out[0] != 0 if the sampled
+ * threshold kept fewer than ncand coordinates and the pass was redone without pruning, out[1] = number of
+ * coordinates on the survivor list, out[2] = the prune threshold as a histogram-bin index (0: nothing pruned). */
 int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out3);
+/* For tests and diagnostics: the rank (from the top) in the sample's histogram that sets the prune threshold;
+ * 0 = derive it from ncand (mean + 6 sigma + 16).  A rank of 1 puts the threshold at the largest sampled
+ * estimate, which forces the unpruned rerun. */
+int ssgd_set_prune_sample_rank(ssgd_ctx* ctx, int64_t rank);
 
 /* Bytes of device scratch needed to run steps with up to ncand_max candidates (host only). */
 int ssgd_workspace_bytes(const ssgd_ctx* ctx, int64_t ncand_max, size_t* out_bytes);

@@ -49,7 +49,6 @@ struct SelBuffers {
     SelState* state;
     uint32_t* chunk_gt;  // [nchunks] counts, then exclusive offsets
     uint32_t* chunk_eq;  // [nchunks]
-    const uint32_t* gate;  // if not NULL: the kernels of this selection run only when *gate != 0
 };
 
 #ifdef __CUDACC__
@@ -69,9 +68,6 @@ __device__ __forceinline__ void load_keys(const float* __restrict__ val, int64_t
     }
 }
 
-// A gated selection is the dense fall-back of the sparse candidate path: its kernels are always
-// enqueued and leave at once unless the sparse path raised the flag (read after pdl_wait()).
-__device__ __forceinline__ bool gate_closed(const uint32_t* gate) { return gate != nullptr && __ldcg(gate) == 0; }
 
 struct SelShared {
     uint32_t hist[H1_BINS];
@@ -144,7 +140,6 @@ k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
-    if (gate_closed(sb.gate)) return;
     const uint32_t d1 = sb.state->d1;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
@@ -171,7 +166,6 @@ k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H3_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
-    if (gate_closed(sb.gate)) return;
     const uint32_t d1 = sb.state->d1, d2 = sb.state->d2;
     const uint32_t prefix = (d1 << H2_BITS) | d2;
     __syncthreads();
@@ -273,7 +267,6 @@ k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nch
     __shared__ SelShared sh;
     pdl_trigger();
     pdl_wait();
-    if (gate_closed(sb.gate)) return;
     const uint32_t T = sb.state->thr_key;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
@@ -300,7 +293,6 @@ __device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, i
     __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
     pdl_trigger();
     pdl_wait();
-    if (gate_closed(sb.gate)) return;
     const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {

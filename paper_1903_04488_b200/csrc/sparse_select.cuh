@@ -14,15 +14,13 @@
 //   * k_unsketch_pruned evaluates every coordinate with that early exit and appends the survivors
 //     (exact estimate in a bin >= bin_lo) to a compact list.  The survivor set does not depend on how the
 //     pruning went: it is exactly { i : bin(|est_i|) >= bin_lo }.
-//   * If the list holds at least ncand entries (and fits), the top-ncand of all d coordinates is the
-//     top-ncand of the list: k_select_sparse, one 8-CTA cluster, runs the radix select on the list
-//     (histograms reduced through distributed shared memory), breaks ties at the threshold by coordinate
-//     index, marks the selected coordinates in a d-bit map and compacts the map in order, so cand_idx
-//     comes out ascending exactly as the dense path produces it.
-//   * Otherwise a flag opens the gate of the dense path (k_unsketch + select.cuh), whose kernels are
-//     always enqueued behind and return at once when the gate is closed.
+//   * If the list holds at least ncand entries, the top-ncand of all d coordinates is the top-ncand of the
+//     list, which the kernels of list_select.cuh extract (cand_idx comes out ascending, exactly as the dense
+//     path produces it).
+//   * Otherwise (the sample misjudged the threshold) the last block of k_unsketch_pruned resets the list
+//     and raises a flag; a second launch of the same kernel, always enqueued behind and returning at once
+//     unless the flag is up, redoes the pass without pruning.  The list has room for all d coordinates.
 #pragma once
-#include <cooperative_groups.h>
 #include <stdint.h>
 
 #include "estimate.cuh"
@@ -36,27 +34,31 @@ namespace ssgd {
 #define SSGD_SAMPLE_SHIFT 6
 #endif
 constexpr int SPARSE_SAMPLE_SHIFT = SSGD_SAMPLE_SHIFT;   // one float4 group in 2^shift is sampled
-constexpr int SPARSE_CLUSTER = 8;                 // CTAs in the selection cluster (portable maximum)
-constexpr int SPARSE_THREADS = 1024;
-constexpr int SPARSE_MAX_TIES = 2048;             // ties at the threshold handled in shared memory
 
 struct SparseState {                              // zeroed before the step
     uint32_t bin_lo;       // prune threshold: H1 bin index; 0 = nothing can be pruned
-    uint32_t n_surv;       // survivors appended (may exceed the capacity; entries beyond it are dropped)
-    uint32_t fallback;     // != 0: the dense path must run (this word is the dense kernels' gate)
-    uint32_t d1, rem1;     // first threshold digit of the survivors' histogram
-    uint32_t ticket[2];
-    uint32_t pad[9];
+    uint32_t n_surv;       // survivors appended to the list
+    uint32_t fallback;     // 1: too few survivors, the unpruned pass must run; 2: it has run
+    uint32_t d1, rem1;     // first threshold digit of the survivors' histogram H1 and the count wanted inside it
+    uint32_t thr_key;      // T: the exact 31-bit threshold key
+    uint32_t quota_eq;     // Q: how many items with key == T are selected (smallest coordinates first)
+    uint32_t ticket[6];    // finished-block counters: sample, pruned, unpruned rerun, list histogram, map count
+    uint32_t pad[3];
 };
 
 struct SparseBuffers {
     uint32_t* h1_sample;   // [H1_BINS] zeroed
     uint32_t* h1;          // [H1_BINS] zeroed: histogram of the survivors' estimates
     SparseState* state;
-    int32_t* list_idx;     // [cap]
+    uint32_t* h2;          // [H2_BINS] zeroed: next 11 key bits of the list items inside the first digit
+    uint32_t* h19;         // [2^19] zeroed: the low 19 key bits of the same items
+    int32_t* list_idx;     // [cap], cap >= d
     float* list_est;       // [cap]
     uint32_t cap;
-    uint32_t* bitmap;      // [ceil(d/32)] zeroed
+    uint32_t* map_a;       // [ceil(d/32)] zeroed: coordinates above the threshold
+    uint32_t* map_b;       // [ceil(d/32)] zeroed: coordinates at the threshold (ties)
+    uint32_t* chunk_a;     // [map chunks] marks per chunk of map words, then exclusive offsets
+    uint32_t* chunk_b;
 };
 
 struct SparseArgs {
@@ -65,11 +67,10 @@ struct SparseArgs {
     SparseBuffers sp;
     uint32_t ncand;
     uint32_t want_sample;  // rank (from the top) in the sample's histogram that defines bin_lo
+    int32_t rerun;         // 0: the pruned pass; 1: the unpruned pass behind it (runs only if fallback == 1)
 };
 
 #ifdef __CUDACC__
-namespace cg = cooperative_groups;
-
 __device__ __forceinline__ uint32_t mix32(uint32_t x) {
     x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
     return x;
@@ -138,7 +139,8 @@ k_unsketch_pruned(const SparseArgs A) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
-    const uint32_t bin_lo = A.sp.state->bin_lo;
+    if (A.rerun && __ldcg(&A.sp.state->fallback) != 1u) return;
+    const uint32_t bin_lo = A.rerun ? 0u : A.sp.state->bin_lo;
     __syncthreads();
     const int lane = threadIdx.x & 31;
     constexpr int NC = SSGD_PRUNED_NC;                     // consecutive coordinates per thread
@@ -223,246 +225,21 @@ k_unsketch_pruned(const SparseArgs A) {
     }
     __syncthreads();
     flush_hist<H1_BINS>(sh.hist, A.sp.h1);
-    if (block_is_last(&A.sp.state->ticket[1], sh)) {
+    if (block_is_last(&A.sp.state->ticket[A.rerun ? 2 : 1], sh)) {
         const uint32_t n = __ldcg(&A.sp.state->n_surv);
-        const bool fb = n < A.ncand || n > A.sp.cap;
-        uint32_t d1 = 0, rem1 = 1;
-        if (!fb) block_find_from_top<H1_BINS>(A.sp.h1, A.ncand, sh, d1, rem1);
-        if (threadIdx.x == 0) { A.sp.state->fallback = fb ? 1u : 0u; A.sp.state->d1 = d1; A.sp.state->rem1 = rem1; }
-    }
-}
-
-// ---- one cluster: radix select on the survivor list, ties by index, bitmap, ordered emit -----------
-struct SparseShared {
-    uint32_t hist[H2_BINS];              // H2, then H3 (in CTA 0: the cluster-wide sums)
-    uint32_t wsum[32];
-    uint32_t found[2];
-    uint32_t thr[2][2];                  // per pass: prefix/threshold and remaining count (valid in CTA 0)
-    uint32_t n_ties;                     // CTA 0
-    int32_t ties[SPARSE_MAX_TIES];       // CTA 0: coordinates with key == T
-    uint32_t cta_total[SPARSE_CLUSTER];  // CTA 0: selected bits per CTA range
-    uint32_t bail;                       // CTA 0
-};
-
-// Largest digit D with count(bins > D) < want <= count(bins >= D) over a shared-memory histogram;
-// all SPARSE_THREADS threads call.  nbins is a multiple of 32 and at most H2_BINS.
-__device__ __forceinline__ void cta_find_from_top(SparseShared& sh, int nbins, uint32_t want, uint32_t& digit, uint32_t& rem) {
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const int per_warp = nbins / 32;                   // 64 or 8 bins per warp
-    uint32_t part = 0;
-    for (int b = lane; b < per_warp; b += 32) part += sh.hist[warp * per_warp + b];
-    for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, off);
-    if (lane == 0) sh.wsum[warp] = part;
-    if (t == 0) { sh.found[0] = 0; sh.found[1] = 1; }
-    __syncthreads();
-    if (warp == 0) {
-        // lane = index of a warp-sized chunk; suffix sums over chunks above this one
-        const uint32_t mine = sh.wsum[lane];
-        uint32_t incl = mine;
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, incl, off);
-            if (lane + off < 32) incl += o;
-        }
-        const uint32_t above = incl - mine;
-        if (above < want && want <= above + mine) {
-            uint32_t acc = above;
-            for (int b = lane * per_warp + per_warp - 1; b >= lane * per_warp; --b) {
-                const uint32_t h = sh.hist[b];
-                if (acc + h >= want) { sh.found[0] = (uint32_t)b; sh.found[1] = want - acc; break; }
-                acc += h;
+        if (!A.rerun && n < A.ncand) {
+            // the sampled threshold was too high: empty the list and its histogram for the unpruned pass
+            for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) A.sp.h1[b] = 0;
+            if (threadIdx.x == 0) { A.sp.state->n_surv = 0; A.sp.state->fallback = 1u; }
+        } else {
+            uint32_t d1 = 0, rem1 = 1;
+            block_find_from_top<H1_BINS>(A.sp.h1, A.ncand, sh, d1, rem1);
+            if (threadIdx.x == 0) {
+                A.sp.state->d1 = d1; A.sp.state->rem1 = rem1;
+                if (A.rerun) A.sp.state->fallback = 2u;
             }
         }
     }
-    __syncthreads();
-    digit = sh.found[0];
-    rem = sh.found[1];
-    __syncthreads();
-}
-
-// LB list entries per thread are loaded together (independent loads in flight), then processed.
-constexpr int LB = 8;
-constexpr uint32_t NO_KEY = 0xFFFFFFFFu;                    // marks "past the end of the list"
-__device__ __forceinline__ void list_keys(const float* __restrict__ est, uint32_t n, uint32_t i0, uint32_t step,
-                                          uint32_t (&keys)[LB]) {
-#pragma unroll
-    for (int u = 0; u < LB; ++u) {
-        const uint32_t i = i0 + (uint32_t)u * step;
-        keys[u] = i < n ? key_of(__ldcg(est + i)) : NO_KEY;
-    }
-}
-
-__global__ void __launch_bounds__(SPARSE_THREADS)
-k_select_sparse(SparseBuffers sp, int64_t d, uint32_t ncand, int32_t* __restrict__ cand_idx) {
-    __shared__ SparseShared sh;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const unsigned rank = cluster.block_rank();
-    const int gthreads = SPARSE_CLUSTER * SPARSE_THREADS;
-    const int gt = rank * SPARSE_THREADS + t;
-    SparseShared* sh0 = cluster.map_shared_rank(&sh, 0);
-    pdl_trigger();
-    pdl_wait();
-    if (__ldcg(&sp.state->fallback) != 0) return;          // uniform over the cluster: the dense path runs instead
-    const uint32_t n = __ldcg(&sp.state->n_surv);
-    const uint32_t d1 = sp.state->d1, rem1 = sp.state->rem1;
-
-    // ---- H2 and H3 over the list: per-CTA histogram, summed into CTA 0 through distributed shared memory
-    uint32_t prefix = d1, want = rem1;
-    uint32_t T = 0, Q = 0;
-    for (int pass = 0; pass < 2; ++pass) {
-        const int nbins = pass == 0 ? H2_BINS : H3_BINS;
-        for (int b = t; b < H2_BINS; b += SPARSE_THREADS) sh.hist[b] = 0;
-        if (pass == 0 && rank == 0 && t == 0) { sh.n_ties = 0; sh.bail = 0; }
-        __syncthreads();
-        for (uint32_t i0 = gt; i0 < n; i0 += gthreads * LB) {
-            uint32_t keys[LB];
-            list_keys(sp.list_est, n, i0, gthreads, keys);
-#pragma unroll
-            for (int u = 0; u < LB; ++u) {
-                const uint32_t key = keys[u];
-                if (key == NO_KEY) continue;
-                if (pass == 0) { if ((key >> H1_SHIFT) == prefix) atomicAdd(&sh.hist[(key >> H2_SHIFT) & (H2_BINS - 1)], 1u); }
-                else           { if ((key >> H2_SHIFT) == prefix) atomicAdd(&sh.hist[key & (H3_BINS - 1)], 1u); }
-            }
-        }
-        cluster.sync();                                     // every CTA's private histogram is complete
-        if (rank == 0) {
-            // CTA 0 sums the eight histograms through distributed shared memory, then finds the digit
-            uint32_t acc[H2_BINS / SPARSE_THREADS];
-#pragma unroll
-            for (int q = 0; q < H2_BINS / SPARSE_THREADS; ++q) {
-                const int b = t + q * SPARSE_THREADS;
-                acc[q] = 0;
-                if (b < nbins)
-                    for (unsigned r2 = 0; r2 < SPARSE_CLUSTER; ++r2) acc[q] += cluster.map_shared_rank(&sh, r2)->hist[b];
-            }
-            __syncthreads();
-#pragma unroll
-            for (int q = 0; q < H2_BINS / SPARSE_THREADS; ++q) {
-                const int b = t + q * SPARSE_THREADS;
-                if (b < nbins) sh.hist[b] = acc[q];
-            }
-            __syncthreads();
-            uint32_t digit, rem;
-            cta_find_from_top(sh, nbins, want, digit, rem);
-            if (t == 0) {
-                sh.thr[pass][0] = (prefix << (pass == 0 ? H2_BITS : H3_BITS)) | digit;
-                sh.thr[pass][1] = rem;
-            }
-        }
-        cluster.sync();                                     // thr[pass] is published; the histograms may be reused
-        prefix = sh0->thr[pass][0];
-        want = sh0->thr[pass][1];
-    }
-    T = prefix;
-    Q = want;
-
-    // ---- ties at the threshold: the Q smallest coordinates win ---------------------------------------
-    for (uint32_t i0 = gt; i0 < n; i0 += gthreads * LB) {
-        uint32_t keys[LB];
-        list_keys(sp.list_est, n, i0, gthreads, keys);
-#pragma unroll
-        for (int u = 0; u < LB; ++u) {
-            if (keys[u] == T) {                                 // NO_KEY is never a threshold (bit 31 set)
-                const uint32_t slot = atomicAdd(&sh0->n_ties, 1u);
-                if (slot < SPARSE_MAX_TIES) sh0->ties[slot] = sp.list_idx[i0 + (uint32_t)u * gthreads];
-            }
-        }
-    }
-    cluster.sync();
-    const uint32_t n_ties = sh0->n_ties;
-    if (n_ties > SPARSE_MAX_TIES) {
-        // too many equal magnitudes to rank here: hand over to the dense path (nothing written yet)
-        if (rank == 0 && t == 0) sp.state->fallback = 1u;
-        cluster.sync();
-        return;
-    }
-    // every CTA takes its own copy of the tied coordinates (remote shared memory is slow to scan)
-    if (rank != 0)
-        for (uint32_t s = t; s < n_ties; s += SPARSE_THREADS) sh.ties[s] = sh0->ties[s];
-    __syncthreads();
-    // selected: key > T, or key == T and fewer than Q tied coordinates are smaller
-    for (uint32_t i0 = gt; i0 < n; i0 += gthreads * LB) {
-        uint32_t keys[LB];
-        int32_t idxs[LB];
-        list_keys(sp.list_est, n, i0, gthreads, keys);
-#pragma unroll
-        for (int u = 0; u < LB; ++u) {
-            const uint32_t i = i0 + (uint32_t)u * gthreads;
-            idxs[u] = i < n ? sp.list_idx[i] : 0;
-        }
-#pragma unroll
-        for (int u = 0; u < LB; ++u) {
-            const uint32_t key = keys[u];
-            if (key == NO_KEY) continue;
-            const int32_t idx = idxs[u];
-            bool sel = key > T;
-            if (key == T) {
-                uint32_t smaller = 0;
-                for (uint32_t s = 0; s < n_ties; ++s) smaller += sh.ties[s] < idx ? 1u : 0u;
-                sel = smaller < Q;
-            }
-            if (sel) atomicOr(&sp.bitmap[(uint32_t)idx >> 5], 1u << ((uint32_t)idx & 31));
-        }
-    }
-    __threadfence();
-    cluster.sync();
-
-    // ---- ordered compaction of the bitmap: each warp owns a contiguous run of words, read 32 at a time
-    const int64_t nwords = (d + 31) >> 5;
-    const int nwarps = gthreads / 32;
-    const int64_t per_warp = ((nwords + nwarps - 1) / nwarps + 31) / 32 * 32;
-    const int64_t w_lo = (int64_t)(gt >> 5) * per_warp;
-    const int64_t w_hi = w_lo + per_warp < nwords ? w_lo + per_warp : nwords;
-    constexpr int BATCH = 8;                                // bitmap words in flight per lane
-    uint32_t mine = 0;
-    for (int64_t wb = w_lo; wb < w_hi; wb += 32 * BATCH) {
-        uint32_t bits[BATCH];
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) {
-            const int64_t w = wb + u * 32 + lane;
-            bits[u] = w < w_hi ? __ldcg(sp.bitmap + w) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) mine += __popc(bits[u]);
-    }
-    for (int off = 16; off; off >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, off);   // warp total
-    if (lane == 0) sh.wsum[warp] = mine;
-    __syncthreads();
-    uint32_t before = 0, cta_sum = 0;
-    for (int w2 = 0; w2 < SPARSE_THREADS / 32; ++w2) { const uint32_t s2 = sh.wsum[w2]; if (w2 < warp) before += s2; cta_sum += s2; }
-    if (t == 0) sh0->cta_total[rank] = cta_sum;
-    cluster.sync();
-    for (unsigned r2 = 0; r2 < rank; ++r2) before += sh0->cta_total[r2];
-    uint32_t run = before;                                  // selected coordinates before this warp's next word group
-    for (int64_t wb = w_lo; wb < w_hi; wb += 32 * BATCH) {
-        uint32_t bits[BATCH];
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) {
-            const int64_t w = wb + u * 32 + lane;
-            bits[u] = w < w_hi ? __ldcg(sp.bitmap + w) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < BATCH; ++u) {
-            const int64_t w = wb + u * 32 + lane;
-            uint32_t b32 = bits[u];
-            const uint32_t c = __popc(b32);
-            uint32_t incl = c;
-            for (int off = 1; off < 32; off <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                if (lane >= off) incl += o;
-            }
-            uint32_t slot = run + incl - c;
-            while (b32) {
-                const int b = __ffs(b32) - 1;
-                b32 &= b32 - 1;
-                if (slot < ncand) cand_idx[slot] = (int32_t)((w << 5) + b);
-                ++slot;
-            }
-            run += __shfl_sync(0xFFFFFFFFu, incl, 31);
-        }
-    }
-    cluster.sync();                                         // CTA 0's shared memory stays alive until all are done
 }
 
 #endif  // __CUDACC__

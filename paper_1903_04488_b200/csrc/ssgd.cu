@@ -33,6 +33,7 @@
 #include "accum_ws.cuh"
 #include "estimate.cuh"
 #include "sparse_select.cuh"
+#include "list_select.cuh"
 #include "heavymix.cuh"
 #include "step_kernels.cuh"
 
@@ -55,8 +56,10 @@ struct ssgd_ctx {
     char* ws; size_t ws_bytes; int64_t ncand_max;
     // workspace layout (byte offsets)
     size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
-    size_t off_sp_hist, off_sp_state, off_bitmap, off_list_idx, off_list_est;   // sparse candidate path
-    int64_t list_cap;
+    size_t off_sp_hist, off_sp_state, off_maps, off_map_chunks, off_list_idx, off_list_est;   // early-exit path
+    size_t map_bytes;
+    int64_t list_cap, nchunk_map;
+    uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
     size_t off_hm;
     int32_t prune_mode;
     size_t persist_bytes;
@@ -107,9 +110,10 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_state_c = o; o += up(sizeof(SelState));
     x->off_hist_f = o;  o += up(SEL_HIST_WORDS * 4);
     x->off_state_f = o; o += up(sizeof(SelState));
-    x->off_sp_hist = o; o += up(2 * H1_BINS * 4);
+    x->off_sp_hist = o; o += up((size_t)(2 * H1_BINS + H2_BINS + H19_BINS) * 4);
     x->off_sp_state = o; o += up(sizeof(SparseState));
-    x->off_bitmap = o;  o += up((size_t)((x->d + 31) / 32) * 4);
+    x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
+    x->off_maps = o;    o += 2 * x->map_bytes;
     x->off_hm = o;      o += up(sizeof(HeavymixState));
     x->off_err = o;     o += up(16);
     x->zero_bytes = o;
@@ -120,8 +124,9 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_chunk_f = o; o += up((size_t)x->nchunk_f * 8);
     x->off_cand = o;    o += up((size_t)ncand_max * 4);
     x->off_xs = o;      o += up((size_t)ncand_max * 4);
-    x->list_cap = 4 * ncand_max > 65536 ? 4 * ncand_max : 65536;
-    if (x->list_cap > x->d) x->list_cap = x->d;
+    x->list_cap = x->d;                                  // the unpruned rerun may list every coordinate
+    x->nchunk_map = ((x->d + 31) / 32 + MAP_CHUNK_WORDS - 1) / MAP_CHUNK_WORDS;
+    x->off_map_chunks = o; o += up((size_t)x->nchunk_map * 8);
     x->off_list_idx = o; o += up((size_t)x->list_cap * 4);
     x->off_list_est = o; o += up((size_t)x->list_cap * 4);
     x->off_oidx = o;    o += up((size_t)x->k * 4);
@@ -379,11 +384,10 @@ int mark(ssgd_ctx* x, int which, cudaStream_t st) {
 }
 
 int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, float* cand_est,
-                    float* est, cudaStream_t st, bool timed = false, const uint32_t* gate = nullptr) {
+                    float* est, cudaStream_t st, bool timed = false) {
     UnsketchArgs A;
     A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk; A.est = est;
     SelBuffers sb = sel_buffers(x, false);
-    sb.gate = gate;
     A.sb = sb; A.want = (uint32_t)ncand;
     int e = launch_unsketch(x, A, st);
     if (e) return e;
@@ -398,12 +402,15 @@ int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* ca
 SparseBuffers sparse_buffers(ssgd_ctx* x) {
     SparseBuffers sp{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + x->off_sp_hist);
-    sp.h1_sample = h; sp.h1 = h + H1_BINS;
+    sp.h1_sample = h; sp.h1 = h + H1_BINS; sp.h2 = h + 2 * H1_BINS; sp.h19 = h + 2 * H1_BINS + H2_BINS;
     sp.state = reinterpret_cast<SparseState*>(x->ws + x->off_sp_state);
     sp.list_idx = reinterpret_cast<int32_t*>(x->ws + x->off_list_idx);
     sp.list_est = reinterpret_cast<float*>(x->ws + x->off_list_est);
     sp.cap = (uint32_t)x->list_cap;
-    sp.bitmap = reinterpret_cast<uint32_t*>(x->ws + x->off_bitmap);
+    sp.map_a = reinterpret_cast<uint32_t*>(x->ws + x->off_maps);
+    sp.map_b = reinterpret_cast<uint32_t*>(x->ws + x->off_maps + x->map_bytes);
+    sp.chunk_a = reinterpret_cast<uint32_t*>(x->ws + x->off_map_chunks);
+    sp.chunk_b = sp.chunk_a + x->nchunk_map;
     return sp;
 }
 
@@ -427,6 +434,12 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
                   grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID), SEL_THREADS, 0, A),
        "launch k_unsketch_pruned");
     LAUNCHED("k_unsketch_pruned");
+    SparseArgs B = A;
+    B.rerun = 1;                                         // returns at once unless the first pass kept too few
+    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>,
+                  grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID), SEL_THREADS, 0, B),
+       "launch k_unsketch_pruned (unpruned rerun)");
+    LAUNCHED("k_unsketch_pruned");
     return SSGD_OK;
 }
 
@@ -434,40 +447,35 @@ int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
     DISPATCH_R(launch_sparse_t, x, A, st)
 }
 
-int launch_select_sparse(ssgd_ctx* x, const SparseBuffers& sp, int64_t ncand, int32_t* cand_idx, cudaStream_t st) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(SPARSE_CLUSTER);
-    cfg.blockDim = dim3(SPARSE_THREADS);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cudaLaunchAttribute at[2];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = SPARSE_CLUSTER; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    at[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at;
-    cfg.numAttrs = pdl_enabled() ? 2 : 1;
-    CU(cudaLaunchKernelEx(&cfg, k_select_sparse, sp, x->d, (uint32_t)ncand, cand_idx), "launch k_select_sparse");
-    LAUNCHED("k_select_sparse");
-    return SSGD_OK;
-}
-
-// Line 9 with early exit: sample -> pruned unsketch -> cluster selection; the dense path follows, gated.
-int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, float* est,
-                           cudaStream_t st) {
+// Line 9 with early exit: sample -> pruned unsketch (-> unpruned rerun if the sample misjudged) -> selection on
+// the survivor list (list_select.cuh).
+int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, cudaStream_t st) {
     SparseArgs A;
     A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk;
     A.sp = sparse_buffers(x);
     A.ncand = (uint32_t)ncand;
+    A.rerun = 0;
     const int64_t groups = (x->d + 3) / 4;
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
     const double mean = (double)ncand * (double)(windows * 4) / (double)x->d;
-    A.want_sample = (uint32_t)(mean + 6.0 * std::sqrt(mean) + 16.0 + 1.0);
+    A.want_sample = x->sample_rank ? x->sample_rank : (uint32_t)(mean + 6.0 * std::sqrt(mean) + 16.0 + 1.0);
     int e = launch_sparse(x, A, st);
     if (e) return e;
     if ((e = mark(x, 2, st))) return e;
-    if ((e = launch_select_sparse(x, A.sp, ncand, cand_idx, st))) return e;
-    return unsketch_select(x, merged, ncand, cand_idx, nullptr, est, st, false, &A.sp.state->fallback);
+    // the list normally holds 1-2 x ncand entries; the kernels stride over whatever it holds
+    const int list_grid = grid_for(4 * ncand, SEL_THREADS * SEL_BATCH, (int64_t)x->sm_count * 8);
+    CU(launch_pdl(st, k_list_hist, list_grid, SEL_THREADS, 0, A.sp), "launch k_list_hist");
+    LAUNCHED("k_list_hist");
+    CU(launch_pdl(st, k_list_mark, list_grid, SEL_THREADS, 0, A.sp), "launch k_list_mark");
+    LAUNCHED("k_list_mark");
+    const int64_t nwords = (x->d + 31) / 32;
+    const int map_grid = grid_for(x->nchunk_map, 1, (int64_t)x->sm_count * 8);
+    CU(launch_pdl(st, k_map_count, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map), "launch k_map_count");
+    LAUNCHED("k_map_count");
+    CU(launch_pdl(st, k_map_emit, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map, (uint32_t)ncand, cand_idx),
+       "launch k_map_emit");
+    LAUNCHED("k_map_emit");
+    return SSGD_OK;
 }
 
 int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
@@ -535,7 +543,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -586,6 +594,12 @@ int ssgd_set_table_persistence(ssgd_ctx* x, int32_t enable) {
     if (carve == 0) return SSGD_OK;
     CU(cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, carve), "set persisting L2 size");
     x->persist_bytes = want;
+    return SSGD_OK;
+}
+
+int ssgd_set_prune_sample_rank(ssgd_ctx* x, int64_t rank) {
+    if (!x || rank < 0 || rank > 0x7FFFFFFF) return SSGD_EINVAL;
+    x->sample_rank = (uint32_t)rank;
     return SSGD_OK;
 }
 
@@ -749,7 +763,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);
     if (use_sparse(x, ncand)) {
-        if ((e = unsketch_select_sparse(x, merged, ncand, cand, est, st))) return e;
+        if ((e = unsketch_select_sparse(x, merged, ncand, cand, st))) return e;
     } else {
         if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
     }

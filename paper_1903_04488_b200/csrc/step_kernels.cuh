@@ -285,7 +285,6 @@ k_unsketch(const UnsketchArgs A) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += K3_THREADS) s_hist[b] = 0;
     pdl_wait();
-    if (gate_closed(A.sb.gate)) return;
     __syncthreads();
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     const int64_t stride = (int64_t)gridDim.x * K3_THREADS;

@@ -31,6 +31,7 @@ SIGNATURES = {
     "ssgd_set_insert_mode": [_vp, _i32],
     "ssgd_set_prune_mode": [_vp, _i32],
     "ssgd_set_insert_split": [_vp, _i64],
+    "ssgd_set_prune_sample_rank": [_vp, _i64],
     "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
@@ -145,6 +146,9 @@ class Ssgd:
 
     def set_prune_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_prune_mode(self._h, mode), "ssgd_set_prune_mode")
+
+    def set_prune_sample_rank(self, rank: int) -> None:
+        self._chk(self._lib.ssgd_set_prune_sample_rank(self._h, rank), "ssgd_set_prune_sample_rank")
 
     def set_insert_split(self, nbytes: int) -> None:
         self._chk(self._lib.ssgd_set_insert_split(self._h, nbytes), "ssgd_set_insert_split")

@@ -186,13 +186,12 @@ def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     assert idx.tolist() == list(range(cfg.k)) and (val == 0).all()
     if prune == S.PRUNE_ON:
         fell_back, survivors, bin_lo = eng.step_used_fallback()
-        assert fell_back and bin_lo == 0 and survivors == cfg.d     # d equal magnitudes: the dense path ranks them
+        assert not fell_back and bin_lo == 0 and survivors == cfg.d   # nothing can be pruned; d ties ranked by index
 
 
-def test_survivor_list_overflow_falls_back_to_the_dense_path(cuda_device):
-    """All estimates equal (zero): nothing can be pruned, the survivors (all d) do not fit the list, and the
-    gated dense path must produce the candidates; ties go to the smallest indices.  A normal gradient right
-    after it takes the pruned path again."""
+def test_nothing_to_prune_lists_every_coordinate(cuda_device):
+    """All estimates equal (zero): the sampled threshold is zero, every coordinate survives (the list has room
+    for all d), and the d-way tie at the threshold goes to the smallest indices."""
     cfg = wl.C2.scaled(d=300_001, W=2, c=1024, ncand=1000, k=500)
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_prune_mode(S.PRUNE_ON)
@@ -200,11 +199,27 @@ def test_survivor_list_overflow_falls_back_to_the_dense_path(cuda_device):
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     fell_back, survivors, bin_lo = eng.step_used_fallback()
-    assert fell_back and survivors == cfg.d and bin_lo == 0
+    assert not fell_back and survivors == cfg.d and bin_lo == 0
     assert idx.tolist() == list(range(cfg.k))
+
+
+def test_misjudged_threshold_reruns_without_pruning(cuda_device):
+    """A prune threshold set at the largest sampled estimate keeps far fewer than ncand coordinates: the last
+    block of the pruned pass must notice, and the unpruned pass behind it must produce the right candidates.
+    The next step, with the normal rank, prunes again."""
+    cfg = wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     st = wl.Structure(cfg, cuda_device)
+    eng.set_prune_sample_rank(1)
     check_step(orc, eng, wl.gradients(st, 0), cfg.rho, cfg.ncand, u_o, v_o)
-    assert not eng.step_used_fallback()[0]
+    fell_back, survivors, bin_lo = eng.step_used_fallback()
+    assert fell_back and survivors == cfg.d and bin_lo > 0
+    eng.set_prune_sample_rank(0)
+    check_step(orc, eng, wl.gradients(st, 1), cfg.rho, cfg.ncand, u_o, v_o)
+    fell_back, survivors, _ = eng.step_used_fallback()
+    assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
 
 
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
