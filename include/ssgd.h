@@ -66,13 +66,19 @@ extern "C" {
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
 #define SSGD_INSERT_WS     4  /* the same pipeline, warp-specialised: separate stream and sketch warps   */
 
-/* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  With pruning, coordinates that
- * provably cannot be among the ncand largest |estimate| stop reading sketch rows early (a median of r
- * values reaches a magnitude only if (r+1)/2 of them do); the candidates are identical either way.
- * AUTO prunes when 5 <= r <= 9, d >= 2^22 and ncand <= d/8 (elsewhere the fixed costs outweigh the saving). */
+/* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  A median of r values reaches a magnitude
+ * only if (r+1)/2 of them do, so with a threshold taken from a sample of the estimates most coordinates can be
+ * ruled out from "is this bucket's magnitude above the threshold" alone.  ON: that test is precomputed as one bit
+ * per bucket and kept in shared memory (if r*c bits, OR-folded up to 32 buckets per bit, fit; otherwise as
+ * EARLY_EXIT).  EARLY_EXIT: the test is applied to the table values themselves and a coordinate stops reading
+ * rows once it cannot pass.  OFF: every coordinate reads all r rows.  The candidates are identical in all modes.
+ * AUTO is ON when d >= 2^22, ncand <= d/8 (below that the fixed costs outweigh the saving) and either the bitmap
+ * fits unfolded or 5 <= r <= 9; else OFF.  Behind a folded bitmap ON measures the bitmap's density each step and
+ * runs the EARLY_EXIT kernel instead when the folded bits would rule out too few coordinates. */
 #define SSGD_PRUNE_AUTO 0
 #define SSGD_PRUNE_OFF  1
 #define SSGD_PRUNE_ON   2
+#define SSGD_PRUNE_EARLY_EXIT 3
 
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
 
@@ -89,7 +95,7 @@ int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
 int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
 /* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
  * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
- * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 48 MiB,
+ * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
  * which leaves tables up to that size untouched). */
 int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
 /* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
@@ -97,10 +103,12 @@ int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
  * device; the launches then carry an access-policy window over the table).  Off by default because the limit
  * is shared with everything else the process runs on that device.  enable = 0 stops attaching the window. */
 int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
-/* Diagnostics of the last ssgd_step's pruned path (waits for the stream): out[0] != 0 if the sampled
- * threshold kept fewer than ncand coordinates and the pass was redone without pruning, out[1] = number of
- * coordinates on the survivor list, out[2] = the prune threshold as a histogram-bin index (0: nothing pruned). */
-int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out3);
+/* Diagnostics of the last ssgd_step's pruned path (waits for the stream), five values: out[0] != 0 if the
+ * sampled threshold kept fewer than ncand coordinates and the pass was redone without pruning, out[1] = number
+ * of coordinates on the survivor list, out[2] = the prune threshold as a histogram-bin index (0: nothing
+ * pruned), out[3] = 1 if a folded bucket bitmap was too dense and the first pass read the table instead,
+ * out[4] = set bits of the folded bitmap (0 if the bitmap is not folded). */
+int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out5);
 /* For tests and diagnostics: the rank (from the top) in the sample's histogram that sets the prune threshold;
  * 0 = derive it from ncand (mean + 6 sigma + 16).  A rank of 1 puts the threshold at the largest sampled
  * estimate, which forces the unpruned rerun. */

@@ -1,0 +1,308 @@
+// filter_unsketch.cuh -- Algorithm 3 line 9, first pass over all d coordinates, with the sketch table replaced
+// by one bit per bucket held in shared memory.
+//
+// The early-exit unsketch of sparse_select.cuh still pays three or more scattered reads of the L2-resident table
+// per coordinate, and the load/store unit's rate for such reads (about one 32-byte sector per clock per SM) is
+// what bounds it.  The test it applies to each value read, "is |table[j][h_j(i)]| in a histogram bin >= bin_lo",
+// depends on the bucket alone, so it can be evaluated once per bucket instead of once per (coordinate, row):
+//
+//   k_bitmap_build     bit (j, b) = 1 iff the magnitude of table[j][b] lies in a bin >= bin_lo   (r*c bits)
+//   k_bitmap_fold      if r*c bits exceed the shared memory of an SM: OR 2^s neighbouring buckets into one bit,
+//                      s <= 5 (a coarser, still necessary, condition; the full bitmap stays in global memory)
+//   k_unsketch_filter  one block per SM copies the (folded) bitmap into shared memory; every thread walks a run of
+//                      consecutive coordinates (one add + conditional subtract per row hash) and counts, per
+//                      coordinate, the rows whose bit is set.  |median of r| >= t needs (r+1)/2 rows of magnitude
+//                      >= t, so a coordinate with fewer set bits is certainly below the threshold and is dropped
+//                      without a single read of global memory.  The few that pass (2 % at C2's shape) are queued
+//                      per warp in shared memory and processed 32 at a time: folded bitmaps are re-checked against
+//                      the full bitmap first (second queue), then the exact estimate is computed from the table
+//                      and the coordinate is appended to the survivor list iff its own bin is >= bin_lo.
+//
+// The survivor set is therefore exactly { i : bin(|est_i|) >= bin_lo }, as with the early-exit kernel, and the rest
+// of the stage (too-few-survivors rerun, selection on the list) is unchanged.
+#pragma once
+#include <stdint.h>
+
+#include "estimate.cuh"
+#include "hash.cuh"
+#include "select.cuh"
+#include "sparse_select.cuh"
+
+namespace ssgd {
+
+// Measured on B200 (C2; sample + bitmap + filter + the skipped rerun launch): 256 threads x 4 coordinates per
+// iteration 0.092 ms; 512 x 1, 2, 4: 0.073, 0.071, 0.073; 1024 x 1, 2: 0.070, 0.067.  With a folded bitmap the
+// kernel needs more than the 64 registers that 1024 threads leave it (d = 2e7, c = 2^20: 0.41 ms against 0.26 ms).
+#ifndef SSGD_FILTER_THREADS
+#define SSGD_FILTER_THREADS 512
+#endif
+#ifndef SSGD_FILTER_NC
+#define SSGD_FILTER_NC 2
+#endif
+constexpr int FILTER_THREADS = SSGD_FILTER_THREADS;
+constexpr int FILTER_WARPS = FILTER_THREADS / 32;
+constexpr int FILTER_QUEUE = 64;                         // entries per warp queue (at most 31 + 32 are ever held)
+constexpr int FILTER_MAX_WORDS = 49152;                  // 192 KiB of bitmap per SM (+ 16 KiB of queues + 16 KiB histogram)
+constexpr int FILTER_MAX_FOLD = 5;                       // a folded bit covers at most one word of the full bitmap
+// Shared memory of the filter kernel besides its static SelShared: the bitmap, then two queues per warp.
+constexpr size_t FILTER_QUEUE_BYTES = (size_t)FILTER_WARPS * 2 * (2 * FILTER_QUEUE) * 4;   // (value, tag) entries
+
+struct FilterArgs {
+    SparseArgs A;
+    uint32_t* bm_full;        // [r][stride_full] words: bit b of row j at word b >> 5, bit b & 31
+    uint32_t* bm_fold;        // [r][stride_fold] words (unused when fold == 0)
+    int32_t stride_full;      // words per row, a multiple of 4
+    int32_t stride_fold;      // words per row of the folded bitmap, a multiple of 4
+    int32_t fold;             // s: a folded bit covers buckets [q << s, (q + 1) << s)
+    int32_t r;
+};
+
+#ifdef __CUDACC__
+
+// ---- bit per bucket ------------------------------------------------------------------------------------------
+// One warp per 32 words (1024 buckets) of one row: 32 coalesced loads, a ballot each; lane k keeps ballot k.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_bitmap_build(const FilterArgs F) {
+    pdl_trigger();
+    pdl_wait();
+    const uint32_t bin_lo = __ldcg(&F.A.sp.state->bin_lo);
+    const int lane = threadIdx.x & 31;
+    const int64_t tasks_per_row = (F.stride_full + 31) / 32;
+    const int64_t tasks = tasks_per_row * F.r;
+    const int64_t nwarps = (int64_t)gridDim.x * SEL_WARPS;
+    for (int64_t task = (int64_t)blockIdx.x * SEL_WARPS + (threadIdx.x >> 5); task < tasks; task += nwarps) {
+        const int64_t j = task / tasks_per_row;
+        const int64_t w0 = (task - j * tasks_per_row) * 32;          // first word of this task in row j
+        const float* row = F.A.table + j * F.A.c;
+        uint32_t mine = 0;
+#pragma unroll 8
+        for (int k = 0; k < 32; ++k) {
+            const int64_t b = (w0 + k) * 32 + lane;
+            const bool big = b < F.A.c && (key_of(__ldcg(row + b)) >> H1_SHIFT) >= bin_lo;
+            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, big);
+            if (lane == k) mine = bal;
+        }
+        if (w0 + lane < F.stride_full) F.bm_full[j * F.stride_full + w0 + lane] = mine;
+    }
+}
+
+// Probability that at least `need` of r independent bits of density p are set.
+__device__ __forceinline__ float binomial_tail(int r, int need, float p) {
+    float tail = 0.f;
+    for (int k = need; k <= r; ++k) {
+        float term = 1.f;                                  // C(r, k) p^k (1-p)^(r-k)
+        for (int t = 0; t < k; ++t) term *= p * (float)(r - t) / (float)(k - t);
+        for (int t = 0; t < r - k; ++t) term *= 1.f - p;
+        tail += term;
+    }
+    return tail;
+}
+
+// A folded bitmap is used only if it passes at most this share of the coordinates (estimated from its density as
+// a binomial tail); otherwise the first pass reads the table.  Measured on B200, r = 5, whole step in ms with the
+// filter / with the table kernel, by estimated share: 0.63 (d = 2e7, c = 2^20, 4 buckets per bit) 2.70 / 2.84;
+// 0.77 (same, ncand doubled) 2.79 / 2.89; 0.86 (ncand x 4) 2.92 / 2.96; 0.88 (d = 9e7, c = 1e6, 4 per bit)
+// 4.83 / 4.92; 0.68 with a 2.6 MB full bitmap behind it (d = 1.1e7, c = 2^22, 16 per bit) 1.25 / 1.25;
+// 0.99 (d = 9e7, c = 2^22, 16 per bit) 9.6 / 8.3; r = 15, 0.95 (d = 9e7, c = 180,000, 2 per bit) 16.7 / 12.5.
+#ifndef SSGD_FILTER_MAX_PASS
+#define SSGD_FILTER_MAX_PASS 0.8f
+#endif
+
+// One thread per folded word: 32 folded bits, each the OR of 2^s consecutive bits of the full bitmap.  The last
+// block to finish turns the density of the folded bitmap into the decision between the two first-pass kernels.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_bitmap_fold(const FilterArgs F) {
+    __shared__ uint32_t s_last;
+    pdl_trigger();
+    pdl_wait();
+    const int s = F.fold;
+    const int64_t total = (int64_t)F.r * F.stride_fold;
+    const uint32_t group = s >= 5 ? 0xFFFFFFFFu : ((1u << (1 << s)) - 1u);
+    uint32_t ones = 0;
+    for (int64_t t = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; t < total; t += (int64_t)gridDim.x * SEL_THREADS) {
+        const int64_t j = t / F.stride_fold;
+        const int64_t fw = t - j * F.stride_fold;
+        const uint32_t* src = F.bm_full + j * F.stride_full;
+        uint32_t out = 0;
+        for (int q = 0; q < 32; ++q) {
+            const int64_t w = (fw << s) + (q >> (5 - s));            // word of the full row holding this group
+            const int off = (q << s) & 31;
+            const uint32_t word = w < F.stride_full ? __ldcg(src + w) : 0u;
+            out |= (((word >> off) & group) != 0u ? 1u : 0u) << q;
+        }
+        F.bm_fold[t] = out;
+        ones += __popc(out);
+    }
+    for (int off = 16; off; off >>= 1) ones += __shfl_xor_sync(0xFFFFFFFFu, ones, off);
+    if ((threadIdx.x & 31) == 0 && ones) atomicAdd(&F.A.sp.state->fold_ones, ones);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(&F.A.sp.state->ticket[5], 1u) == gridDim.x - 1 ? 1u : 0u;
+    __syncthreads();
+    if (s_last && threadIdx.x == 0) {
+        const float bits = (float)F.r * (float)((F.A.c + (1 << s) - 1) >> s);
+        const float p = fminf(1.f, (float)__ldcg(&F.A.sp.state->fold_ones) / bits);
+        F.A.sp.state->use_table = binomial_tail(F.r, (F.r + 1) / 2, p) > SSGD_FILTER_MAX_PASS ? 1u : 0u;
+    }
+}
+
+// ---- the filter pass ---------------------------------------------------------------------------------------------
+struct WarpQueue {
+    uint32_t* buf;     // FILTER_QUEUE entries of this warp in shared memory, then FILTER_QUEUE tags
+    int count;         // warp-uniform
+    // every lane calls; lanes with `take` append (value, tag)
+    __device__ __forceinline__ void push(bool take, uint32_t value, uint32_t tag, int lane) {
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, take);
+        if (bal == 0u) return;
+        if (take) {
+            const int pos = count + __popc(bal & ((1u << lane) - 1u));
+            buf[pos] = value;
+            buf[FILTER_QUEUE + pos] = tag;
+        }
+        count += __popc(bal);
+        __syncwarp();
+    }
+    // every lane calls; removes up to 32 entries from the top; returns whether this lane got one
+    __device__ __forceinline__ bool pop(uint32_t& value, uint32_t& tag, int lane) {
+        const int n = count < 32 ? count : 32;
+        const bool got = lane < n;
+        if (got) { value = buf[count - n + lane]; tag = buf[FILTER_QUEUE + count - n + lane]; }
+        count -= n;
+        __syncwarp();
+        return got;
+    }
+};
+
+template <int R, bool POW2, bool FOLD>
+__global__ void __launch_bounds__(FILTER_THREADS, 1)
+k_unsketch_filter(const FilterArgs F) {
+    __shared__ SelShared sh;
+    extern __shared__ __align__(16) uint32_t dyn[];
+    constexpr int NEED = (R + 1) / 2;
+    const SparseArgs& A = F.A;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int fold = FOLD ? F.fold : 0;                  // FOLD == (F.fold != 0)
+    const int stride_s = fold ? F.stride_fold : F.stride_full;
+    const int nw = R * stride_s;
+    uint32_t* bm = dyn;
+    WarpQueue q2{dyn + nw + (warp * 2 + 0) * (2 * FILTER_QUEUE), 0};
+    WarpQueue q3{dyn + nw + (warp * 2 + 1) * (2 * FILTER_QUEUE), 0};
+    pdl_trigger();
+    for (int b = threadIdx.x; b < H1_BINS; b += FILTER_THREADS) sh.hist[b] = 0;
+    pdl_wait();
+    if (FOLD && __ldcg(&A.sp.state->use_table) != 0u) return;   // too dense to prune: the table kernel behind runs
+    const uint32_t bin_lo = __ldcg(&A.sp.state->bin_lo);
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(fold ? F.bm_fold : F.bm_full);
+        uint4* dst = reinterpret_cast<uint4*>(bm);
+        for (int w = threadIdx.x; w < nw / 4; w += FILTER_THREADS) dst[w] = __ldcg(src + w);
+    }
+    __syncthreads();
+
+    // exact estimate of one queued coordinate; append to the list iff its bin is >= bin_lo
+    auto exact = [&](uint32_t i, bool have) {
+        float m = 0.f;
+        bool keep = false;
+        if (have) {
+            float rowv[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                uint32_t hb[1];
+                row_hashes<POW2, 1>(A.hp.row[j], A.bk, i, hb);
+                rowv[j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[0] & P31)), hb[0]);
+            }
+            m = median_of<R>(rowv);
+            keep = (key_of(m) >> H1_SHIFT) >= bin_lo;
+        }
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
+        if (bal == 0u) return;
+        uint32_t base = 0;
+        if (lane == 0) base = atomicAdd(&A.sp.state->n_surv, (uint32_t)__popc(bal));
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        if (keep) {
+            const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
+            if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)i; A.sp.list_est[pos] = m; }
+            atomicAdd(&sh.hist[key_of(m) >> H1_SHIFT], 1u);
+        }
+    };
+    // folded bitmaps only: the rows whose folded bit was set (`rows`) are looked up in the full bitmap (global
+    // memory, L2-resident); the other rows are known to be below the threshold
+    auto recheck = [&](uint32_t i, uint32_t rows, bool have) {
+        bool pass = false;
+        if (have) {
+            uint32_t word[R], b[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j) {                // all loads issued before any is used
+                b[j] = bucket_of<POW2>(lin_hash(A.hp.row[j].a, A.hp.row[j].b, i), A.bk);
+                word[j] = 0u;
+                if ((rows >> j) & 1u) word[j] = __ldg(F.bm_full + (int64_t)j * F.stride_full + (b[j] >> 5));
+            }
+            int cnt = 0;
+#pragma unroll
+            for (int j = 0; j < R; ++j) cnt += (int)(__funnelshift_r(word[j], 0u, b[j]) & 1u);
+            pass = cnt >= NEED;
+        }
+        q3.push(pass, i, 0u, lane);
+        if (q3.count >= 32) { uint32_t c = 0, tag = 0; const bool got = q3.pop(c, tag, lane); exact(c, got); }
+    };
+    auto drain2 = [&]() {
+        uint32_t c = 0, rows = 0;
+        const bool got = q2.pop(c, rows, lane);
+        if (FOLD) recheck(c, rows, got); else exact(c, got);
+    };
+
+    // this thread's run of consecutive coordinates
+    const uint32_t total_threads = gridDim.x * FILTER_THREADS;
+    constexpr int NC = SSGD_FILTER_NC;                   // coordinates per loop iteration (independent lookups)
+    const uint32_t per = (uint32_t)((A.d + total_threads - 1) / total_threads + NC - 1) / NC * NC;
+    const uint32_t gtid = blockIdx.x * FILTER_THREADS + threadIdx.x;
+    const uint64_t begin64 = (uint64_t)gtid * per;
+    const uint32_t i_begin = begin64 < (uint64_t)A.d ? (uint32_t)begin64 : (uint32_t)A.d;
+    const uint32_t i_end = begin64 + per < (uint64_t)A.d ? (uint32_t)(begin64 + per) : (uint32_t)A.d;
+    uint32_t y[R];
+    const uint32_t* row_base[R];
+#pragma unroll
+    for (int j = 0; j < R; ++j) { y[j] = lin_hash(A.hp.row[j].a, A.hp.row[j].b, i_begin); row_base[j] = bm + j * stride_s; }
+    for (uint32_t t = 0; t < per; t += NC) {             // warp-uniform trip count
+        uint32_t rows[NC];                               // bit j: row j's bit is set
+#pragma unroll
+        for (int e = 0; e < NC; ++e) rows[e] = 0;
+#pragma unroll
+        for (int e = 0; e < NC; ++e) {
+#pragma unroll
+            for (int j = 0; j < R; ++j) {
+                const uint32_t b = bucket_of<POW2>(y[j], A.bk) >> fold;
+                const uint32_t bit = __funnelshift_r(row_base[j][b >> 5], 0u, b) & 1u;   // shift amount taken mod 32
+                if (FOLD) rows[e] |= bit << j; else rows[e] += bit;
+                y[j] = next_hash(y[j], A.hp.row[j].a);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < NC; ++e) {
+            const uint32_t i = i_begin + t + e;
+            const int cnt = FOLD ? __popc(rows[e]) : (int)rows[e];
+            q2.push(i < i_end && cnt >= NEED, i, rows[e], lane);
+            if (q2.count >= 32) drain2();
+        }
+    }
+    if (q2.count > 0) drain2();
+    if (FOLD && q3.count > 0) { uint32_t c = 0, tag = 0; const bool got = q3.pop(c, tag, lane); exact(c, got); }
+
+    __syncthreads();
+    flush_hist<H1_BINS>(sh.hist, A.sp.h1);
+    if (block_is_last(&A.sp.state->ticket[1], sh)) {
+        const uint32_t n = __ldcg(&A.sp.state->n_surv);
+        if (n < A.ncand) {
+            // the sampled threshold was too high: empty the list and its histogram for the unpruned pass
+            for (int b = threadIdx.x; b < H1_BINS; b += FILTER_THREADS) A.sp.h1[b] = 0;
+            if (threadIdx.x == 0) { A.sp.state->n_surv = 0; A.sp.state->fallback = 1u; }
+        } else {
+            uint32_t d1 = 0, rem1 = 1;
+            block_find_from_top<H1_BINS>(A.sp.h1, A.ncand, sh, d1, rem1);
+            if (threadIdx.x == 0) { A.sp.state->d1 = d1; A.sp.state->rem1 = rem1; }
+        }
+    }
+}
+
+#endif  // __CUDACC__
+}  // namespace ssgd

@@ -87,35 +87,41 @@ __device__ __forceinline__ bool block_is_last(uint32_t* ticket, SelShared& sh) {
 }
 
 // Largest digit D with count(bins > D) < want <= count(bins >= D); rem = want - count(bins > D).
-// Whole block (SEL_THREADS threads) must call.  Requires 1 <= want <= total count.
+// The whole block must call (SEL_THREADS threads or more; the first SEL_THREADS do the search).
+// Requires 1 <= want <= total count.
 template <int NBINS>
 __device__ __forceinline__ void block_find_from_top(const uint32_t* __restrict__ gh, uint32_t want,
                                                     SelShared& sh, uint32_t& digit, uint32_t& rem) {
     constexpr int PER = NBINS / SEL_THREADS;  // 16, 8, 1
     static_assert(PER >= 1 && PER * SEL_THREADS == NBINS, "bins must be a multiple of the block");
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    for (int b = t; b < NBINS; b += SEL_THREADS) sh.hist[b] = __ldcg(gh + b);  // L2: other blocks' atomics
+    const bool searcher = t < SEL_THREADS;    // warp-uniform
+    for (int b = t; b < NBINS; b += blockDim.x) sh.hist[b] = __ldcg(gh + b);  // L2: other blocks' atomics
     if (t == 0) { sh.found[0] = 0; sh.found[1] = 1; }
     __syncthreads();
-    uint32_t sum = 0;
+    uint32_t sum = 0, incl = 0;
+    if (searcher) {
 #pragma unroll
-    for (int s = 0; s < PER; ++s) sum += sh.hist[t * PER + ((s + t) % PER)];  // rotated: no bank conflicts
-    uint32_t incl = sum;  // sum over lanes >= lane of this warp
+        for (int s = 0; s < PER; ++s) sum += sh.hist[t * PER + ((s + t) % PER)];  // rotated: no bank conflicts
+        incl = sum;  // sum over lanes >= lane of this warp
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, incl, off);
-        if (lane + off < 32) incl += o;
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, incl, off);
+            if (lane + off < 32) incl += o;
+        }
+        if (lane == 0) sh.warp_sum[warp] = incl;
     }
-    if (lane == 0) sh.warp_sum[warp] = incl;
     __syncthreads();
-    uint32_t above = incl - sum;
-    for (int w2 = warp + 1; w2 < SEL_WARPS; ++w2) above += sh.warp_sum[w2];
-    if (above < want && want <= above + sum) {
-        uint32_t acc = above;
-        for (int b = t * PER + PER - 1; b >= t * PER; --b) {
-            const uint32_t h = sh.hist[b];
-            if (acc + h >= want) { sh.found[0] = (uint32_t)b; sh.found[1] = want - acc; break; }
-            acc += h;
+    if (searcher) {
+        uint32_t above = incl - sum;
+        for (int w2 = warp + 1; w2 < SEL_WARPS; ++w2) above += sh.warp_sum[w2];
+        if (above < want && want <= above + sum) {
+            uint32_t acc = above;
+            for (int b = t * PER + PER - 1; b >= t * PER; --b) {
+                const uint32_t h = sh.hist[b];
+                if (acc + h >= want) { sh.found[0] = (uint32_t)b; sh.found[1] = want - acc; break; }
+                acc += h;
+            }
         }
     }
     __syncthreads();

@@ -42,8 +42,10 @@ struct SparseState {                              // zeroed before the step
     uint32_t d1, rem1;     // first threshold digit of the survivors' histogram H1 and the count wanted inside it
     uint32_t thr_key;      // T: the exact 31-bit threshold key
     uint32_t quota_eq;     // Q: how many items with key == T are selected (smallest coordinates first)
-    uint32_t ticket[6];    // finished-block counters: sample, pruned, unpruned rerun, list histogram, map count
-    uint32_t pad[3];
+    uint32_t ticket[6];    // finished-block counters: sample, first pass, unpruned rerun, list histogram, map count, fold
+    uint32_t fold_ones;    // set bits of the folded bucket bitmap (filter_unsketch.cuh)
+    uint32_t use_table;    // 1: the folded bitmap is too dense to prune; the first pass reads the table instead
+    uint32_t pad[1];
 };
 
 struct SparseBuffers {
@@ -68,6 +70,7 @@ struct SparseArgs {
     uint32_t ncand;
     uint32_t want_sample;  // rank (from the top) in the sample's histogram that defines bin_lo
     int32_t rerun;         // 0: the pruned pass; 1: the unpruned pass behind it (runs only if fallback == 1)
+    int32_t gated;         // 1: the pruned pass runs only if use_table is set (it follows a bitmap filter that declined)
 };
 
 #ifdef __CUDACC__
@@ -140,6 +143,7 @@ k_unsketch_pruned(const SparseArgs A) {
     for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
     if (A.rerun && __ldcg(&A.sp.state->fallback) != 1u) return;
+    if (A.gated && __ldcg(&A.sp.state->use_table) == 0u) return;
     const uint32_t bin_lo = A.rerun ? 0u : A.sp.state->bin_lo;
     __syncthreads();
     const int lane = threadIdx.x & 31;

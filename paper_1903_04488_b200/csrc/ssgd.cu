@@ -33,6 +33,7 @@
 #include "accum_ws.cuh"
 #include "estimate.cuh"
 #include "sparse_select.cuh"
+#include "filter_unsketch.cuh"
 #include "list_select.cuh"
 #include "heavymix.cuh"
 #include "step_kernels.cuh"
@@ -59,6 +60,9 @@ struct ssgd_ctx {
     size_t off_sp_hist, off_sp_state, off_maps, off_map_chunks, off_list_idx, off_list_est;   // early-exit path
     size_t map_bytes;
     int64_t list_cap, nchunk_map;
+    size_t off_bm_full, off_bm_fold;                       // bit-per-bucket filter (filter_unsketch.cuh)
+    int32_t bm_stride_full, bm_stride_fold, bm_fold;       // bm_fold < 0: the bitmap cannot be folded into shared memory
+    bool filter_ready;                                     // shared-memory attribute of the filter kernel set
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
     size_t off_hm;
     int32_t prune_mode;
@@ -131,6 +135,16 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_list_est = o; o += up((size_t)x->list_cap * 4);
     x->off_oidx = o;    o += up((size_t)x->k * 4);
     x->off_oval = o;    o += up((size_t)x->k * 4);
+    // bit-per-bucket filter: rows padded to 16 bytes; folded by 2^s until r rows fit the shared-memory budget
+    auto round4 = [](int64_t w) { return (w + 3) / 4 * 4; };
+    const int64_t sf = round4((x->c + 31) / 32);
+    int s = 0;
+    while (s <= FILTER_MAX_FOLD && x->r * round4((sf + (1 << s) - 1) >> s) > FILTER_MAX_WORDS) ++s;
+    x->bm_stride_full = (int32_t)sf;
+    x->bm_fold = s <= FILTER_MAX_FOLD ? s : -1;
+    x->bm_stride_fold = s <= FILTER_MAX_FOLD ? (int32_t)round4((sf + (1 << s) - 1) >> s) : 0;
+    x->off_bm_full = o; o += up((size_t)x->r * sf * 4);
+    x->off_bm_fold = o; o += up((size_t)x->r * x->bm_stride_fold * 4);
     x->total_bytes = o;
 }
 
@@ -414,13 +428,22 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
     return sp;
 }
 
-// Whether ssgd_step takes the early-exit unsketch + sparse selection (sparse_select.cuh).
+// Whether ssgd_step takes the pruned first pass + selection on the survivor list (filter_unsketch.cuh,
+// sparse_select.cuh, list_select.cuh) instead of the dense unsketch + selection over all d estimates.
 bool use_sparse(const ssgd_ctx* x, int64_t ncand) {
     if (x->prune_mode == SSGD_PRUNE_OFF) return false;
-    if (x->prune_mode == SSGD_PRUNE_ON) return true;
-    // measured at C2's shape: the early exit saves 25-45 us for r = 5, 7, 9 and costs 34 us for r = 3 (only one
-    // row can be skipped); at r = 15 with ncand = 1.6e6 the dense kernel is faster (4.78 vs 5.72 ms)
-    return x->r >= 5 && x->r <= 9 && x->d >= (1 << 22) && ncand * 8 <= x->d;
+    if (x->prune_mode == SSGD_PRUNE_ON || x->prune_mode == SSGD_PRUNE_EARLY_EXIT) return true;
+    if (x->d < (1 << 22) || ncand * 8 > x->d) return false;      // fixed costs outweigh the saving
+    // an unfolded bucket bitmap pays for every r; behind a folded one the table kernel may have to run, which was
+    // measured to pay for r = 5, 7, 9 only (r = 3: one row can be skipped; r = 15, ncand = 1.6e6: 5.8 vs 4.9 ms)
+    return x->bm_fold == 0 || (x->r >= 5 && x->r <= 9);
+}
+
+// The first pass over all coordinates: the bit-per-bucket filter when the (folded) bitmap fits an SM's shared
+// memory, else the early-exit kernel that reads the table.
+bool use_filter(const ssgd_ctx* x) {
+    return x->prune_mode != SSGD_PRUNE_EARLY_EXIT && x->bm_fold >= 0 &&
+           sizeof(SelShared) + FILTER_QUEUE_BYTES + (size_t)FILTER_MAX_WORDS * 4 <= (size_t)x->max_smem_optin;
 }
 
 template <int R, bool POW2>
@@ -430,15 +453,47 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
     CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count), SEL_THREADS, 0, A),
        "launch k_unsketch_sample");
     LAUNCHED("k_unsketch_sample");
-    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>,
-                  grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID), SEL_THREADS, 0, A),
-       "launch k_unsketch_pruned");
-    LAUNCHED("k_unsketch_pruned");
+    const int pruned_grid = grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID);
+    if (use_filter(x)) {
+        FilterArgs F;
+        F.A = A;
+        F.bm_full = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_full);
+        F.bm_fold = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_fold);
+        F.stride_full = x->bm_stride_full; F.stride_fold = x->bm_stride_fold; F.fold = x->bm_fold; F.r = x->r;
+        const int64_t build_tasks = (int64_t)x->r * ((x->bm_stride_full + 31) / 32);
+        CU(launch_pdl(st, k_bitmap_build, grid_for(build_tasks, SEL_WARPS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, F),
+           "launch k_bitmap_build");
+        LAUNCHED("k_bitmap_build");
+        if (F.fold) {
+            CU(launch_pdl(st, k_bitmap_fold, grid_for((int64_t)x->r * F.stride_fold, SEL_THREADS, (int64_t)x->sm_count * 8),
+                          SEL_THREADS, 0, F), "launch k_bitmap_fold");
+            LAUNCHED("k_bitmap_fold");
+        }
+        auto kern = F.fold ? k_unsketch_filter<R, POW2, true> : k_unsketch_filter<R, POW2, false>;
+        const size_t smem = (size_t)x->r * (F.fold ? F.stride_fold : F.stride_full) * 4 + FILTER_QUEUE_BYTES;
+        if (!x->filter_ready) {
+            CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)((size_t)FILTER_MAX_WORDS * 4 + FILTER_QUEUE_BYTES)), "smem attribute");
+            x->filter_ready = true;
+        }
+        CU(launch_pdl(st, kern, grid_for(A.d, FILTER_THREADS, (int64_t)x->sm_count), FILTER_THREADS, smem, F),
+           "launch k_unsketch_filter");
+        LAUNCHED("k_unsketch_filter");
+        if (F.fold) {                                    // runs only if the folded bitmap turned out too dense
+            SparseArgs G = A;
+            G.gated = 1;
+            // plain stream order, no programmatic launch: measured on B200, blocks of this kernel that become
+            // resident while the declining filter kernel drains cost 4 ms (d = 9e7)
+            k_unsketch_pruned<R, POW2><<<pruned_grid, SEL_THREADS, 0, st>>>(G);
+            LAUNCHED("k_unsketch_pruned");
+        }
+    } else {
+        CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, A), "launch k_unsketch_pruned");
+        LAUNCHED("k_unsketch_pruned");
+    }
     SparseArgs B = A;
     B.rerun = 1;                                         // returns at once unless the first pass kept too few
-    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>,
-                  grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID), SEL_THREADS, 0, B),
-       "launch k_unsketch_pruned (unpruned rerun)");
+    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, B), "launch k_unsketch_pruned (unpruned rerun)");
     LAUNCHED("k_unsketch_pruned");
     return SSGD_OK;
 }
@@ -455,6 +510,7 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     A.sp = sparse_buffers(x);
     A.ncand = (uint32_t)ncand;
     A.rerun = 0;
+    A.gated = 0;
     const int64_t groups = (x->d + 3) / 4;
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
     const double mean = (double)ncand * (double)(windows * 4) / (double)x->d;
@@ -543,7 +599,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -610,7 +666,7 @@ int ssgd_set_insert_split(ssgd_ctx* x, int64_t bytes) {
 }
 
 int ssgd_set_prune_mode(ssgd_ctx* x, int32_t mode) {
-    if (!x || mode < SSGD_PRUNE_AUTO || mode > SSGD_PRUNE_ON) return SSGD_EINVAL;
+    if (!x || mode < SSGD_PRUNE_AUTO || mode > SSGD_PRUNE_EARLY_EXIT) return SSGD_EINVAL;
     x->prune_mode = mode;
     return SSGD_OK;
 }
@@ -623,6 +679,7 @@ int ssgd_step_used_fallback(ssgd_ctx* x, void* stream, int32_t* out) {
     SparseState s;
     CU(cudaMemcpy(&s, x->ws + x->off_sp_state, sizeof(s), cudaMemcpyDeviceToHost), "read sparse state");
     out[0] = (int32_t)s.fallback; out[1] = (int32_t)s.n_surv; out[2] = (int32_t)s.bin_lo;
+    out[3] = (int32_t)s.use_table; out[4] = (int32_t)s.fold_ones;
     return SSGD_OK;
 }
 

@@ -12,14 +12,15 @@
 #include "hash.cuh"
 #include "select.cuh"
 
+// Table bytes one insert kernel may scatter into; larger tables are inserted in row slices.  Measured on B200
+// (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each): 1 row per kernel 6.43 ms, 2 rows 6.25, 3 rows 6.60,
+// 4 rows 6.89, all 5 rows in one kernel 7.80.
+#ifndef SSGD_SPLIT_BYTES_DEFAULT
+#define SSGD_SPLIT_BYTES_DEFAULT ((size_t)40 << 20)
+#endif
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
-#ifndef SSGD_SPLIT_BYTES_DEFAULT
-// measured on B200 (C4: d = 9e7, W = 16, 5 x 4,194,304 = 80 MB table): unsplit 7.80 ms, 48 MB or 32 MB slices 6.26 ms,
-// 16 MB slices 6.44 ms
-#define SSGD_SPLIT_BYTES_DEFAULT ((size_t)48 << 20)
-#endif
 #ifndef SSGD_PRUNED_GRID
 #define SSGD_PRUNED_GRID 4
 #endif

@@ -17,7 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libssgd.so")
 OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA, INSERT_WS = 0, 1, 2, 3, 4
-PRUNE_AUTO, PRUNE_OFF, PRUNE_ON = 0, 1, 2
+PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT = 0, 1, 2, 3
 FMT_F16, FMT_BF16 = 0, 1
 MAX_R = 15
 
@@ -157,10 +157,16 @@ class Ssgd:
         self._chk(self._lib.ssgd_set_table_persistence(self._h, 1 if enable else 0), "ssgd_set_table_persistence")
 
     def step_used_fallback(self):
-        """(fell back to the dense path?, survivors of the early exit, prune threshold bin) of the last step."""
-        out = (_i32 * 3)()
+        """(redone without pruning?, survivors on the list, prune threshold bin) of the last step."""
+        out = (_i32 * 5)()
         self._chk(self._lib.ssgd_step_used_fallback(self._h, _stream(), out), "ssgd_step_used_fallback")
         return bool(out[0]), int(out[1]), int(out[2])
+
+    def step_first_pass(self):
+        """(folded bitmap declined and the table was read instead?, set bits of the folded bitmap) of the last step."""
+        out = (_i32 * 5)()
+        self._chk(self._lib.ssgd_step_used_fallback(self._h, _stream(), out), "ssgd_step_used_fallback")
+        return bool(out[3]), int(out[4])
 
     def workspace_bytes(self, ncand_max: int) -> int:
         out = _sz()

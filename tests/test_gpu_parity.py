@@ -156,11 +156,11 @@ STEP_CASES = [
 
 @pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
 @pytest.mark.parametrize("mode", [S.INSERT_WS, S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
 def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
     if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
         pytest.skip("table does not fit the shared-memory variant")
-    if prune == S.PRUNE_ON and mode != S.INSERT_GLOBAL:
+    if prune != S.PRUNE_OFF and mode != S.INSERT_GLOBAL:
         pytest.skip("the candidate path does not depend on the insert variant: one combination suffices")
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_insert_mode(mode)
@@ -175,7 +175,7 @@ def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
         assert all(r["final_sym_diff_vs_unadopted"] == 0 for r in report)
 
 
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
 def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     cfg = wl.C2.scaled(d=10_001, W=3, c=256, ncand=700, k=300)
     eng, orc, u, v = make(cfg, cuda_device)
@@ -184,17 +184,18 @@ def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     assert idx.tolist() == list(range(cfg.k)) and (val == 0).all()
-    if prune == S.PRUNE_ON:
+    if prune != S.PRUNE_OFF:
         fell_back, survivors, bin_lo = eng.step_used_fallback()
         assert not fell_back and bin_lo == 0 and survivors == cfg.d   # nothing can be pruned; d ties ranked by index
 
 
-def test_nothing_to_prune_lists_every_coordinate(cuda_device):
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT])
+def test_nothing_to_prune_lists_every_coordinate(cuda_device, prune):
     """All estimates equal (zero): the sampled threshold is zero, every coordinate survives (the list has room
     for all d), and the d-way tie at the threshold goes to the smallest indices."""
     cfg = wl.C2.scaled(d=300_001, W=2, c=1024, ncand=1000, k=500)
     eng, orc, u, v = make(cfg, cuda_device)
-    eng.set_prune_mode(S.PRUNE_ON)
+    eng.set_prune_mode(prune)
     g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
@@ -203,13 +204,14 @@ def test_nothing_to_prune_lists_every_coordinate(cuda_device):
     assert idx.tolist() == list(range(cfg.k))
 
 
-def test_misjudged_threshold_reruns_without_pruning(cuda_device):
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT])
+def test_misjudged_threshold_reruns_without_pruning(cuda_device, prune):
     """A prune threshold set at the largest sampled estimate keeps far fewer than ncand coordinates: the last
     block of the pruned pass must notice, and the unpruned pass behind it must produce the right candidates.
     The next step, with the normal rank, prunes again."""
     cfg = wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000)
     eng, orc, u, v = make(cfg, cuda_device)
-    eng.set_prune_mode(S.PRUNE_ON)
+    eng.set_prune_mode(prune)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     st = wl.Structure(cfg, cuda_device)
     eng.set_prune_sample_rank(1)
@@ -222,7 +224,7 @@ def test_misjudged_threshold_reruns_without_pruning(cuda_device):
     assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
 
 
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_OFF])
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
 def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
     cfg = wl.C2.scaled(d=40_000, W=2, r=1, c=40_000, ncand=1000, k=400)
@@ -258,12 +260,13 @@ def test_row_split_insert(cuda_device):
     assert eng.launch_count() - n0 > 0
 
 
-def test_pruned_path_is_taken_and_prunes(cuda_device):
-    """On a gradient-shaped input the early-exit path must do its job: no fall-back, a non-trivial
-    threshold, at least ncand survivors and far fewer than d; a few ties at the threshold are ranked by index."""
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT])
+def test_pruned_path_is_taken_and_prunes(cuda_device, prune):
+    """On a gradient-shaped input the pruned path must do its job: no rerun, a non-trivial threshold, at
+    least ncand survivors and far fewer than d; a few ties at the threshold are ranked by index."""
     cfg = wl.C2.scaled(d=600_001, W=4, c=16_384, ncand=6000, k=3000)
     eng, orc, u, v = make(cfg, cuda_device)
-    eng.set_prune_mode(S.PRUNE_ON)
+    eng.set_prune_mode(prune)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     st = wl.Structure(cfg, cuda_device)
     for t in range(2):
@@ -271,6 +274,49 @@ def test_pruned_path_is_taken_and_prunes(cuda_device):
         fell_back, survivors, bin_lo = eng.step_used_fallback()
         assert not fell_back and bin_lo > 0
         assert cfg.ncand <= survivors <= cfg.d // 10
+
+
+FOLD_CASES = [
+    wl.C3.scaled(d=600_011, W=3, r=5, c=524_288, ncand=5000, k=2000),       # 5 x 2^19 bits: two buckets per bit
+    wl.P1.scaled(d=400_003, W=2, r=15, c=180_000, ncand=8000, k=500),       # the paper's 15 x 180,000: two per bit
+    wl.C4.scaled(d=500_009, W=2, r=5, c=6_000_001, ncand=4000, k=1000),     # 32 buckets per bit, c not a power of two
+]
+
+
+@pytest.mark.parametrize("cfg", FOLD_CASES, ids=lambda c: f"{c.name}-r{c.r}-c{c.c}")
+def test_bucket_bitmap_folded_into_shared_memory(cuda_device, cfg):
+    """Sketches whose one-bit-per-bucket filter exceeds an SM's shared memory: neighbouring buckets share a bit
+    there and the full bitmap is consulted in global memory before the table is read."""
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    for t in range(2):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
+        fell_back, survivors, bin_lo = eng.step_used_fallback()
+        assert not fell_back and bin_lo > 0 and cfg.ncand <= survivors < cfg.d // 4
+        declined, ones = eng.step_first_pass()
+        assert not declined and 0 < ones < cfg.r * cfg.c // 8
+
+
+def test_dense_folded_bitmap_hands_over_to_the_table_kernel(cuda_device):
+    """A folded bitmap that would rule out too few coordinates (here: all estimates zero, threshold zero, every
+    bit set) makes the filter kernel return at once; the table kernel enqueued behind it does the first pass."""
+    cfg = wl.C3.scaled(d=300_007, W=2, r=5, c=524_288, ncand=1000, k=500)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
+    fell_back, survivors, bin_lo = eng.step_used_fallback()
+    declined, ones = eng.step_first_pass()
+    assert declined and ones == cfg.r * (cfg.c // 2)
+    assert not fell_back and survivors == cfg.d and bin_lo == 0
+    assert idx.tolist() == list(range(cfg.k))
+    st = wl.Structure(cfg, cuda_device)                    # a real gradient next: the filter takes over again
+    check_step(orc, eng, wl.gradients(st, 0), cfg.rho, cfg.ncand, u_o, v_o)
+    declined, ones = eng.step_first_pass()
+    assert not declined and 0 < ones < cfg.r * cfg.c // 8
 
 
 def test_planted_heavy_coordinates_recovered(cuda_device):
