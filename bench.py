@@ -211,6 +211,7 @@ def run_ours(args, cfg):
     u, v = wl.zero_state(cfg, dev)
     eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
     eng.bind(u, v, cfg.ncand)
+    eng.set_prune_mode({"auto": S.PRUNE_AUTO, "off": S.PRUNE_OFF, "on": S.PRUNE_ON, "early_exit": S.PRUNE_EARLY_EXIT}[args.prune])
     out_idx = torch.empty(cfg.k, dtype=torch.int32, device=dev)
     out_val = torch.empty(cfg.k, dtype=torch.float32, device=dev)
 
@@ -328,6 +329,8 @@ def main():
     ap.add_argument("--workload", default="C2")
     ap.add_argument("--mode", choices=["fused", "faithful"], default="fused",
                     help="fused: ssgd_step; faithful: per-worker sketches materialised and merged (stage calls)")
+    ap.add_argument("--prune", choices=["auto", "off", "on", "early_exit"], default="auto",
+                    help="how Algorithm 3 line 9 is evaluated (profiling runs; the default is what a user gets)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--d", type=int, default=0, help="override the number of coordinates (small profiling cases)")

@@ -193,9 +193,13 @@ k_unsketch_filter(const FilterArgs F) {
     if (FOLD && __ldcg(&A.sp.state->use_table) != 0u) return;   // too dense to prune: the table kernel behind runs
     const uint32_t bin_lo = __ldcg(&A.sp.state->bin_lo);
     {
+        // asynchronous 16-byte copies, all in flight at once: the fill costs one L2 round trip, not one per piece
         const uint4* src = reinterpret_cast<const uint4*>(fold ? F.bm_fold : F.bm_full);
-        uint4* dst = reinterpret_cast<uint4*>(bm);
-        for (int w = threadIdx.x; w < nw / 4; w += FILTER_THREADS) dst[w] = __ldcg(src + w);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bm);
+        for (int w = threadIdx.x; w < nw / 4; w += FILTER_THREADS)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)w * 16u), "l"(src + w) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     __syncthreads();
 
