@@ -97,6 +97,20 @@ int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
  * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
  * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
  * which leaves tables up to that size untouched). */
+/* When ssgd_step applies Algorithm 3 line 13 (u, v <- 0 at the k chosen coordinates).
+ * DEFERRED (default): ssgd_step only marks the chosen coordinates in a d-bit map inside the workspace; the NEXT
+ * ssgd_step reads marked coordinates of u and v as +0 inside the kernel that streams all of u and v anyway, so
+ * the zero-out costs no scattered writes.  Until then the memory of u and v still holds the old values at those
+ * coordinates: call ssgd_flush before reading u or v yourself.  The library's own entry points that read u or v
+ * (ssgd_sketch_accumulate, ssgd_exact_topk, ssgd_heavymix) flush first; ssgd_exact_topk_static has no context
+ * and cannot.  Every result (chosen coordinates, values, the state after a flush) is identical in both modes.
+ * EAGER: ssgd_step writes the zeros before it returns control to the stream's next operation. */
+#define SSGD_ZERO_DEFERRED 0
+#define SSGD_ZERO_EAGER    1
+int ssgd_set_zero_mode(ssgd_ctx* ctx, int32_t mode);
+/* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Cheap when
+ * nothing is pending (one pass over d/8 bytes). */
+int ssgd_flush(ssgd_ctx* ctx, void* stream);
 int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
 /* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
  * (cudaLimitPersistingL2CacheSize of this process's CUDA context is raised to the table size, capped by the
@@ -160,7 +174,8 @@ int ssgd_exact_topk(ssgd_ctx* ctx, const int32_t* cand_idx, int64_t ncand, int32
 
 /* Algorithm 3 lines 5-13 in one call: the stages above, with the workers' values summed before the
  * insert (sum_w S(v_w) = S(sum_w v_w), Section 3), so no per-worker table is materialised.
- * out_idx/out_val: [k] device outputs, ascending coordinate order. */
+ * out_idx/out_val: [k] device outputs, ascending coordinate order.  Line 13 is applied as ssgd_set_zero_mode
+ * says: by default it is deferred into the next ssgd_step (or ssgd_flush). */
 int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t ncand,
               int32_t* out_idx, float* out_val, void* stream);
 
@@ -175,7 +190,8 @@ int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t nc
  *           |est| (compared without the last mantissa bit) are kept.
  *   line 5  out_val[t] = sum over the workers of the bound v at out_idx[t] (fp64, worker order).
  * out_idx / out_val: [k] device outputs, ascending coordinate order.  l2_out (device double) and nheavy_out
- * (device int32) are optional.  The bound state is read, not modified.  Asynchronous on `stream`. */
+ * (device int32) are optional.  The bound state is read, not modified (a deferred zero-out is applied first).
+ * Asynchronous on `stream`. */
 int ssgd_heavymix(ssgd_ctx* ctx, const float* merged, uint64_t fill_seed, int32_t* out_idx, float* out_val,
                   double* l2_out, int32_t* nheavy_out, void* stream);
 

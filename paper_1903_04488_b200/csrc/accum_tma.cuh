@@ -35,6 +35,9 @@ struct AccumArgs {
     // write the per-coordinate sum over workers to xsum[d] so that k_insert_rows can do the remaining rows
     int32_t rows_here;
     float* xsum;
+    // d-bit map of coordinates whose zero-out (Algorithm 3 line 13) is still pending from the previous step: their
+    // u and v are read as +0.  NULL: nothing is pending.
+    const uint32_t* pending;
 };
 
 #ifndef SSGD_KT_STAGES
@@ -56,6 +59,20 @@ struct KtShared {
 };
 
 #ifdef __CUDACC__
+// The four pending bits of the float4 group that starts at coordinate i0 (a multiple of 4).
+__device__ __forceinline__ uint32_t pending_bits4(const uint32_t* __restrict__ pending, int64_t i0) {
+    return pending ? (__ldg(pending + (i0 >> 5)) >> (i0 & 31)) & 0xFu : 0u;
+}
+__device__ __forceinline__ bool pending_bit(const uint32_t* __restrict__ pending, int64_t i) {
+    return pending && ((__ldg(pending + (i >> 5)) >> (i & 31)) & 1u);
+}
+// Applies the pending zero-out to one worker's u, v of that group before they are used.
+__device__ __forceinline__ void drop_pending(uint32_t bits, float4& u4, float4& v4) {
+    if (bits & 1u) { u4.x = 0.f; v4.x = 0.f; }
+    if (bits & 2u) { u4.y = 0.f; v4.y = 0.f; }
+    if (bits & 4u) { u4.z = 0.f; v4.z = 0.f; }
+    if (bits & 8u) { u4.w = 0.f; v4.w = 0.f; }
+}
 
 __device__ __forceinline__ void red_add(float* addr, float x) {
     asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(x) : "memory");
@@ -164,13 +181,15 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
             const int64_t i0 = tile * KT_TC + 4 * tid;
             const bool active = i0 < d_main;
             float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;   // sum over workers of the new v, worker order
+            const uint32_t pend = active ? pending_bits4(A.pending, i0) : 0u;
             for (int w = 0; w < A.W; ++w, ++n) {
                 const int s = n % KT_STAGES;
                 if (!mbar_wait(&S.full[s], (n / KT_STAGES) & 1, &S.abort)) { ok = false; break; }
                 if (active) {
                     const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[4 * tid]);
-                    const float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * tid]);
-                    const float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * tid]);
+                    float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * tid]);
+                    float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * tid]);
+                    if (pend) drop_pending(pend, u4, v4);
                     float4 un, vn;
                     un.x = __fmaf_rn(A.rho, u4.x, g4.x); vn.x = __fadd_rn(v4.x, un.x);
                     un.y = __fmaf_rn(A.rho, u4.y, g4.y); vn.y = __fadd_rn(v4.y, un.y);
@@ -202,9 +221,10 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
         if (ok && blockIdx.x == 0 && tid == 0) {
             for (int64_t i = d_main; i < A.d; ++i) {
                 float x = 0.f;
+                const bool pend = pending_bit(A.pending, i);
                 for (int64_t w = 0; w < A.W; ++w) {
-                    const float un = __fmaf_rn(A.rho, A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
-                    const float vn = __fadd_rn(A.v[w * A.ld + i], un);
+                    const float un = __fmaf_rn(A.rho, pend ? 0.f : A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
+                    const float vn = __fadd_rn(pend ? 0.f : A.v[w * A.ld + i], un);
                     A.u[w * A.ld + i] = un;
                     A.v[w * A.ld + i] = vn;
                     x = __fadd_rn(x, vn);

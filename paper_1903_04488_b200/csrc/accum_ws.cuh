@@ -108,13 +108,15 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
             const int64_t i0 = tile * WS_TC + 4 * st;
             const bool active = i0 < d_main;
             float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
+            const uint32_t pend = active ? pending_bits4(A.pending, i0) : 0u;
             for (int w = 0; w < A.W; ++w, ++n) {
                 const int s = n % WS_STAGES;
                 if (!mbar_wait(&S.full[s], (n / WS_STAGES) & 1, &S.abort)) { ok = false; break; }
                 if (active) {
                     const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[4 * st]);
-                    const float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * st]);
-                    const float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * st]);
+                    float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * st]);
+                    float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * st]);
+                    if (pend) drop_pending(pend, u4, v4);
                     float4 un, vn;
                     un.x = __fmaf_rn(A.rho, u4.x, g4.x); vn.x = __fadd_rn(v4.x, un.x);
                     un.y = __fmaf_rn(A.rho, u4.y, g4.y); vn.y = __fadd_rn(v4.y, un.y);
@@ -141,9 +143,10 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
         if (ok && blockIdx.x == 0 && st == 0) {
             for (int64_t i = d_main; i < A.d; ++i) {
                 float x = 0.f;
+                const bool pend = pending_bit(A.pending, i);
                 for (int64_t w = 0; w < A.W; ++w) {
-                    const float un = __fmaf_rn(A.rho, A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
-                    const float vn = __fadd_rn(A.v[w * A.ld + i], un);
+                    const float un = __fmaf_rn(A.rho, pend ? 0.f : A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
+                    const float vn = __fadd_rn(pend ? 0.f : A.v[w * A.ld + i], un);
                     A.u[w * A.ld + i] = un;
                     A.v[w * A.ld + i] = vn;
                     x = __fadd_rn(x, vn);

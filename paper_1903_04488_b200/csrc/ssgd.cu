@@ -64,6 +64,9 @@ struct ssgd_ctx {
     int32_t bm_stride_full, bm_stride_fold, bm_fold;       // bm_fold < 0: the bitmap cannot be folded into shared memory
     bool filter_ready;                                     // shared-memory attribute of the filter kernel set
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
+    size_t off_pending;     // d-bit map of the deferred zero-out; survives from step to step
+    int32_t zero_mode;      // SSGD_ZERO_DEFERRED / SSGD_ZERO_EAGER
+    bool pending_dirty;     // a deferred ssgd_step has run since the last flush: u, v may await their zero-out
     size_t off_hm;
     int32_t prune_mode;
     size_t persist_bytes;
@@ -143,6 +146,7 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->bm_stride_full = (int32_t)sf;
     x->bm_fold = s <= FILTER_MAX_FOLD ? s : -1;
     x->bm_stride_fold = s <= FILTER_MAX_FOLD ? (int32_t)round4((sf + (1 << s) - 1) >> s) : 0;
+    x->off_pending = o; o += x->map_bytes;
     x->off_bm_full = o; o += up((size_t)x->r * sf * 4);
     x->off_bm_fold = o; o += up((size_t)x->r * x->bm_stride_fold * 4);
     x->total_bytes = o;
@@ -534,23 +538,42 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     return SSGD_OK;
 }
 
+uint32_t* pending_map(ssgd_ctx* x) { return reinterpret_cast<uint32_t*>(x->ws + x->off_pending); }
+
+// Applies a deferred zero-out to u and v (no-op on an empty map).
+int flush_pending(ssgd_ctx* x, cudaStream_t st) {
+    const int64_t nwords = (x->d + 31) / 32;
+    CU(launch_pdl(st, k_flush_pending, grid_for(nwords, 256, (int64_t)x->sm_count * 16), 256, 0, pending_map(x), nwords,
+                  x->u, x->v, x->ld, x->W, x->d), "launch k_flush_pending");
+    LAUNCHED("k_flush_pending");
+    x->pending_dirty = false;
+    return SSGD_OK;
+}
+
+// Lines 10, 11, 13.  deferred: the chosen coordinates are marked in the pending map instead of being zeroed now
+// (the caller's accumulate kernel has consumed the previous marks; k_gather empties the map before the new ones).
 int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
-                       cudaStream_t st) {
+                       cudaStream_t st, bool deferred) {
     float* xs = reinterpret_cast<float*>(x->ws + x->off_xs);
     int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
     SelBuffers sb = sel_buffers(x, true);
     const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
+    uint32_t* pend = pending_map(x);                     // whatever the accumulate kernel consumed is cleared here
     CU(launch_pdl(st, k_gather, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, (const float*)x->v, x->ld, x->W,
-                  x->d, xs, sb, (uint32_t)x->k, err), "launch k_gather");
+                  x->d, xs, sb, (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather");
     LAUNCHED("k_gather");
     int e = launch_select(x, xs, ncand, sb, nch, st);
     if (e) return e;
     CU(launch_pdl(st, k_emit_final, grid_for(nch, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)xs, ncand, sb,
-                  cand, out_idx, out_val, (uint32_t)x->k, nch), "launch k_emit_final");
+                  cand, out_idx, out_val, (uint32_t)x->k, nch, deferred ? pending_map(x) : (uint32_t*)nullptr), "launch k_emit_final");
     LAUNCHED("k_emit_final");
-    CU(launch_pdl(st, k_zero, grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, (const int32_t*)out_idx,
-                  x->k, x->u, x->v, x->ld, x->W, x->d), "launch k_zero");
-    LAUNCHED("k_zero");
+    if (deferred) {
+        x->pending_dirty = true;
+    } else {
+        CU(launch_pdl(st, k_zero, grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, (const int32_t*)out_idx,
+                      x->k, x->u, x->v, x->ld, x->W, x->d), "launch k_zero");
+        LAUNCHED("k_zero");
+    }
     return SSGD_OK;
 }
 
@@ -599,7 +622,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -710,6 +733,8 @@ int ssgd_bind(ssgd_ctx* x, float* u, float* v, int64_t ld, void* workspace, size
     int e = ensure_device(x);
     if (e) return e;
     CU(cudaMemset(x->ws + x->off_err, 0, 16), "clear error flag");
+    CU(cudaMemset(x->ws + x->off_pending, 0, x->map_bytes), "clear pending map");   // nothing awaits its zero-out
+    x->pending_dirty = false;
     return SSGD_OK;
 }
 
@@ -720,11 +745,12 @@ int ssgd_sketch_accumulate(ssgd_ctx* x, const float* g, int64_t ld_g, float rho,
     if (!tables) return SSGD_EINVAL;
     if ((e = ensure_device(x))) return e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x->pending_dirty && (e = flush_pending(x, st))) return e;
     CU(cudaMemsetAsync(tables, 0, (size_t)x->W * x->r * x->c * 4, st), "memset tables");
     x->launches++;
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
-    A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
+    A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr; A.pending = nullptr;
     return launch_accum(x, A, INS_PER_WORKER, st);
 }
 
@@ -782,9 +808,10 @@ int ssgd_exact_topk(ssgd_ctx* x, const int32_t* cand_idx, int64_t ncand, int32_t
     if (ncand > x->ncand_max) return SSGD_EWORKSPACE;
     if ((e = ensure_device(x))) return e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x->pending_dirty && (e = flush_pending(x, st))) return e;
     CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_err - x->off_hist_f, st), "memset hist");
     x->launches++;
-    return gather_select_zero(x, cand_idx, ncand, out_idx, out_val, st);
+    return gather_select_zero(x, cand_idx, ncand, out_idx, out_val, st, false);
 }
 
 int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncand, int32_t* out_idx,
@@ -805,6 +832,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
+    A.pending = pending_map(x);      // the previous step's deferred zero-out, applied while u and v stream past
     // a table that cannot stay in L2 next to the stream is inserted a slice of rows at a time
     const size_t row_bytes = (size_t)x->c * 4;
     const int rows_fit = (int)(x->split_bytes / row_bytes);
@@ -825,10 +853,23 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
         if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
     }
     if ((e = mark(x, 3, st))) return e;
-    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st))) return e;
+    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED))) return e;
     if ((e = mark(x, 4, st))) return e;
     if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
     return SSGD_OK;
+}
+
+int ssgd_set_zero_mode(ssgd_ctx* x, int32_t mode) {
+    if (!x || (mode != SSGD_ZERO_DEFERRED && mode != SSGD_ZERO_EAGER)) return SSGD_EINVAL;
+    x->zero_mode = mode;
+    return SSGD_OK;
+}
+
+int ssgd_flush(ssgd_ctx* x, void* stream) {
+    int e = check_bound(x);
+    if (e) return e;
+    if ((e = ensure_device(x))) return e;
+    return flush_pending(x, static_cast<cudaStream_t>(stream));
 }
 
 int ssgd_set_timing(ssgd_ctx* x, int32_t enable) {
@@ -865,6 +906,7 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     if (!merged || !out_idx || !out_val) return SSGD_EINVAL;
     if ((e = ensure_device(x))) return e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x->pending_dirty && (e = flush_pending(x, st))) return e;   // line 5 reads v
     // histograms + state of the candidate selection, and the HEAVYMIX state
     CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->off_hist_f - x->off_hist_c, st), "memset hist");
     CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_sp_hist - x->off_hist_f, st), "memset hist");
@@ -888,8 +930,8 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     // line 5: exact values of the chosen coordinates, summed over the workers
     SelBuffers sf = sel_buffers(x, true);
     CU(launch_pdl(st, k_gather, grid_for(x->k, 256, (int64_t)1 << 30), 256, 0, (const int32_t*)out_idx, x->k, (const float*)x->v,
-                  x->ld, x->W, x->d, out_val, sf, (uint32_t)1, reinterpret_cast<int32_t*>(x->ws + x->off_err)),
-       "launch k_gather");
+                  x->ld, x->W, x->d, out_val, sf, (uint32_t)1, reinterpret_cast<int32_t*>(x->ws + x->off_err),
+                  (uint32_t*)nullptr, (int64_t)0), "launch k_gather");
     LAUNCHED("k_gather");
     if (l2_out || nheavy_out) {
         // l2 = median of the row sums: computed on the host side of the copy-out by the caller would need a
@@ -1030,12 +1072,12 @@ int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, con
     sb.chunk_eq = sb.chunk_gt + nch;
     float* xs = reinterpret_cast<float*>(base + ST_OFF_XS);
     int32_t* err = reinterpret_cast<int32_t*>(base + ST_OFF_ERR);
-    k_gather<<<grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, st>>>(cand_idx, ncand, v, ld, W, d, xs, sb, (uint32_t)k, err);
+    k_gather<<<grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, st>>>(cand_idx, ncand, v, ld, W, d, xs, sb, (uint32_t)k, err, nullptr, 0);
     const int grid = grid_for(ncand, SEL_THREADS * 8, (int64_t)sd->sm_count * 8);
     k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
     k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
     k_sel_count<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, nch);
-    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k, nch);
+    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k, nch, nullptr);
     return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ECUDA;
 }
 

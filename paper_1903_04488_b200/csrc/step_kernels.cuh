@@ -74,6 +74,7 @@ k_accum_insert(const AccumArgs A) {
         }
         float x[4] = {0.f, 0.f, 0.f, 0.f};  // sum over workers of the new v (worker order)
         if (i0 + 3 < A.d) {
+            const uint32_t pend = pending_bits4(A.pending, i0);
             constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : K1_UNROLL;
             for (int w0 = 0; w0 < A.W; w0 += U) {
                 float4 gg[U], uu[U], vv[U];
@@ -85,6 +86,10 @@ k_accum_insert(const AccumArgs A) {
                         uu[s] = __ldcs(reinterpret_cast<const float4*>(A.u + w * A.ld + i0));
                         vv[s] = __ldcs(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
                     }
+                }
+                if (pend) {                              // rare: a coordinate of this group was chosen last step
+#pragma unroll
+                    for (int s = 0; s < U; ++s) drop_pending(pend, uu[s], vv[s]);
                 }
 #pragma unroll
                 for (int s = 0; s < U; ++s) {
@@ -118,9 +123,10 @@ k_accum_insert(const AccumArgs A) {
             for (int e = 0; e < 4; ++e) {
                 const int64_t i = i0 + e;
                 if (i >= A.d) break;
+                const bool pend = pending_bit(A.pending, i);
                 for (int64_t w = 0; w < A.W; ++w) {
-                    const float un = __fmaf_rn(A.rho, A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
-                    const float vn = __fadd_rn(A.v[w * A.ld + i], un);
+                    const float un = __fmaf_rn(A.rho, pend ? 0.f : A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
+                    const float vn = __fadd_rn(pend ? 0.f : A.v[w * A.ld + i], un);
                     A.u[w * A.ld + i] = un;
                     A.v[w * A.ld + i] = vn;
                     if (MODE == INS_PER_WORKER) {
@@ -344,7 +350,8 @@ constexpr int GATHER_UNROLL = SSGD_GATHER_UNROLL;   // scattered loads in flight
 
 __global__ void __launch_bounds__(256)
 k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ v, int64_t ld, int32_t W,
-         int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag) {
+         int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag,
+         uint32_t* __restrict__ pending_clear, int64_t pending_words) {
     __shared__ SelShared sh;
     uint32_t* s_hist = sh.hist;
     pdl_trigger();
@@ -352,6 +359,9 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
     pdl_wait();
     __syncthreads();
     const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    // the accumulate kernel of this step has applied the pending zero-out: empty the map for k_emit_final
+    if (pending_clear)
+        for (int64_t t = m; t < pending_words; t += (int64_t)gridDim.x * 256) pending_clear[t] = 0u;
     if (m < ncand) {
         const int64_t i = cand[m];
         float out = 0.0f;
@@ -384,12 +394,37 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const int32_t* __restrict__ cand,
-             int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap, int64_t nchunks) {
+             int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap, int64_t nchunks,
+             uint32_t* __restrict__ pending) {
     sel_emit_chunks(xs, ncand, sb, nchunks, [&](uint32_t slot, int64_t m) {
         if (slot >= cap) return;
-        out_idx[slot] = cand[m];
+        const int32_t i = cand[m];
+        out_idx[slot] = i;
         out_val[slot] = xs[m];
+        if (pending) atomicOr(pending + (i >> 5), 1u << (i & 31));   // deferred line 13: see k_flush_pending
     });
+}
+
+// The deferred form of line 13: the chosen coordinates are marked in a d-bit map, and the next step's
+// accumulate kernel, which reads every u and v anyway, treats marked coordinates as zero.  This kernel applies
+// the map to memory for callers that read u or v in between: one thread per map word.
+__global__ void __launch_bounds__(256)
+k_flush_pending(uint32_t* __restrict__ pending, int64_t nwords, float* __restrict__ u, float* __restrict__ v,
+                int64_t ld, int32_t W, int64_t d) {
+    pdl_trigger();
+    pdl_wait();
+    const int64_t stride = (int64_t)gridDim.x * 256;
+    for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < nwords; t += stride) {
+        uint32_t bits = pending[t];
+        if (bits == 0u) continue;
+        pending[t] = 0u;
+        while (bits) {
+            const int64_t i = t * 32 + (__ffs(bits) - 1);
+            bits &= bits - 1;
+            if (i < d)
+                for (int64_t w = 0; w < W; ++w) { u[w * ld + i] = 0.0f; v[w * ld + i] = 0.0f; }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(256)

@@ -18,6 +18,7 @@ OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, 
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA, INSERT_WS = 0, 1, 2, 3, 4
 PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT = 0, 1, 2, 3
+ZERO_DEFERRED, ZERO_EAGER = 0, 1
 FMT_F16, FMT_BF16 = 0, 1
 MAX_R = 15
 
@@ -34,6 +35,8 @@ SIGNATURES = {
     "ssgd_set_prune_sample_rank": [_vp, _i64],
     "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
+    "ssgd_set_zero_mode": [_vp, _i32],
+    "ssgd_flush": [_vp, _vp],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
     "ssgd_sketch_accumulate": [_vp, _vp, _i64, _f32, _vp, _vp],
@@ -120,6 +123,7 @@ class Ssgd:
         self._h = h
         self.d, self.r, self.c, self.k, self.W, self.seed = d, r, c, k, W, seed
         self._keep = None  # tensors bound to the context stay referenced here
+        self.zero_mode = ZERO_DEFERRED
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
@@ -155,6 +159,14 @@ class Ssgd:
 
     def set_table_persistence(self, enable: bool) -> None:
         self._chk(self._lib.ssgd_set_table_persistence(self._h, 1 if enable else 0), "ssgd_set_table_persistence")
+
+    def set_zero_mode(self, mode: int) -> None:
+        self._chk(self._lib.ssgd_set_zero_mode(self._h, mode), "ssgd_set_zero_mode")
+        self.zero_mode = mode
+
+    def flush(self) -> None:
+        """Applies a deferred zero-out (Algorithm 3 line 13) to the bound u and v on the current stream."""
+        self._chk(self._lib.ssgd_flush(self._h, _stream()), "ssgd_flush")
 
     def step_used_fallback(self):
         """(redone without pruning?, survivors on the list, prune threshold bin) of the last step."""

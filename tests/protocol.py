@@ -22,6 +22,7 @@ import numpy as np
 import torch
 
 from oracle import select as oracle_select
+from paper_1903_04488_b200 import ssgd as S
 
 TABLE_RTOL = 1e-5   # relative to the L1 mass hashed into the bucket
 
@@ -65,11 +66,14 @@ def oracle_intermediates(orc, g_h, rho, u_o, v_o, ncand, by_linearity):
     return T, M, est, cand, None
 
 
-def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=None, by_linearity=False):
+def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=None, by_linearity=False,
+               flush=False):
     """Runs eng.step on g_dev and the oracle on the same g; asserts the protocol; adopts.
 
     orc: oracle.Oracle; eng: bound Ssgd; u_o, v_o: the oracle's numpy state, bit-identical to the
-    engine's bound state on entry and again on exit.  Returns (out_idx, out_val) as numpy arrays."""
+    engine's bound state on entry and again on exit (with flush=True: the state in memory after ssgd_flush;
+    otherwise, in the deferred zero mode, the state with the pending zero-out applied on the host copy).
+    Returns (out_idx, out_val) as numpy arrays."""
     d, W, k = orc.d, orc.W, orc.k
     dev = g_dev.device
     out_idx = torch.empty(k, dtype=torch.int32, device=dev)
@@ -87,7 +91,15 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
     est_g = est_t.cpu().numpy()
     assert (cand_dense.cpu().numpy() == cand_g).all(), "step and dense stage call disagree on the candidates"
     out_idx_g, out_val_g = out_idx.cpu().numpy(), out_val.cpu().numpy()
+    if flush:
+        eng.flush()
     u_g_h, v_g_h = u_g.cpu().numpy(), v_g.cpu().numpy()
+    if eng.zero_mode == S.ZERO_DEFERRED and not flush:
+        # line 13 is pending: the engine has only marked the chosen coordinates, and its next step reads them as
+        # zero.  The stale values in memory are masked here; the marks themselves are checked by the next step's
+        # comparison (a missing or extra mark changes u and v there) and by the flushed comparisons.
+        u_g_h[:, out_idx_g] = 0.0
+        v_g_h[:, out_idx_g] = 0.0
 
     # oracle, without its own zero-out
     g_h = g_dev.cpu().numpy()

@@ -170,7 +170,7 @@ def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
     report = []
     for t in range(steps):
         g = wl.gradients(st, t)
-        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report)
+        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report, flush=(t == steps - 1))
     if cfg.ncand == cfg.d:
         assert all(r["final_sym_diff_vs_unadopted"] == 0 for r in report)
 
@@ -375,7 +375,10 @@ def test_step_host_matches_step(cuda_device):
     oi = torch.empty(cfg.k, dtype=torch.int32).pin_memory()
     ov = torch.empty(cfg.k, dtype=torch.float32).pin_memory()
     eng2.step_host(g_host, cfg.rho, cfg.ncand, stage, oi, ov)
-    assert (u2 == u).all() and (v2 == v).all()
+    assert (u2 == u).all() and (v2 == v).all()            # the accumulation (zero-out still pending in both)
+    if (out_idx.cpu() == oi).all():
+        eng.flush(); eng2.flush()
+        assert (u2 == u).all() and (v2 == v).all() and int((v[0, :cfg.d] == 0).sum().item()) >= cfg.k
     # same table up to reduction order -> the selections agree except near ties; values of common ones match
     a, b = out_idx.cpu().numpy(), oi.numpy()
     common, ia, ib = np.intersect1d(a, b, return_indices=True)
@@ -394,7 +397,7 @@ def run_full(cfg, dev, steps, by_linearity):
     g = None
     for t in range(steps):
         g = wl.gradients(st, t, out=g)
-        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report,
+        check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, report=report, flush=(t == steps - 1),
                    by_linearity=by_linearity[t] if isinstance(by_linearity, (list, tuple)) else by_linearity)
     return report
 
@@ -463,6 +466,7 @@ def test_stored_small_case_is_reproduced_exactly(cuda_device):
             assert cand.cpu().tolist() == step["cand"]
             assert oi.cpu().tolist() == step["out_idx"]
             assert ov.cpu().tolist() == step["out_val"]
+        eng.flush()
         state = u.cpu().numpy()[:, :sh["d"]].tobytes() + v.cpu().numpy()[:, :sh["d"]].tobytes()
         assert hashlib.sha256(state).hexdigest() == want["state_sha256"]
 
@@ -498,7 +502,74 @@ def test_step_can_be_captured_in_a_cuda_graph(cuda_device):
         common, ia, ib = np.intersect1d(a, b, return_indices=True)
         assert common.size >= 0.995 * cfg.k
         assert (eager_val.cpu().numpy()[ia] == ov.cpu().numpy()[ib]).all()
+        eng.flush()                                       # the replayed step only marked its k coordinates
         assert int((v[0, :cfg.d] == 0).sum().item()) >= cfg.k
+
+
+# ------------------------------------------------------------------------------------------------
+# Algorithm 3 line 13, deferred into the next step's streaming kernel
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("mode", [S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_SMEM])
+def test_deferred_zero_equals_eager_zero(cuda_device, mode):
+    """Two engines on the same inputs, one zeroing at once and one deferring: identical outputs every step, the
+    deferring one's memory still holds the old values at the chosen coordinates until its next step or a flush,
+    and after a flush the two states are identical bit for bit.  d is not a multiple of 4 (ragged tail), the
+    flushes fall on different steps, and a step after a flush must not zero anything twice."""
+    cfg = wl.C2.scaled(d=90_003, W=5, c=2048, ncand=3000, k=2000)
+    dev = cuda_device
+    st = wl.Structure(cfg, dev)
+    eng_e, _, u_e, v_e = make(cfg, dev)
+    eng_d, _, u_d, v_d = make(cfg, dev)
+    for eng in (eng_e, eng_d):
+        eng.set_insert_mode(mode)
+    eng_e.set_zero_mode(S.ZERO_EAGER)
+    oi_e = torch.empty(cfg.k, dtype=torch.int32, device=dev); ov_e = torch.empty(cfg.k, device=dev)
+    oi_d = torch.empty_like(oi_e); ov_d = torch.empty_like(ov_e)
+    for t in range(6):
+        g = wl.gradients(st, t)
+        g[:, cfg.d - 1] = 100.0 * (t + 1)                  # the last coordinate (ragged tail) is chosen every step
+        eng_e.step(g, cfg.rho, cfg.ncand, oi_e, ov_e)
+        eng_d.step(g, cfg.rho, cfg.ncand, oi_d, ov_d)
+        assert eng_e.status() == S.OK and eng_d.status() == S.OK
+        if not (oi_e == oi_d).all():
+            pytest.skip("the two tables differ in reduction order and a near-tie fell differently")
+        assert (ov_e == ov_d).all() and int(oi_d[-1].item()) == cfg.d - 1
+        chosen = oi_d.long()
+        assert (u_e[:, chosen] == 0).all() and (v_e[:, chosen] == 0).all()
+        assert (v_d[:, chosen] != 0).any()                  # still the accumulated values in memory
+        keep = torch.ones(cfg.ld, dtype=torch.bool, device=dev)
+        keep[chosen] = False
+        assert (u_d[:, keep] == u_e[:, keep]).all() and (v_d[:, keep] == v_e[:, keep]).all()
+        if t in (1, 2, 5):
+            eng_d.flush()
+            assert (u_d == u_e).all() and (v_d == v_e).all()
+    eng_d.flush()                                           # nothing pending: must change nothing
+    assert (u_d == u_e).all() and (v_d == v_e).all()
+
+
+def test_stage_calls_apply_a_pending_zero_out_first(cuda_device):
+    """ssgd_exact_topk and ssgd_sketch_accumulate read the bound state: after a deferred step they must see it
+    zeroed at the chosen coordinates."""
+    cfg = wl.C2.scaled(d=60_001, W=3, c=1024, ncand=1500, k=700)
+    dev = cuda_device
+    st = wl.Structure(cfg, dev)
+    eng, _, u, v = make(cfg, dev)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=dev); ov = torch.empty(cfg.k, device=dev)
+    eng.step(wl.gradients(st, 0), cfg.rho, cfg.ncand, oi, ov)
+    chosen = oi.clone()
+    assert (v[:, chosen.long()] != 0).any()
+    o2 = torch.empty_like(oi); v2 = torch.empty_like(ov)
+    cand = torch.arange(cfg.ncand, dtype=torch.int32, device=dev)
+    eng.exact_topk(cand, o2, v2)
+    assert eng.status() == S.OK
+    assert (v[:, chosen.long()] == 0).all() and (u[:, chosen.long()] == 0).all()
+    # and the other reader
+    eng.step(wl.gradients(st, 1), cfg.rho, cfg.ncand, oi, ov)
+    chosen = oi.clone()
+    tables = torch.empty((cfg.W, cfg.r, cfg.c), device=dev)
+    before_u = u.clone()
+    eng.sketch_accumulate(torch.zeros_like(u), 0.0, tables)   # rho = 0, g = 0: u <- 0, v <- v
+    assert (u == 0).all() and (v[:, chosen.long()] == 0).all() and (before_u[:, chosen.long()] != 0).any()
 
 
 # ------------------------------------------------------------------------------------------------
