@@ -74,7 +74,6 @@ k_accum_insert(const AccumArgs A) {
         }
         float x[4] = {0.f, 0.f, 0.f, 0.f};  // sum over workers of the new v (worker order)
         if (i0 + 3 < A.d) {
-            const uint32_t pend = pending_bits4(A.pending, i0);
             constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : K1_UNROLL;
             for (int w0 = 0; w0 < A.W; w0 += U) {
                 float4 gg[U], uu[U], vv[U];
@@ -87,6 +86,7 @@ k_accum_insert(const AccumArgs A) {
                         vv[s] = __ldcs(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
                     }
                 }
+                const uint32_t pend = pending_bits4(A.pending, i0);   // after the wide loads are on their way
                 if (pend) {                              // rare: a coordinate of this group was chosen last step
 #pragma unroll
                     for (int s = 0; s < U; ++s) drop_pending(pend, uu[s], vv[s]);
