@@ -45,6 +45,10 @@ enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2
 #endif
 // Measured on B200 (C2, W = 16): 256 threads x 4 workers in flight 4.93 TB/s; 128 x 8 5.38; 128 x 16 5.58;
 // 64 x 16 5.56; forcing more resident blocks (fewer registers) or 32 workers in flight is slower.
+// The grid has one float4 group per thread on purpose: capping it at 2, 4, 8, 16, 40 blocks per SM (each
+// thread then loops over 74 ... 4 groups) took 0.887, 0.860, 0.814, 0.724, 0.654 ms against 0.635 ms, and
+// deferring a group's reductions until the next group's loads are issued recovered only part of that (0.805 ms
+// at 2 blocks per SM).
 #ifndef SSGD_K1_THREADS
 #define SSGD_K1_THREADS 128
 #endif

@@ -94,12 +94,7 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
     if flush:
         eng.flush()
     u_g_h, v_g_h = u_g.cpu().numpy(), v_g.cpu().numpy()
-    if eng.zero_mode == S.ZERO_DEFERRED and not flush:
-        # line 13 is pending: the engine has only marked the chosen coordinates, and its next step reads them as
-        # zero.  The stale values in memory are masked here; the marks themselves are checked by the next step's
-        # comparison (a missing or extra mark changes u and v there) and by the flushed comparisons.
-        u_g_h[:, out_idx_g] = 0.0
-        v_g_h[:, out_idx_g] = 0.0
+    pending = eng.zero_mode == S.ZERO_DEFERRED and not flush
 
     # oracle, without its own zero-out
     g_h = g_dev.cpu().numpy()
@@ -146,10 +141,17 @@ def check_step(orc, eng, g_dev, rho, ncand, u_o, v_o, *, check_est=True, report=
         report[-1]["final_sym_diff_vs_unadopted"] = int(np.setxor1d(out_idx_g, out_idx_o).size)
 
     # 5 + 6: adopt the GPU's selection (the oracle zeroes u, v there, every worker); then the whole state
-    # must agree bit for bit: +0.0f at the chosen coordinates, the oracle's accumulation everywhere else
-    orc.zero(u_o, v_o, out_idx_g)
+    # must agree bit for bit: +0.0f at the chosen coordinates, the oracle's accumulation everywhere else.
+    # In the deferred zero mode without a flush, line 13 is still pending on the GPU side: its memory must then
+    # equal the oracle's state BEFORE the zero-out, bit for bit and everywhere (nothing but the accumulation has
+    # touched it); that the engine has marked exactly the chosen coordinates shows in the next step's comparison
+    # (a missing or extra mark changes u and v there) and in the flushed comparisons.
+    if not pending:
+        orc.zero(u_o, v_o, out_idx_g)
     for name, got, want in (("u", u_g_h, u_o), ("v", v_g_h, v_o)):
         for w in range(W):
             assert (got[w].view(np.uint32) == want[w].view(np.uint32)).all(), \
                 f"{name}[{w}]: state differs from the oracle's (accumulation or zero-out mask)"
+    if pending:
+        orc.zero(u_o, v_o, out_idx_g)
     return out_idx_g, out_val_g
