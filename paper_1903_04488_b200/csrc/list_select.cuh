@@ -1,14 +1,14 @@
 // list_select.cuh -- exact top-ncand of the survivor list written by k_unsketch_pruned (Algorithm 3 line 9),
 // emitted in ascending coordinate order.
 //
-// The list is short (1-2 x ncand entries out of d coordinates) and unordered.  Four grid-wide launches:
+// The list is short (1-2 x ncand entries out of d coordinates) and unordered.  Three grid-wide launches:
 //
 //   k_list_hist     one pass over the list: for the items inside the first threshold digit (12 bits, found by
 //                   the producer's last block) count the next 11 key bits in H2 and the low 19 key bits in a
 //                   2^19-bin table; the last block finds the second digit in H2 and the third among the 256
 //                   bins of the big table under it: the exact threshold key T and the tie quota Q.
-//   k_list_mark     items above T set their coordinate's bit in map A, items equal to T in map B.
-//   k_map_count     marks per chunk of map words; the last block turns them into exclusive offsets.
+//   k_list_mark     items above T set their coordinate's bit in map A, items equal to T in map B, and count
+//                   themselves on their chunk of map words; the last block turns the counts into exclusive offsets.
 //   k_map_emit      walks the maps in coordinate order: an A bit with a A-bits and b B-bits before it goes to
 //                   slot a + min(b, Q); a B bit with b < Q to slot a + b.  Ties at the threshold therefore go
 //                   to the smallest coordinates, without a sort and without a limit on their number.
@@ -22,8 +22,6 @@
 
 namespace ssgd {
 
-constexpr int H19_BITS = H2_BITS + H3_BITS;            // 19
-constexpr int H19_BINS = 1 << H19_BITS;
 constexpr int MAP_CHUNK_WORDS = SEL_THREADS * 8;       // map words per block in count/emit (8 per thread)
 
 #ifdef __CUDACC__
@@ -63,13 +61,21 @@ k_list_hist(SparseBuffers sp) {
     }
 }
 
-// ---- mark: coordinates above the threshold in map A, at the threshold in map B ---------------------------
+// ---- mark: coordinates above the threshold in map A, at the threshold in map B; marks per chunk of map words ---
+// Every list item is a distinct coordinate, so the marks a chunk of the maps receives can be counted here, one
+// atomic per marked item on the chunk's counter (zeroed with the maps); the last block turns the counts into
+// exclusive offsets for k_map_emit.
 __global__ void __launch_bounds__(SEL_THREADS)
-k_list_mark(SparseBuffers sp) {
+k_list_mark(SparseBuffers sp, int64_t nchunks) {
+    __shared__ SelShared sh;
+    // chunk counters are hot addresses (a few hundred of them for 1e5 marks): count in shared memory first
+    const bool local = 2 * nchunks <= H1_BINS;
     pdl_trigger();
+    if (local) for (int b = threadIdx.x; b < 2 * nchunks; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
     const uint32_t n = __ldcg(&sp.state->n_surv);
     const uint32_t T = __ldcg(&sp.state->thr_key);
+    __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
     for (int64_t i0 = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i0 < n; i0 += stride * SEL_BATCH) {
         uint32_t keys[SEL_BATCH];
@@ -78,8 +84,25 @@ k_list_mark(SparseBuffers sp) {
         for (int u = 0; u < SEL_BATCH; ++u) {
             if (keys[u] == NO_ITEM || keys[u] < T) continue;
             const uint32_t c = (uint32_t)sp.list_idx[i0 + u * stride];
-            atomicOr((keys[u] > T ? sp.map_a : sp.map_b) + (c >> 5), 1u << (c & 31));
+            const bool above = keys[u] > T;
+            atomicOr((above ? sp.map_a : sp.map_b) + (c >> 5), 1u << (c & 31));
+            const uint32_t chunk = (c >> 5) / MAP_CHUNK_WORDS;
+            if (local) atomicAdd(&sh.hist[(above ? 0 : nchunks) + chunk], 1u);
+            else atomicAdd((above ? sp.chunk_a : sp.chunk_b) + chunk, 1u);
         }
+    }
+    if (local) {
+        __syncthreads();
+        for (int b = threadIdx.x; b < 2 * nchunks; b += SEL_THREADS) {
+            const uint32_t h = sh.hist[b];
+            if (h) atomicAdd(b < nchunks ? sp.chunk_a + b : sp.chunk_b + (b - nchunks), h);
+        }
+    }
+    if (block_is_last(&sp.state->ticket[4], sh)) {
+        SelBuffers sb{};
+        sb.chunk_gt = sp.chunk_a;
+        sb.chunk_eq = sp.chunk_b;
+        block_scan_chunks(sb, nchunks, sh);
     }
 }
 
@@ -91,41 +114,6 @@ __device__ __forceinline__ void load_map_words(const SparseBuffers& sp, int64_t 
         const int64_t w = chunk_base + it * SEL_THREADS + threadIdx.x;
         wa[it] = w < nwords ? __ldcg(sp.map_a + w) : 0u;
         wb[it] = w < nwords ? __ldcg(sp.map_b + w) : 0u;
-    }
-}
-
-// ---- count: marks per chunk of map words; the last block scans ---------------------------------------------
-__global__ void __launch_bounds__(SEL_THREADS)
-k_map_count(SparseBuffers sp, int64_t nwords, int64_t nchunks) {
-    __shared__ SelShared sh;
-    pdl_trigger();
-    pdl_wait();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-        uint32_t wa[8], wb[8];
-        load_map_words(sp, nwords, chunk * MAP_CHUNK_WORDS, wa, wb);
-        uint32_t ca = 0, cb = 0;
-#pragma unroll
-        for (int it = 0; it < 8; ++it) { ca += __popc(wa[it]); cb += __popc(wb[it]); }
-        for (int off = 16; off; off >>= 1) {
-            ca += __shfl_xor_sync(0xFFFFFFFFu, ca, off);
-            cb += __shfl_xor_sync(0xFFFFFFFFu, cb, off);
-        }
-        if (lane == 0) { sh.hist[warp] = ca; sh.hist[SEL_WARPS + warp] = cb; }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t a = 0, b = 0;
-            for (int w = 0; w < SEL_WARPS; ++w) { a += sh.hist[w]; b += sh.hist[SEL_WARPS + w]; }
-            sp.chunk_a[chunk] = a;
-            sp.chunk_b[chunk] = b;
-        }
-        __syncthreads();
-    }
-    if (block_is_last(&sp.state->ticket[4], sh)) {
-        SelBuffers sb{};
-        sb.chunk_gt = sp.chunk_a;
-        sb.chunk_eq = sp.chunk_b;
-        block_scan_chunks(sb, nchunks, sh);
     }
 }
 

@@ -31,6 +31,10 @@ constexpr int H1_BINS = 1 << H1_BITS, H2_BINS = 1 << H2_BITS, H3_BINS = 1 << H3_
 constexpr int H1_SHIFT = 31 - H1_BITS;                 // 19
 constexpr int H2_SHIFT = H1_SHIFT - H2_BITS;           // 8
 constexpr int SEL_HIST_WORDS = H1_BINS + H2_BINS + H3_BINS;
+constexpr int H19_BITS = H2_BITS + H3_BITS;            // 19: the key bits below the first digit
+constexpr int H19_BINS = 1 << H19_BITS;
+constexpr int SEL_ITEMS_SMALL = 4;                     // items per thread in count/emit of short inputs (more blocks)
+constexpr int SEL_CHUNK_SMALL = SEL_THREADS * SEL_ITEMS_SMALL;
 
 // Per-selection state, zeroed before the producer runs.
 struct SelState {
@@ -49,6 +53,7 @@ struct SelBuffers {
     SelState* state;
     uint32_t* chunk_gt;  // [nchunks] counts, then exclusive offsets
     uint32_t* chunk_eq;  // [nchunks]
+    uint32_t* h19;       // [H19_BINS] zeroed, or NULL: with it, k_sel_pass23 replaces k_sel_pass2 + k_sel_pass3
 };
 
 #ifdef __CUDACC__
@@ -195,6 +200,44 @@ k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     }
 }
 
+// ---- passes 2 and 3 in one: H2 in shared memory and, in the same pass, the low 19 key bits of the items inside
+// the first digit in a 2^19-bin table in global memory (few items: the first digit has already cut the input
+// down to one bin in 4096).  The last block finds the second digit in H2 and the third among the 256 bins of the
+// big table under it: the exact threshold key T and the tie quota Q.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_sel_pass23(const float* __restrict__ val, int64_t n, SelBuffers sb) {
+    __shared__ SelShared sh;
+    pdl_trigger();
+    for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    pdl_wait();
+    const uint32_t d1 = sb.state->d1;
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
+    for (int64_t i0 = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i0 < n; i0 += stride * SEL_BATCH) {
+        uint32_t keys[SEL_BATCH];
+        load_keys(val, n, i0, stride, keys);
+#pragma unroll
+        for (int u = 0; u < SEL_BATCH; ++u) {
+            if (keys[u] != NO_ITEM && (keys[u] >> H1_SHIFT) == d1) {
+                atomicAdd(&sh.hist[(keys[u] >> H2_SHIFT) & (H2_BINS - 1)], 1u);
+                atomicAdd(&sb.h19[keys[u] & (H19_BINS - 1)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    flush_hist<H2_BINS>(sh.hist, sb.h2);
+    if (block_is_last(&sb.state->ticket[1], sh)) {
+        uint32_t d2, rem2, d3, rem3;
+        block_find_from_top<H2_BINS>(sb.h2, sb.state->rem1, sh, d2, rem2);
+        block_find_from_top<H3_BINS>(sb.h19 + ((size_t)d2 << H3_BITS), rem2, sh, d3, rem3);
+        if (threadIdx.x == 0) {
+            sb.state->d2 = d2; sb.state->rem2 = rem2;
+            sb.state->thr_key = (d1 << H1_SHIFT) | (d2 << H2_SHIFT) | d3;
+            sb.state->quota_eq = rem3;
+        }
+    }
+}
+
 // For producer kernels (SEL_THREADS threads, histogram H1 already flushed): the last block turns H1
 // into the first threshold digit.  `want` = how many items the selection keeps.
 __device__ __forceinline__ void producer_epilogue(const SelBuffers& sb, uint32_t want, SelShared& sh) {
@@ -205,21 +248,23 @@ __device__ __forceinline__ void producer_epilogue(const SelBuffers& sb, uint32_t
     }
 }
 
-// Warp w of a block owns items [chunk*SEL_CHUNK + w*512, +512), read 32 at a time (coalesced).
+// A chunk is SEL_THREADS * ITEMS items (one block's share); warp w of the block owns items
+// [chunk_base + w*32*ITEMS, +32*ITEMS), read 32 at a time (coalesced).
 // Returns, as ballots per iteration, which lanes hold key > T (bg) and key == T (be).
+template <int ITEMS>
 __device__ __forceinline__ void chunk_ballots(const float* __restrict__ val, int64_t n, int64_t warp_base,
-                                              uint32_t T, uint32_t (&bg)[SEL_ITEMS], uint32_t (&be)[SEL_ITEMS],
+                                              uint32_t T, uint32_t (&bg)[ITEMS], uint32_t (&be)[ITEMS],
                                               uint32_t& ngt, uint32_t& neq) {
     const int lane = threadIdx.x & 31;
     ngt = 0; neq = 0;
-    uint32_t keys[SEL_ITEMS];                               // all of the lane's items are loaded before any is used
+    uint32_t keys[ITEMS];                                   // all of the lane's items are loaded before any is used
 #pragma unroll
-    for (int it = 0; it < SEL_ITEMS; ++it) {
+    for (int it = 0; it < ITEMS; ++it) {
         const int64_t i = warp_base + it * 32 + lane;
         keys[it] = i < n ? key_of(val[i]) : NO_ITEM;
     }
 #pragma unroll
-    for (int it = 0; it < SEL_ITEMS; ++it) {
+    for (int it = 0; it < ITEMS; ++it) {
         const bool ok = keys[it] != NO_ITEM;
         bg[it] = __ballot_sync(0xFFFFFFFFu, ok && keys[it] > T);
         be[it] = __ballot_sync(0xFFFFFFFFu, ok && keys[it] == T);
@@ -268,6 +313,7 @@ __device__ __forceinline__ void block_scan_chunks(const SelBuffers& sb, int64_t 
     }
 }
 
+template <int ITEMS>
 __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nchunks) {
     __shared__ SelShared sh;
@@ -276,8 +322,8 @@ k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nch
     const uint32_t T = sb.state->thr_key;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-        uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
-        chunk_ballots(val, n, chunk * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS), T, bg, be, ngt, neq);
+        uint32_t bg[ITEMS], be[ITEMS], ngt, neq;
+        chunk_ballots<ITEMS>(val, n, (chunk * SEL_THREADS + warp * 32) * ITEMS, T, bg, be, ngt, neq);
         if (lane == 0) { sh.hist[warp] = ngt; sh.hist[SEL_WARPS + warp] = neq; }
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -293,7 +339,7 @@ k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nch
 
 // ---- emit: ordered compaction of the selected items -----------------------------------------------
 // `sink(slot, i)` is called once for every selected item i with its output slot (0 .. m-1).
-template <typename Sink>
+template <int ITEMS, typename Sink>
 __device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, int64_t n, const SelBuffers& sb,
                                                 int64_t nchunks, Sink sink) {
     __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
@@ -302,9 +348,9 @@ __device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, i
     const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
-    const int64_t warp_base = chunk * SEL_CHUNK + warp * (SEL_CHUNK / SEL_WARPS);
-    uint32_t bg[SEL_ITEMS], be[SEL_ITEMS], ngt, neq;
-    chunk_ballots(val, n, warp_base, T, bg, be, ngt, neq);
+    const int64_t warp_base = (chunk * SEL_THREADS + warp * 32) * ITEMS;
+    uint32_t bg[ITEMS], be[ITEMS], ngt, neq;
+    chunk_ballots<ITEMS>(val, n, warp_base, T, bg, be, ngt, neq);
     __syncthreads();                       // the previous chunk's readers are done with s_wg, s_we
     if (lane == 0) { s_wg[warp] = ngt; s_we[warp] = neq; }
     __syncthreads();
@@ -312,7 +358,7 @@ __device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, i
     for (int w = 0; w < warp; ++w) { gt_before += s_wg[w]; eq_before += s_we[w]; }
     const uint32_t lt_mask = (1u << lane) - 1u;
 #pragma unroll
-    for (int it = 0; it < SEL_ITEMS; ++it) {
+    for (int it = 0; it < ITEMS; ++it) {
         const uint32_t g = gt_before + __popc(bg[it] & lt_mask);
         const uint32_t e = eq_before + __popc(be[it] & lt_mask);
         const bool is_gt = (bg[it] >> lane) & 1u, is_eq = (be[it] >> lane) & 1u;

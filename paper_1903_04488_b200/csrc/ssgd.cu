@@ -113,27 +113,27 @@ void derive_params(uint64_t seed, int32_t r, HashParams& hp) {
 void layout(ssgd_ctx* x, int64_t ncand_max) {
     size_t o = 0;
     x->off_table = o;   o += up((size_t)x->r * x->c * 4);
-    x->off_hist_c = o;  o += up(SEL_HIST_WORDS * 4);
+    x->off_hist_c = o;  o += up((size_t)(SEL_HIST_WORDS + H19_BINS) * 4);
     x->off_state_c = o; o += up(sizeof(SelState));
-    x->off_hist_f = o;  o += up(SEL_HIST_WORDS * 4);
+    x->off_hist_f = o;  o += up((size_t)(SEL_HIST_WORDS + H19_BINS) * 4);
     x->off_state_f = o; o += up(sizeof(SelState));
-    x->off_sp_hist = o; o += up((size_t)(2 * H1_BINS + H2_BINS + H19_BINS) * 4);
+    x->off_sp_hist = o; o += up((size_t)(2 * H1_BINS + H2_BINS) * 4);   // its 2^19-bin table is the candidate selection's
     x->off_sp_state = o; o += up(sizeof(SparseState));
     x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
     x->off_maps = o;    o += 2 * x->map_bytes;
+    x->nchunk_map = ((x->d + 31) / 32 + MAP_CHUNK_WORDS - 1) / MAP_CHUNK_WORDS;
+    x->off_map_chunks = o; o += up((size_t)x->nchunk_map * 8);   // marks per chunk of map words: counted from zero
     x->off_hm = o;      o += up(sizeof(HeavymixState));
     x->off_err = o;     o += up(16);
     x->zero_bytes = o;
     x->nchunk_c = (x->d + SEL_CHUNK - 1) / SEL_CHUNK;
-    x->nchunk_f = (ncand_max + SEL_CHUNK - 1) / SEL_CHUNK;
+    x->nchunk_f = (ncand_max + SEL_CHUNK_SMALL - 1) / SEL_CHUNK_SMALL;
     x->off_est = o;     o += up((size_t)x->d * 4);
     x->off_chunk_c = o; o += up((size_t)x->nchunk_c * 8);
     x->off_chunk_f = o; o += up((size_t)x->nchunk_f * 8);
     x->off_cand = o;    o += up((size_t)ncand_max * 4);
     x->off_xs = o;      o += up((size_t)ncand_max * 4);
     x->list_cap = x->d;                                  // the unpruned rerun may list every coordinate
-    x->nchunk_map = ((x->d + 31) / 32 + MAP_CHUNK_WORDS - 1) / MAP_CHUNK_WORDS;
-    x->off_map_chunks = o; o += up((size_t)x->nchunk_map * 8);
     x->off_list_idx = o; o += up((size_t)x->list_cap * 4);
     x->off_list_est = o; o += up((size_t)x->list_cap * 4);
     x->off_oidx = o;    o += up((size_t)x->k * 4);
@@ -155,7 +155,7 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
 SelBuffers sel_buffers(ssgd_ctx* x, bool final_stage) {
     SelBuffers sb{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_hist_f : x->off_hist_c));
-    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
+    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS; sb.h19 = h + SEL_HIST_WORDS;
     sb.state = reinterpret_cast<SelState*>(x->ws + (final_stage ? x->off_state_f : x->off_state_c));
     uint32_t* ch = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_chunk_f : x->off_chunk_c));
     const int64_t nch = final_stage ? x->nchunk_f : x->nchunk_c;
@@ -370,14 +370,23 @@ int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
 // Radix-select passes after the producer filled H1: leaves thresholds in sb.state and exclusive
 // chunk offsets in sb.chunk_*; the caller launches the emit kernel over `nchunks` blocks.
 int launch_select(ssgd_ctx* x, const float* val, int64_t n, const SelBuffers& sb, int64_t nchunks,
-                  cudaStream_t st) {
+                  cudaStream_t st, bool small_chunks) {
     const int grid = grid_for(n, SEL_THREADS * 8, (int64_t)x->sm_count * 8);
-    CU(launch_pdl(st, k_sel_pass2, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass2");
-    LAUNCHED("k_sel_pass2");
-    CU(launch_pdl(st, k_sel_pass3, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass3");
-    LAUNCHED("k_sel_pass3");
-    CU(launch_pdl(st, k_sel_count, grid_for(nchunks, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, val, n, sb, nchunks),
-       "launch k_sel_count");
+    if (sb.h19) {
+        CU(launch_pdl(st, k_sel_pass23, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass23");
+        LAUNCHED("k_sel_pass23");
+    } else {
+        CU(launch_pdl(st, k_sel_pass2, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass2");
+        LAUNCHED("k_sel_pass2");
+        CU(launch_pdl(st, k_sel_pass3, grid, SEL_THREADS, 0, val, n, sb), "launch k_sel_pass3");
+        LAUNCHED("k_sel_pass3");
+    }
+    if (small_chunks)
+        CU(launch_pdl(st, k_sel_count<SEL_ITEMS_SMALL>, grid_for(nchunks, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, val, n, sb,
+                      nchunks), "launch k_sel_count");
+    else
+        CU(launch_pdl(st, k_sel_count<SEL_ITEMS>, grid_for(nchunks, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, val, n, sb,
+                      nchunks), "launch k_sel_count");
     LAUNCHED("k_sel_count");
     return SSGD_OK;
 }
@@ -410,7 +419,7 @@ int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* ca
     int e = launch_unsketch(x, A, st);
     if (e) return e;
     if (timed && (e = mark(x, 2, st))) return e;
-    if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st))) return e;
+    if ((e = launch_select(x, est, x->d, sb, x->nchunk_c, st, false))) return e;
     CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)est,
                   x->d, sb, cand_idx, cand_est, (uint32_t)ncand, x->nchunk_c), "launch k_emit_candidates");
     LAUNCHED("k_emit_candidates");
@@ -420,7 +429,8 @@ int unsketch_select(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* ca
 SparseBuffers sparse_buffers(ssgd_ctx* x) {
     SparseBuffers sp{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + x->off_sp_hist);
-    sp.h1_sample = h; sp.h1 = h + H1_BINS; sp.h2 = h + 2 * H1_BINS; sp.h19 = h + 2 * H1_BINS + H2_BINS;
+    sp.h1_sample = h; sp.h1 = h + H1_BINS; sp.h2 = h + 2 * H1_BINS;
+    sp.h19 = reinterpret_cast<uint32_t*>(x->ws + x->off_hist_c) + SEL_HIST_WORDS;   // never used by both in one step
     sp.state = reinterpret_cast<SparseState*>(x->ws + x->off_sp_state);
     sp.list_idx = reinterpret_cast<int32_t*>(x->ws + x->off_list_idx);
     sp.list_est = reinterpret_cast<float*>(x->ws + x->off_list_est);
@@ -526,12 +536,10 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     const int list_grid = grid_for(4 * ncand, SEL_THREADS * SEL_BATCH, (int64_t)x->sm_count * 8);
     CU(launch_pdl(st, k_list_hist, list_grid, SEL_THREADS, 0, A.sp), "launch k_list_hist");
     LAUNCHED("k_list_hist");
-    CU(launch_pdl(st, k_list_mark, list_grid, SEL_THREADS, 0, A.sp), "launch k_list_mark");
+    CU(launch_pdl(st, k_list_mark, list_grid, SEL_THREADS, 0, A.sp, x->nchunk_map), "launch k_list_mark");
     LAUNCHED("k_list_mark");
     const int64_t nwords = (x->d + 31) / 32;
     const int map_grid = grid_for(x->nchunk_map, 1, (int64_t)x->sm_count * 8);
-    CU(launch_pdl(st, k_map_count, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map), "launch k_map_count");
-    LAUNCHED("k_map_count");
     CU(launch_pdl(st, k_map_emit, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map, (uint32_t)ncand, cand_idx),
        "launch k_map_emit");
     LAUNCHED("k_map_emit");
@@ -557,14 +565,14 @@ int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t*
     float* xs = reinterpret_cast<float*>(x->ws + x->off_xs);
     int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
     SelBuffers sb = sel_buffers(x, true);
-    const int64_t nch = (ncand + SEL_CHUNK - 1) / SEL_CHUNK;
+    const int64_t nch = (ncand + SEL_CHUNK_SMALL - 1) / SEL_CHUNK_SMALL;
     uint32_t* pend = pending_map(x);                     // whatever the accumulate kernel consumed is cleared here
     CU(launch_pdl(st, k_gather, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, (const float*)x->v, x->ld, x->W,
                   x->d, xs, sb, (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather");
     LAUNCHED("k_gather");
-    int e = launch_select(x, xs, ncand, sb, nch, st);
+    int e = launch_select(x, xs, ncand, sb, nch, st, true);
     if (e) return e;
-    CU(launch_pdl(st, k_emit_final, grid_for(nch, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)xs, ncand, sb,
+    CU(launch_pdl(st, k_emit_final<SEL_ITEMS_SMALL>, grid_for(nch, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)xs, ncand, sb,
                   cand, out_idx, out_val, (uint32_t)x->k, nch, deferred ? pending_map(x) : (uint32_t*)nullptr), "launch k_emit_final");
     LAUNCHED("k_emit_final");
     if (deferred) {
@@ -923,7 +931,7 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     k_row_sumsq<<<grid, 256, 0, st>>>(merged, x->c, A.hm);
     LAUNCHED("k_row_sumsq");
     if ((e = launch_heavymix_keys(x, A, st))) return e;
-    if ((e = launch_select(x, A.keys, x->d, A.sb, x->nchunk_c, st))) return e;
+    if ((e = launch_select(x, A.keys, x->d, A.sb, x->nchunk_c, st, false))) return e;
     CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)A.keys,
                   x->d, A.sb, out_idx, (float*)nullptr, (uint32_t)x->k, x->nchunk_c), "launch k_emit_candidates");
     LAUNCHED("k_emit_candidates");
@@ -1076,8 +1084,8 @@ int ssgd_exact_topk_static(const float* v, int64_t ld, int32_t W, int64_t d, con
     const int grid = grid_for(ncand, SEL_THREADS * 8, (int64_t)sd->sm_count * 8);
     k_sel_pass2<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
     k_sel_pass3<<<grid, SEL_THREADS, 0, st>>>(xs, ncand, sb);
-    k_sel_count<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, nch);
-    k_emit_final<<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k, nch, nullptr);
+    k_sel_count<SEL_ITEMS><<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, nch);
+    k_emit_final<SEL_ITEMS><<<(int)nch, SEL_THREADS, 0, st>>>(xs, ncand, sb, cand_idx, out_idx, out_val, (uint32_t)k, nch, nullptr);
     return cudaGetLastError() == cudaSuccess ? SSGD_OK : SSGD_ECUDA;
 }
 

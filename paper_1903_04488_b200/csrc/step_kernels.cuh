@@ -337,7 +337,7 @@ k_unsketch(const UnsketchArgs A) {
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32_t* __restrict__ cand_idx,
                   float* __restrict__ cand_est, uint32_t cap, int64_t nchunks) {
-    sel_emit_chunks(est, d, sb, nchunks, [&](uint32_t slot, int64_t i) {
+    sel_emit_chunks<SEL_ITEMS>(est, d, sb, nchunks, [&](uint32_t slot, int64_t i) {
         if (slot >= cap) return;  // cannot happen with consistent histograms; never write past the list
         cand_idx[slot] = (int32_t)i;
         if (cand_est) cand_est[slot] = est[i];
@@ -396,11 +396,12 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
 // ------------------------------------------------------------------------------------------------
 // final emit (line 11) and zero-out (line 13)
 // ------------------------------------------------------------------------------------------------
+template <int ITEMS>
 __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const int32_t* __restrict__ cand,
              int32_t* __restrict__ out_idx, float* __restrict__ out_val, uint32_t cap, int64_t nchunks,
              uint32_t* __restrict__ pending) {
-    sel_emit_chunks(xs, ncand, sb, nchunks, [&](uint32_t slot, int64_t m) {
+    sel_emit_chunks<ITEMS>(xs, ncand, sb, nchunks, [&](uint32_t slot, int64_t m) {
         if (slot >= cap) return;
         const int32_t i = cand[m];
         out_idx[slot] = i;
