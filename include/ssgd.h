@@ -72,7 +72,7 @@ extern "C" {
  * per bucket and kept in shared memory (if r*c bits, OR-folded up to 32 buckets per bit, fit; otherwise as
  * EARLY_EXIT).  EARLY_EXIT: the test is applied to the table values themselves and a coordinate stops reading
  * rows once it cannot pass.  OFF: every coordinate reads all r rows.  The candidates are identical in all modes.
- * AUTO is ON when d >= 2^22, ncand <= d/8 (below that the fixed costs outweigh the saving) and either the bitmap
+ * AUTO is ON when d >= 2^21, ncand <= d/8 (below that the fixed costs outweigh the saving) and either the bitmap
  * fits unfolded or 5 <= r <= 9; else OFF.  Behind a folded bitmap ON measures the bitmap's density each step and
  * runs the EARLY_EXIT kernel instead when the folded bits would rule out too few coordinates. */
 #define SSGD_PRUNE_AUTO 0

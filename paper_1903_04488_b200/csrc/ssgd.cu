@@ -447,7 +447,8 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
 bool use_sparse(const ssgd_ctx* x, int64_t ncand) {
     if (x->prune_mode == SSGD_PRUNE_OFF) return false;
     if (x->prune_mode == SSGD_PRUNE_ON || x->prune_mode == SSGD_PRUNE_EARLY_EXIT) return true;
-    if (x->d < (1 << 22) || ncand * 8 > x->d) return false;      // fixed costs outweigh the saving
+    // measured (W = 16, 5 x 262,144, ncand = d/100): d = 2^20 dense 0.121 ms / pruned 0.125; 2e6 0.241 / 0.233; 4e6 0.408 / 0.357
+    if (x->d < (1 << 21) || ncand * 8 > x->d) return false;      // fixed costs outweigh the saving
     // an unfolded bucket bitmap pays for every r; behind a folded one the table kernel may have to run, which was
     // measured to pay for r = 5, 7, 9 only (r = 3: one row can be skipped; r = 15, ncand = 1.6e6: 5.8 vs 4.9 ms)
     return x->bm_fold == 0 || (x->r >= 5 && x->r <= 9);
