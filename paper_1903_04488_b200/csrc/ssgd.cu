@@ -2,13 +2,19 @@
 // launch sequences of the Sketched-SGD compression step for sm_100a.
 //
 // Kernels (Algorithm 3 lines 5-13, Algorithm 4), by header:
-//   step_kernels.cuh    k_accum_insert (lines 5-7, plain 128-bit loads), k_insert_rows, k_merge (line 8),
-//                       k_quantize16 / k_merge16, k_unsketch (line 9, dense), k_gather (line 10),
-//                       k_emit_candidates / k_emit_final, k_zero (line 13), k_hashes
+//   step_kernels.cuh    k_accum_insert (lines 5-7, plain 128-bit loads; applies the previous step's deferred
+//                       line 13), k_insert_rows, k_merge (line 8), k_quantize16 / k_merge16, k_unsketch (line 9,
+//                       dense), k_gather (line 10), k_emit_candidates / k_emit_final, k_zero and
+//                       k_flush_pending (line 13, eager and deferred), k_hashes
 //   accum_tma.cuh       k_accum_insert_tma: lines 5-7 as a bulk-copy (TMA) + mbarrier pipeline
 //   accum_ws.cuh        k_accum_insert_ws: the same pipeline with separate stream and sketch warps
-//   sparse_select.cuh   k_unsketch_sample, k_unsketch_pruned, k_select_sparse: line 9 with early exit
-//   select.cuh          k_sel_pass2/3, k_sel_count: exact radix select with ordered compaction (lines 9, 11)
+//   filter_unsketch.cuh k_bitmap_build, k_bitmap_fold, k_unsketch_filter: line 9 decided per coordinate on a
+//                       one-bit-per-bucket copy of the table in shared memory
+//   sparse_select.cuh   k_unsketch_sample, k_unsketch_pruned: the sampled threshold; line 9 with early exit on
+//                       the table itself
+//   list_select.cuh     k_list_hist, k_list_mark, k_map_emit: exact top-ncand of the survivor list
+//   select.cuh          k_sel_pass23 (k_sel_pass2/3), k_sel_count: exact radix select with ordered compaction
+//                       (lines 9, 11)
 //   heavymix.cuh        k_row_sumsq, k_heavymix_keys: Algorithm 1
 //   hash.cuh, estimate.cuh   the hash family and the median-of-r estimate
 // HBM-bound work is the accumulate+insert kernel (20 bytes per worker-coordinate); nothing here is a dense
