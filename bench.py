@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 ORACLE_COORDS_PER_S = 4.0e6        # conservative single-thread estimate used to size oracle samples
 # DRAM bytes per launch of k_accum_insert from an ncu capture (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by workload (None where no capture exists).
-NCU_TRAFFIC_BYTES = {"C2": 3.505e9}   # 1881.9 MB at d = 6,000,002 scaled in proportion to d (profiles/k_accum_insert_C2_d6M.md)
+NCU_TRAFFIC_BYTES = {"C2": 3.550e9}   # 1906.1 MB at d = 6,000,002 scaled in proportion to d (profiles/k_accum_insert_C2_d6M.md)
 
 
 def peaks():

@@ -174,6 +174,8 @@ int ssgd_exact_topk(ssgd_ctx* ctx, const int32_t* cand_idx, int64_t ncand, int32
 
 /* Algorithm 3 lines 5-13 in one call: the stages above, with the workers' values summed before the
  * insert (sum_w S(v_w) = S(sum_w v_w), Section 3), so no per-worker table is materialised.
+ * The same kernel keeps each coordinate's sum over the workers (fp64, worker order, rounded once), so line 10
+ * reads one number per candidate instead of W values of v; the result is bit-identical to ssgd_exact_topk's.
  * out_idx/out_val: [k] device outputs, ascending coordinate order.  Line 13 is applied as ssgd_set_zero_mode
  * says: by default it is deferred into the next ssgd_step (or ssgd_flush). */
 int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t ncand,

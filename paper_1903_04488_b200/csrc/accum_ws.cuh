@@ -107,7 +107,7 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
         for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x, ++nt) {
             const int64_t i0 = tile * WS_TC + 4 * st;
             const bool active = i0 < d_main;
-            float x0 = 0.f, x1 = 0.f, x2 = 0.f, x3 = 0.f;
+            double x0 = 0., x1 = 0., x2 = 0., x3 = 0.;
             const uint32_t pend = active ? pending_bits4(A.pending, i0) : 0u;
             for (int w = 0; w < A.W; ++w, ++n) {
                 const int s = n % WS_STAGES;
@@ -124,8 +124,8 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
                     un.w = __fmaf_rn(A.rho, u4.w, g4.w); vn.w = __fadd_rn(v4.w, un.w);
                     __stcs(reinterpret_cast<float4*>(A.u + (int64_t)w * A.ld + i0), un);
                     __stcs(reinterpret_cast<float4*>(A.v + (int64_t)w * A.ld + i0), vn);
-                    x0 = __fadd_rn(x0, vn.x); x1 = __fadd_rn(x1, vn.y);
-                    x2 = __fadd_rn(x2, vn.z); x3 = __fadd_rn(x3, vn.w);
+                    x0 = __dadd_rn(x0, (double)vn.x); x1 = __dadd_rn(x1, (double)vn.y);
+                    x2 = __dadd_rn(x2, (double)vn.z); x3 = __dadd_rn(x3, (double)vn.w);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.empty[s]);
@@ -134,7 +134,9 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
             // hand the tile's sums to the sketch warps
             const int b = nt & 1;
             if (nt >= 2 && !mbar_wait(&S.x_empty[b], ((nt >> 1) - 1) & 1, &S.abort)) { ok = false; break; }
-            *reinterpret_cast<float4*>(&S.x[b][4 * st]) = make_float4(x0, x1, x2, x3);
+            const float4 xf = make_float4((float)x0, (float)x1, (float)x2, (float)x3);
+            *reinterpret_cast<float4*>(&S.x[b][4 * st]) = xf;
+            if (active && A.xsum) __stcs(reinterpret_cast<float4*>(A.xsum + i0), xf);
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.x_full[b]);
         }
@@ -142,15 +144,17 @@ k_accum_insert_ws(const AccumArgs A, int32_t* __restrict__ errflag) {
         // ragged tail (d not a multiple of 4): at most three coordinates, plain loads, one thread
         if (ok && blockIdx.x == 0 && st == 0) {
             for (int64_t i = d_main; i < A.d; ++i) {
-                float x = 0.f;
+                double xd = 0.;
                 const bool pend = pending_bit(A.pending, i);
                 for (int64_t w = 0; w < A.W; ++w) {
                     const float un = __fmaf_rn(A.rho, pend ? 0.f : A.u[w * A.ld + i], A.g[w * A.ld_g + i]);
                     const float vn = __fadd_rn(pend ? 0.f : A.v[w * A.ld + i], un);
                     A.u[w * A.ld + i] = un;
                     A.v[w * A.ld + i] = vn;
-                    x = __fadd_rn(x, vn);
+                    xd = __dadd_rn(xd, (double)vn);
                 }
+                const float x = (float)xd;
+                if (A.xsum) A.xsum[i] = x;
                 for (int j = 0; j < R; ++j) {
                     uint32_t hb[1];
                     row_hashes<POW2, 1>(A.hp.row[j], A.bk, (uint32_t)i, hb);

@@ -77,6 +77,7 @@ struct ssgd_ctx {
     int32_t prune_mode;
     size_t persist_bytes;
     size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel   // > 0: launches that touch the table carry an L2 access-policy window of this size
+    size_t off_xsum;        // per-coordinate sums over the workers of the new v, written by ssgd_step's accumulate kernel
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;
     // device facts
@@ -135,6 +136,7 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->nchunk_c = (x->d + SEL_CHUNK - 1) / SEL_CHUNK;
     x->nchunk_f = (ncand_max + SEL_CHUNK_SMALL - 1) / SEL_CHUNK_SMALL;
     x->off_est = o;     o += up((size_t)x->d * 4);
+    x->off_xsum = o;    o += up((size_t)x->d * 4);
     x->off_chunk_c = o; o += up((size_t)x->nchunk_c * 8);
     x->off_chunk_f = o; o += up((size_t)x->nchunk_f * 8);
     x->off_cand = o;    o += up((size_t)ncand_max * 4);
@@ -567,16 +569,23 @@ int flush_pending(ssgd_ctx* x, cudaStream_t st) {
 
 // Lines 10, 11, 13.  deferred: the chosen coordinates are marked in the pending map instead of being zeroed now
 // (the caller's accumulate kernel has consumed the previous marks; k_gather empties the map before the new ones).
+// sums: the accumulate kernel's per-coordinate sums over the workers (ssgd_step), or NULL to read v (stage call).
 int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
-                       cudaStream_t st, bool deferred) {
+                       cudaStream_t st, bool deferred, const float* sums) {
     float* xs = reinterpret_cast<float*>(x->ws + x->off_xs);
     int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
     SelBuffers sb = sel_buffers(x, true);
     const int64_t nch = (ncand + SEL_CHUNK_SMALL - 1) / SEL_CHUNK_SMALL;
     uint32_t* pend = pending_map(x);                     // whatever the accumulate kernel consumed is cleared here
-    CU(launch_pdl(st, k_gather, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, (const float*)x->v, x->ld, x->W,
-                  x->d, xs, sb, (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather");
-    LAUNCHED("k_gather");
+    if (sums) {
+        CU(launch_pdl(st, k_gather_sums, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, sums, x->d, xs, sb,
+                      (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather_sums");
+        LAUNCHED("k_gather_sums");
+    } else {
+        CU(launch_pdl(st, k_gather, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, (const float*)x->v, x->ld, x->W,
+                      x->d, xs, sb, (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather");
+        LAUNCHED("k_gather");
+    }
     int e = launch_select(x, xs, ncand, sb, nch, st, true);
     if (e) return e;
     CU(launch_pdl(st, k_emit_final<SEL_ITEMS_SMALL>, grid_for(nch, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)xs, ncand, sb,
@@ -826,7 +835,7 @@ int ssgd_exact_topk(ssgd_ctx* x, const int32_t* cand_idx, int64_t ncand, int32_t
     if (x->pending_dirty && (e = flush_pending(x, st))) return e;
     CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_err - x->off_hist_f, st), "memset hist");
     x->launches++;
-    return gather_select_zero(x, cand_idx, ncand, out_idx, out_val, st, false);
+    return gather_select_zero(x, cand_idx, ncand, out_idx, out_val, st, false, nullptr);
 }
 
 int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncand, int32_t* out_idx,
@@ -852,7 +861,8 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     const size_t row_bytes = (size_t)x->c * 4;
     const int rows_fit = (int)(x->split_bytes / row_bytes);
     const bool split = mode == INS_MERGED_GLOBAL && x->split_bytes > 0 && rows_fit >= 1 && rows_fit < x->r;
-    if (split) { A.rows_here = rows_fit; A.xsum = reinterpret_cast<float*>(x->ws + x->off_est); }
+    A.xsum = reinterpret_cast<float*>(x->ws + x->off_xsum);   // the second round reads these instead of W values of v
+    if (split) A.rows_here = rows_fit;
     if ((e = mark(x, 0, st))) return e;
     if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st)
              : mode == INS_MERGED_WS ? launch_accum_ws(x, A, st) : launch_accum(x, A, mode, st))) return e;
@@ -868,7 +878,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
         if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
     }
     if ((e = mark(x, 3, st))) return e;
-    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED))) return e;
+    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED, A.xsum))) return e;
     if ((e = mark(x, 4, st))) return e;
     if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
     return SSGD_OK;

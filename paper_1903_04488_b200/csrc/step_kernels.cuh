@@ -76,7 +76,10 @@ k_accum_insert(const AccumArgs A) {
 #pragma unroll
             for (int j = 0; j < R; ++j) row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb[j]);
         }
-        float x[4] = {0.f, 0.f, 0.f, 0.f};  // sum over workers of the new v (worker order)
+        // sum over workers of the new v, in fp64 and worker order, rounded once: the value that is sketched and,
+        // through xsum, the second round's exact sum (Algorithm 3 line 10) of this coordinate
+        double xd[4] = {0., 0., 0., 0.};
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
         if (i0 + 3 < A.d) {
             constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : K1_UNROLL;
             for (int w0 = 0; w0 < A.W; w0 += U) {
@@ -116,8 +119,8 @@ k_accum_insert(const AccumArgs A) {
                                     if (vals[e] != 0.0f)
                                         red_add(tw + (int64_t)j * A.c + (hb[j][e] & P31), apply_sign(vals[e], hb[j][e]));
                         } else {
-                            x[0] = __fadd_rn(x[0], vn.x); x[1] = __fadd_rn(x[1], vn.y);
-                            x[2] = __fadd_rn(x[2], vn.z); x[3] = __fadd_rn(x[3], vn.w);
+                            xd[0] = __dadd_rn(xd[0], (double)vn.x); xd[1] = __dadd_rn(xd[1], (double)vn.y);
+                            xd[2] = __dadd_rn(xd[2], (double)vn.z); xd[3] = __dadd_rn(xd[3], (double)vn.w);
                         }
                     }
                 }
@@ -140,14 +143,17 @@ k_accum_insert(const AccumArgs A) {
                                 red_add(A.table + w * rc + (int64_t)j * A.c + (hb[j][e] & P31),
                                         apply_sign(vn, hb[j][e]));
                     } else {
-                        x[e] = __fadd_rn(x[e], vn);
+                        xd[e] = __dadd_rn(xd[e], (double)vn);
                     }
                 }
             }
         }
         if (MODE != INS_PER_WORKER) {
-            if (MODE == INS_MERGED_GLOBAL && A.xsum != nullptr) {
-                if (i0 + 3 < A.d) *reinterpret_cast<float4*>(A.xsum + i0) = make_float4(x[0], x[1], x[2], x[3]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) x[e] = (float)xd[e];
+            if (A.xsum != nullptr) {
+                // streaming store: measured 7 us faster at C2 than a store that competes with the table for L2
+                if (i0 + 3 < A.d) __stcs(reinterpret_cast<float4*>(A.xsum + i0), make_float4(x[0], x[1], x[2], x[3]));
                 else for (int e = 0; e < 4 && i0 + e < A.d; ++e) A.xsum[i0 + e] = x[e];
             }
 #pragma unroll
@@ -385,6 +391,35 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
             for (; w < W; ++w) acc = __dadd_rn(acc, (double)__ldg(p + (int64_t)w * ld));
             out = (float)acc;
         }
+        xs[m] = out;
+        atomicAdd(&s_hist[key_of(out) >> H1_SHIFT], 1u);
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(s_hist, sb.h1);
+    producer_epilogue(sb, want, sh);
+}
+
+// Line 10 inside ssgd_step: the accumulate kernel has already summed every coordinate's new v over the workers
+// (fp64, worker order, rounded once) on its way to the sketch, so the second round's exact sum of a candidate is
+// one read of that array instead of W scattered reads of v.
+__global__ void __launch_bounds__(256)
+k_gather_sums(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ xsum, int64_t d,
+              float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag,
+              uint32_t* __restrict__ pending_clear, int64_t pending_words) {
+    __shared__ SelShared sh;
+    uint32_t* s_hist = sh.hist;
+    pdl_trigger();
+    for (int b = threadIdx.x; b < H1_BINS; b += 256) s_hist[b] = 0;
+    pdl_wait();
+    __syncthreads();
+    const int64_t m = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    if (pending_clear)
+        for (int64_t t = m; t < pending_words; t += (int64_t)gridDim.x * 256) pending_clear[t] = 0u;
+    if (m < ncand) {
+        const int64_t i = cand[m];
+        float out = 0.0f;
+        if (i < 0 || i >= d) atomicExch(errflag, ERR_BAD_INDEX);
+        else out = __ldg(xsum + i);
         xs[m] = out;
         atomicAdd(&s_hist[key_of(out) >> H1_SHIFT], 1u);
     }

@@ -67,7 +67,7 @@ def test_workspace_bytes(lib):
     d, r, c, k, W = 11_173_962, 5, 262_144, 50_000, 16
     eng = S.Ssgd(d, r, c, k, W, 0)
     n = eng.workspace_bytes(100_000)
-    floor = 4 * r * c + 4 * d + 8 * 100_000          # table + estimates + candidates and their sums
+    floor = 4 * r * c + 8 * d + 8 * 100_000          # table + estimates + per-coordinate sums + candidates and their sums
     extra = 3 * (d // 8) + 8 * d + (1 << 22)         # three coordinate bitmaps (two of the list selection, one of the
     extra += r * c // 8                              # deferred zero-out), a survivor list with room for every coordinate,
     assert floor + extra <= n <= floor + extra + (1 << 20)   # two 2^19-bin histograms, one bit per bucket
