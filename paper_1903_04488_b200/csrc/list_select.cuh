@@ -11,7 +11,8 @@
 //                   themselves on their chunk of map words; the last block turns the counts into exclusive offsets.
 //   k_map_emit      walks the maps in coordinate order: an A bit with a A-bits and b B-bits before it goes to
 //                   slot a + min(b, Q); a B bit with b < Q to slot a + b.  Ties at the threshold therefore go
-//                   to the smallest coordinates, without a sort and without a limit on their number.
+//                   to the smallest coordinates, without a sort and without a limit on their number.  In ssgd_step
+//                   the second round's read of each candidate's exact sum rides on this kernel.
 //
 // Nothing here waits on another block: "last block" means the block that draws the last ticket after a fence.
 #pragma once
@@ -121,13 +122,35 @@ __device__ __forceinline__ void load_map_words(const SparseBuffers& sp, int64_t 
 // Word order inside a chunk is (it, tid): word = base + it*256 + tid, so "before" means smaller it, or the same
 // it and a smaller thread.  Per it, a block-wide exclusive scan of the words' A and B counts gives each word the
 // number of A and B bits before it.
+// Optional second round (Algorithm 3 line 10) riding on the emit: with the per-coordinate sums over the workers
+// at hand (ssgd_step), the exact sum of each emitted candidate is read here, written to xs[slot] and counted in
+// the final selection's first histogram, so no separate gather launch follows.
+struct EmitSecondRound {
+    const float* xsum;         // [d], or NULL: emit only
+    float* xs;                 // [ncand]
+    SelBuffers sb;             // final selection: h1 is filled here, its first digit found by the last block
+    uint32_t want;             // k
+    uint32_t* pending_clear;   // the deferred zero-out's map, emptied here (or NULL)
+    int64_t pending_words;
+};
+
 __global__ void __launch_bounds__(SEL_THREADS)
-k_map_emit(SparseBuffers sp, int64_t nwords, int64_t nchunks, uint32_t m, int32_t* __restrict__ cand_idx) {
+k_map_emit(SparseBuffers sp, int64_t nwords, int64_t nchunks, uint32_t m, int32_t* __restrict__ cand_idx,
+           EmitSecondRound E) {
+    __shared__ SelShared sh;
     __shared__ uint32_t s_wa[SEL_WARPS], s_wb[SEL_WARPS];
     pdl_trigger();
+    if (E.xsum) for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
+    if (E.xsum && E.pending_clear)
+        for (int64_t t = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; t < E.pending_words; t += (int64_t)gridDim.x * SEL_THREADS)
+            E.pending_clear[t] = 0u;
+    __syncthreads();
     const uint32_t Q = __ldcg(&sp.state->quota_eq);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    auto emit = [&](uint32_t slot, int64_t coord) {
+        if (slot < m) cand_idx[slot] = (int32_t)coord;
+    };
     for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
         if (__ldcg(sp.chunk_a + chunk) + __ldcg(sp.chunk_b + chunk) ==
             (chunk + 1 < nchunks ? __ldcg(sp.chunk_a + chunk + 1) + __ldcg(sp.chunk_b + chunk + 1) : 0xFFFFFFFFu))
@@ -136,6 +159,7 @@ k_map_emit(SparseBuffers sp, int64_t nwords, int64_t nchunks, uint32_t m, int32_
         const int64_t base = chunk * MAP_CHUNK_WORDS;
         load_map_words(sp, nwords, base, wa, wb);
         uint32_t run_a = __ldcg(sp.chunk_a + chunk), run_b = __ldcg(sp.chunk_b + chunk);
+        const uint32_t slot_lo = run_a + (run_b < Q ? run_b : Q);      // this chunk's candidates fill [slot_lo, slot_hi)
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
             const uint32_t ca = __popc(wa[it]), cb = __popc(wb[it]);
@@ -159,17 +183,33 @@ k_map_emit(SparseBuffers sp, int64_t nwords, int64_t nchunks, uint32_t m, int32_
                 const int bit = __ffs(bits) - 1;
                 bits &= bits - 1;
                 if ((wa[it] >> bit) & 1u) {
-                    const uint32_t slot = a + (b < Q ? b : Q);
-                    if (slot < m) cand_idx[slot] = (int32_t)(w0 + bit);
+                    emit(a + (b < Q ? b : Q), w0 + bit);
                     ++a;
                 } else {
-                    if (b < Q) { const uint32_t slot = a + b; if (slot < m) cand_idx[slot] = (int32_t)(w0 + bit); }
+                    if (b < Q) emit(a + b, w0 + bit);
                     ++b;
                 }
             }
             run_a += ta;
             run_b += tb;
         }
+        if (E.xsum) {
+            // second round for this chunk's candidates, all threads of the block in parallel (the loop above hands
+            // a thread its candidates one after another: reading the sums there would serialise the latencies)
+            uint32_t slot_hi = run_a + (run_b < Q ? run_b : Q);
+            if (slot_hi > m) slot_hi = m;
+            __syncthreads();                                 // the block's cand_idx stores are visible to the block
+            for (uint32_t slot = slot_lo + threadIdx.x; slot < slot_hi; slot += SEL_THREADS) {
+                const float x = __ldg(E.xsum + cand_idx[slot]);
+                E.xs[slot] = x;
+                atomicAdd(&sh.hist[key_of(x) >> H1_SHIFT], 1u);
+            }
+        }
+    }
+    if (E.xsum) {
+        __syncthreads();
+        flush_hist<H1_BINS>(sh.hist, E.sb.h1);
+        producer_epilogue(E.sb, E.want, sh);
     }
 }
 

@@ -527,7 +527,9 @@ int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
 
 // Line 9 with early exit: sample -> pruned unsketch (-> unpruned rerun if the sample misjudged) -> selection on
 // the survivor list (list_select.cuh).
-int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, cudaStream_t st) {
+// sums != NULL: the emit kernel also performs the second round (xs, first histogram of the final selection).
+int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int32_t* cand_idx, cudaStream_t st,
+                           const float* sums) {
     SparseArgs A;
     A.table = merged; A.c = x->c; A.d = x->d; A.hp = x->hp; A.bk = x->bk;
     A.sp = sparse_buffers(x);
@@ -549,7 +551,16 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     LAUNCHED("k_list_mark");
     const int64_t nwords = (x->d + 31) / 32;
     const int map_grid = grid_for(x->nchunk_map, 1, (int64_t)x->sm_count * 8);
-    CU(launch_pdl(st, k_map_emit, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map, (uint32_t)ncand, cand_idx),
+    EmitSecondRound E{};
+    if (sums) {
+        E.xsum = sums;
+        E.xs = reinterpret_cast<float*>(x->ws + x->off_xs);
+        E.sb = sel_buffers(x, true);
+        E.want = (uint32_t)x->k;
+        E.pending_clear = reinterpret_cast<uint32_t*>(x->ws + x->off_pending);
+        E.pending_words = nwords;
+    }
+    CU(launch_pdl(st, k_map_emit, map_grid, SEL_THREADS, 0, A.sp, nwords, x->nchunk_map, (uint32_t)ncand, cand_idx, E),
        "launch k_map_emit");
     LAUNCHED("k_map_emit");
     return SSGD_OK;
@@ -570,14 +581,16 @@ int flush_pending(ssgd_ctx* x, cudaStream_t st) {
 // Lines 10, 11, 13.  deferred: the chosen coordinates are marked in the pending map instead of being zeroed now
 // (the caller's accumulate kernel has consumed the previous marks; k_gather empties the map before the new ones).
 // sums: the accumulate kernel's per-coordinate sums over the workers (ssgd_step), or NULL to read v (stage call).
+// xs_ready: the candidate stage has already produced xs and the first histogram (k_map_emit's second round).
 int gather_select_zero(ssgd_ctx* x, const int32_t* cand, int64_t ncand, int32_t* out_idx, float* out_val,
-                       cudaStream_t st, bool deferred, const float* sums) {
+                       cudaStream_t st, bool deferred, const float* sums, bool xs_ready = false) {
     float* xs = reinterpret_cast<float*>(x->ws + x->off_xs);
     int32_t* err = reinterpret_cast<int32_t*>(x->ws + x->off_err);
     SelBuffers sb = sel_buffers(x, true);
     const int64_t nch = (ncand + SEL_CHUNK_SMALL - 1) / SEL_CHUNK_SMALL;
     uint32_t* pend = pending_map(x);                     // whatever the accumulate kernel consumed is cleared here
-    if (sums) {
+    if (xs_ready) {
+    } else if (sums) {
         CU(launch_pdl(st, k_gather_sums, grid_for(ncand, 256, (int64_t)1 << 30), 256, 0, cand, ncand, sums, x->d, xs, sb,
                       (uint32_t)x->k, err, pend, (int64_t)((x->d + 31) / 32)), "launch k_gather_sums");
         LAUNCHED("k_gather_sums");
@@ -872,13 +885,14 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);
-    if (use_sparse(x, ncand)) {
-        if ((e = unsketch_select_sparse(x, merged, ncand, cand, st))) return e;
+    const bool sparse = use_sparse(x, ncand);
+    if (sparse) {
+        if ((e = unsketch_select_sparse(x, merged, ncand, cand, st, A.xsum))) return e;
     } else {
         if ((e = unsketch_select(x, merged, ncand, cand, nullptr, est, st, true))) return e;
     }
     if ((e = mark(x, 3, st))) return e;
-    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED, A.xsum))) return e;
+    if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED, A.xsum, sparse))) return e;
     if ((e = mark(x, 4, st))) return e;
     if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
     return SSGD_OK;
