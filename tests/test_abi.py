@@ -90,7 +90,21 @@ def test_unbound_context_refuses_to_run(lib):
     assert lib.ssgd_bind(eng._h, 16, 16, 102, 256, 1 << 30, 20) == S.EALIGN      # ld % 4 != 0
     assert lib.ssgd_bind(eng._h, 16, 16, 96, 256, 1 << 30, 20) == S.EINVAL       # ld < d
     assert lib.ssgd_bind(eng._h, 16, 16, 100, 256, 64, 20) == S.EWORKSPACE
+    assert lib.ssgd_flush(eng._h, None) == S.ENOTBOUND
     assert eng.launch_count() == 0
+
+
+def test_mode_setters_check_their_argument(lib):
+    eng = S.Ssgd(100, 5, 16, 10, 2, 1)
+    for fn, good, bad in ((lib.ssgd_set_zero_mode, (S.ZERO_DEFERRED, S.ZERO_EAGER), (-1, 2)),
+                          (lib.ssgd_set_prune_mode, (S.PRUNE_AUTO, S.PRUNE_OFF, S.PRUNE_ON, S.PRUNE_EARLY_EXIT), (-1, 4)),
+                          (lib.ssgd_set_insert_mode, (S.INSERT_AUTO, S.INSERT_GLOBAL, S.INSERT_SMEM, S.INSERT_TMA, S.INSERT_WS),
+                           (-1, 5))):
+        for m in good:
+            assert fn(eng._h, m) == S.OK
+        for m in bad:
+            assert fn(eng._h, m) == S.EINVAL
+        assert fn(None, good[0]) == S.EINVAL
 
 
 def test_error_strings(lib):
