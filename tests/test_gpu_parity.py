@@ -148,6 +148,8 @@ STEP_CASES = [
     (wl.C2.scaled(d=70_001, W=17, r=3, c=999, ncand=300, k=300), 2),       # k == ncand, odd W
     (wl.C2.scaled(d=20_000, W=1, r=1, c=64, ncand=20_000, k=50), 2),       # ncand == d: true top-k
     (wl.C1.scaled(d=3, W=2, r=5, c=16, ncand=2, k=1), 2),                  # d < 4
+    (wl.C2.scaled(d=1, W=1, r=1, c=1, ncand=1, k=1), 2),                   # the smallest problem there is
+    (wl.C2.scaled(d=4097, W=2, r=9, c=33, ncand=4097, k=4097), 2),         # k == ncand == d: everything is chosen
     (wl.P1.scaled(d=400_000, c=1_800, ncand=8_000, k=500), 2),             # the paper's 15-row sketch, P = 16
     (wl.P2.scaled(d=500_000, c=10_000, ncand=18_000, k=500), 2),           # the paper's 5 x 1M sketch, P = 36
     (wl.P3.scaled(d=365_000, c=900, ncand=13_000, k=500), 2),              # the paper's LSTM sketch, P = 26
