@@ -433,6 +433,14 @@ def test_full_size_C5_worker_sweep(cuda_device, W):
     run_full(cfg, cuda_device, 1, True)
 
 
+def test_full_size_many_coordinates_few_workers(cuda_device):
+    """d = 1.5e8 with one worker: more map chunks than the mark kernel's block-local counters hold (it falls back
+    to global counters), 4.7e6 map words, a survivor list with room for 1.5e8 entries, indices above 2^27."""
+    cfg = wl.C2.scaled(name="big_d", d=150_000_001, W=1, ncand=60_000, k=20_000, steps=1)
+    assert ((cfg.d + 31) // 32 + 2047) // 2048 > 2048         # chunks of 2048 map words: more than 2048 of them
+    run_full(cfg, cuda_device, 1, True)
+
+
 def test_stored_small_case_is_reproduced_exactly(cuda_device):
     """Integer gradients and rho = 1/2 make every operation exact, reductions included, so the library must
     reproduce the stored case (written by the oracle alone) bit for bit: table, candidates, k-set, values."""
