@@ -75,10 +75,15 @@ k_bitmap_build(const FilterArgs F) {
         const int64_t w0 = (task - j * tasks_per_row) * 32;          // first word of this task in row j
         const float* row = F.A.table + j * F.A.c;
         uint32_t mine = 0;
-#pragma unroll 8
+        uint32_t key[32];                                    // all 32 loads in flight: one L2 round trip per task
+#pragma unroll
         for (int k = 0; k < 32; ++k) {
             const int64_t b = (w0 + k) * 32 + lane;
-            const bool big = b < F.A.c && (key_of(__ldcg(row + b)) >> H1_SHIFT) >= bin_lo;
+            key[k] = b < F.A.c ? key_of(__ldcg(row + b)) : 0xFFFFFFFFu;
+        }
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+            const bool big = key[k] != 0xFFFFFFFFu && (key[k] >> H1_SHIFT) >= bin_lo;
             const uint32_t bal = __ballot_sync(0xFFFFFFFFu, big);
             if (lane == k) mine = bal;
         }

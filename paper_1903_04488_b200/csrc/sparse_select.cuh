@@ -69,6 +69,7 @@ struct SparseArgs {
     SparseBuffers sp;
     uint32_t ncand;
     uint32_t want_sample;  // rank (from the top) in the sample's histogram that defines bin_lo
+    uint32_t n_sampled_min; // a lower bound of the number of sampled coordinates: 4 * (windows - 2)
     int32_t rerun;         // 0: the pruned pass; 1: the unpruned pass behind it (runs only if fallback == 1)
     int32_t gated;         // 1: the pruned pass runs only if use_table is set (it follows a bitmap filter that declined)
 };
@@ -111,19 +112,12 @@ k_unsketch_sample(const SparseArgs A) {
     __syncthreads();
     flush_hist<H1_BINS>(sh.hist, A.sp.h1_sample);
     if (block_is_last(&A.sp.state->ticket[0], sh)) {
-        // total sampled; if the sample is too small to place the rank, prune nothing (bin_lo stays 0)
+        // if the sample is too small to place the rank, prune nothing (bin_lo stays 0); the number of sampled
+        // coordinates is a function of d alone: every window holds one group of 4, the last group may be short
         uint32_t digit = 0, rem = 0;
         block_find_from_top<H1_BINS>(A.sp.h1_sample, A.want_sample, sh, digit, rem);
-        uint32_t part = 0;
-        for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) part += __ldcg(A.sp.h1_sample + b);
-        for (int off = 16; off; off >>= 1) part += __shfl_xor_sync(0xFFFFFFFFu, part, off);
-        if ((threadIdx.x & 31) == 0) sh.warp_sum[threadIdx.x >> 5] = part;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t total = 0;
-            for (int w = 0; w < SEL_WARPS; ++w) total += sh.warp_sum[w];
-            A.sp.state->bin_lo = (A.want_sample >= 1 && A.want_sample <= total) ? digit : 0u;
-        }
+        if (threadIdx.x == 0)
+            A.sp.state->bin_lo = (A.want_sample >= 1 && A.want_sample <= A.n_sampled_min) ? digit : 0u;
     }
 }
 

@@ -473,7 +473,7 @@ template <int R, bool POW2>
 int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
     const int64_t groups = (A.d + 3) / 4;
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
-    CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count), SEL_THREADS, 0, A),
+    CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, A),
        "launch k_unsketch_sample");
     LAUNCHED("k_unsketch_sample");
     const int pruned_grid = grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID);
@@ -540,6 +540,7 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
     const double mean = (double)ncand * (double)(windows * 4) / (double)x->d;
     A.want_sample = x->sample_rank ? x->sample_rank : (uint32_t)(mean + 6.0 * std::sqrt(mean) + 16.0 + 1.0);
+    A.n_sampled_min = windows > 2 ? (uint32_t)(4 * (windows - 2)) : 0u;   // the last window may point past d, the last group may be short
     int e = launch_sparse(x, A, st);
     if (e) return e;
     if ((e = mark(x, 2, st))) return e;
