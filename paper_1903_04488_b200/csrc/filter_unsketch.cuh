@@ -199,6 +199,7 @@ k_unsketch_filter(const FilterArgs F) {
     const uint32_t bin_lo = __ldcg(&A.sp.state->bin_lo);
     {
         // asynchronous 16-byte copies, all in flight at once: the fill costs one L2 round trip, not one per piece
+        // (measured at C2: five 32 KiB bulk copies issued by one thread and awaited on an mbarrier take 2.5 us longer)
         const uint4* src = reinterpret_cast<const uint4*>(fold ? F.bm_fold : F.bm_full);
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(bm);
         for (int w = threadIdx.x; w < nw / 4; w += FILTER_THREADS)
