@@ -2,6 +2,8 @@
 whole step, on the same seeded inputs.  Integer work (hashes, signs, selections given their inputs,
 the zero-out mask, u and v) is compared bit for bit; the sketch table within 1e-5 of the L1 mass of
 each bucket, because the order of the reductions is not fixed."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -514,6 +516,42 @@ def test_step_can_be_captured_in_a_cuda_graph(cuda_device):
         assert (eager_val.cpu().numpy()[ia] == ov.cpu().numpy()[ib]).all()
         eng.flush()                                       # the replayed step only marked its k coordinates
         assert int((v[0, :cfg.d] == 0).sum().item()) >= cfg.k
+
+
+# ------------------------------------------------------------------------------------------------
+# seeded random shapes: every combination of sizes a user could pass, small enough for the oracle
+# ------------------------------------------------------------------------------------------------
+def _random_case(seed):
+    rng = np.random.default_rng(seed)
+    kind = ["lognormal_planted", "block_gauss", "block_laplace", "embedding_mix"][int(rng.integers(4))]
+    base = {"lognormal_planted": wl.C1, "block_gauss": wl.C2, "block_laplace": wl.C3, "embedding_mix": wl.C4}[kind]
+    d = int(rng.choice([int(rng.integers(1, 64)), int(rng.integers(64, 5000)), int(rng.integers(5000, 400_000))]))
+    r = int(rng.choice([1, 3, 5, 7, 9, 11, 13, 15]))
+    # power-of-two and arbitrary column counts, from one bucket to sketches whose bucket bitmap must be folded
+    c = int(rng.choice([1 << int(rng.integers(0, 21)), int(rng.integers(1, 3_000_000))]))
+    if r * c * 4 > (96 << 20):
+        c = max(1, (96 << 20) // (4 * r))
+    W = int(rng.choice([1, 2, 3, 5, 8, 17]))
+    ncand = int(rng.integers(1, d + 1))
+    k = int(rng.integers(1, ncand + 1))
+    prune = int(rng.choice([S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_AUTO]))
+    mode = int(rng.choice([S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_AUTO]))
+    zero = int(rng.choice([S.ZERO_DEFERRED, S.ZERO_EAGER]))
+    cfg = base.scaled(name=f"rnd{seed}", d=d, W=W, r=r, c=c, ncand=ncand, k=k, base_seed=1000 + seed)
+    return cfg, prune, mode, zero
+
+
+@pytest.mark.parametrize("seed", range(int(os.environ.get("SSGD_RANDOM_CASES", "48"))))
+def test_random_shapes_lockstep(cuda_device, seed):
+    cfg, prune, mode, zero = _random_case(seed)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_insert_mode(mode)
+    eng.set_prune_mode(prune)
+    eng.set_zero_mode(zero)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    for t in range(3):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o, flush=(t == 2))
 
 
 # ------------------------------------------------------------------------------------------------
