@@ -106,11 +106,11 @@ __device__ __forceinline__ float binomial_tail(int r, int need, float p) {
 // A folded bitmap is used only if it passes at most this share of the coordinates (estimated from its density as
 // a binomial tail); otherwise the first pass reads the table.  Measured on B200, r = 5, whole step in ms with the
 // filter / with the table kernel, by estimated share: 0.63 (d = 2e7, c = 2^20, 4 buckets per bit) 2.70 / 2.84;
-// 0.77 (same, ncand doubled) 2.79 / 2.89; 0.86 (ncand x 4) 2.92 / 2.96; 0.88 (d = 9e7, c = 1e6, 4 per bit)
-// 4.83 / 4.92; 0.68 with a 2.6 MB full bitmap behind it (d = 1.1e7, c = 2^22, 16 per bit) 1.25 / 1.25;
-// 0.99 (d = 9e7, c = 2^22, 16 per bit) 9.6 / 8.3; r = 15, 0.95 (d = 9e7, c = 180,000, 2 per bit) 16.7 / 12.5.
+// 0.77 (same, ncand doubled) 2.79 / 2.89; 0.88 (d = 9e7, c = 1e6, 4 per bit) 4.82 / 4.91; 0.90 (d = 9e7, c = 2^22,
+// 16 per bit, ncand = 5e4) 7.49 / 7.85; 0.96 (d = 2e7, c = 2^20, ncand = 1.6e6) 2.65 / 2.60; 0.99 (d = 9e7, c = 2^22,
+// ncand = 2e5) 7.97 / 7.99; r = 15, 0.95 (d = 9e7, c = 180,000, 2 per bit) 16.7 / 12.5.
 #ifndef SSGD_FILTER_MAX_PASS
-#define SSGD_FILTER_MAX_PASS 0.8f
+#define SSGD_FILTER_MAX_PASS 0.93f
 #endif
 
 // One thread per folded word: 32 folded bits, each the OR of 2^s consecutive bits of the full bitmap.  The last
