@@ -624,7 +624,9 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     if (x->insert_mode == SSGD_INSERT_WS) return INS_MERGED_WS;
     // measured on B200: the bulk-copy pipeline wins once a tile's walk over the workers is long
     // (W = 128: 5.73 vs 5.43 TB/s), plain loads win for short walks (W = 16: 4.93 vs 4.83 TB/s)
-    return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
+    // measured at C2's d (plain / bulk-copy, TB/s): W = 32 5.98 / 5.36; 96 5.79 / 5.64; 128 5.72 / 5.69; 192 5.53 / 5.71;
+    // 256 5.43 / 5.70 -- the plain kernel's threads loop over the workers 16 at a time, and loop less well than they start
+    return x->W > 128 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
 template <int R, bool POW2>
