@@ -264,8 +264,17 @@ int launch_accum_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
         k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, smem, st>>>(A);
     } else {
         const int grid = grid_for(groups, K1_THREADS, (int64_t)1 << 30);
-        CU(launch_pdl_w(st, L2Window{MODE == INS_MERGED_GLOBAL ? A.table : nullptr, x->persist_bytes},
-                        k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
+        bool few = false;
+        if constexpr (MODE == INS_MERGED_GLOBAL) {
+            if (A.W <= K1_UNROLL_FEW) {
+                few = true;
+                CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, k_accum_insert<R, POW2, MODE, K1_UNROLL_FEW>, grid,
+                                K1_THREADS, 0, A), "launch k_accum_insert");
+            }
+        }
+        if (!few)
+            CU(launch_pdl_w(st, L2Window{MODE == INS_MERGED_GLOBAL ? A.table : nullptr, x->persist_bytes},
+                            k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
     }
     LAUNCHED("k_accum_insert");
     return SSGD_OK;

@@ -56,7 +56,11 @@ constexpr int K1_THREADS = SSGD_K1_THREADS;
 constexpr int K1_UNROLL = SSGD_K1_UNROLL;  // workers in flight per thread: 3 x 16 B loads each
 constexpr int K1_UNROLL_PW = 4;            // same, for the per-worker-table mode (it also holds 4r hashes)
 
-template <int R, bool POW2, int MODE>
+// UM: workers in flight per thread in the merged modes.  Measured on B200 with 4 workers (d = 7.3e7 / 9e7, r = 5):
+// 16 -> 4 brings the kernel from 2.44 / 3.03 ms to 2.18 / 2.69 ms (a third of the registers, more resident blocks
+// to cover the stream while the reductions issue); with 8 workers 4, 8 and 16 are equal.
+constexpr int K1_UNROLL_FEW = 4;
+template <int R, bool POW2, int MODE, int UM = K1_UNROLL>
 __global__ void __launch_bounds__(K1_THREADS, SSGD_K1_MINBLOCKS)
 k_accum_insert(const AccumArgs A) {
     extern __shared__ float s_table[];  // MODE == INS_MERGED_SMEM: [R][c]
@@ -81,7 +85,7 @@ k_accum_insert(const AccumArgs A) {
         double xd[4] = {0., 0., 0., 0.};
         float x[4] = {0.f, 0.f, 0.f, 0.f};
         if (i0 + 3 < A.d) {
-            constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : K1_UNROLL;
+            constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : UM;
             for (int w0 = 0; w0 < A.W; w0 += U) {
                 float4 gg[U], uu[U], vv[U];
 #pragma unroll
