@@ -64,7 +64,6 @@ extern "C" {
 #define SSGD_INSERT_GLOBAL 1  /* plain 128-bit loads; reductions straight into the L2-resident table    */
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
-#define SSGD_INSERT_WS     4  /* the same pipeline, warp-specialised: separate stream and sketch warps   */
 
 /* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  A median of r values reaches a magnitude
  * only if (r+1)/2 of them do, so with a threshold taken from a sample of the estimates most coordinates can be
@@ -188,8 +187,9 @@ int ssgd_step(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, int64_t nc
  *           a 30-bit priority mixed from (fill_seed, i) -- z = fill_seed + (i+1)*0x9E3779B97F4A7C15,
  *           z = (z^(z>>30))*0xBF58476D1CE4E5B9, z = (z^(z>>27))*0x94D049BB133111EB, z ^= z>>31, priority = z>>34
  *           -- and the non-heavy coordinates with the largest priorities are taken (ties: smaller index).
- *           Should more than k coordinates be heavy (outside the paper's guarantee), the k with the largest
- *           |est| (compared without the last mantissa bit) are kept.
+ *           Should more than k coordinates be heavy (outside the paper's guarantee), the k heavy coordinates
+ *           with the largest |est| are kept (fp32 bit pattern of the magnitude, ties: smaller index) and
+ *           nothing else.
  *   line 5  out_val[t] = sum over the workers of the bound v at out_idx[t] (fp64, worker order).
  * out_idx / out_val: [k] device outputs, ascending coordinate order.  l2_out (device double) and nheavy_out
  * (device int32) are optional.  The bound state is read, not modified (a deferred zero-out is applied first).

@@ -361,26 +361,33 @@ int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const floa
         (g2 >= thr ? H : NH).push_back((int32_t)i);
     }
     if (nheavy_out) *nheavy_out = (int64_t)H.size();
-    // line 4: Top_k = H + rand_l(NH).  One ordering expresses it: heavy coordinates come first (among
-    // themselves by magnitude), the others in the order of their fill priority; the k first are taken.
-    std::vector<uint32_t> key((size_t)x->d);
-    {
-        std::vector<int64_t> all((size_t)x->d);
-        for (int64_t i = 0; i < x->d; ++i) all[(size_t)i] = i;
-        std::vector<uint32_t> prio((size_t)x->d);
-        if ((e = ssgd_oracle_fill_priority(fill_seed, x->d, all.data(), prio.data()))) return e;
-        for (int64_t i = 0; i < x->d; ++i) {
-            const double g2 = (double)est[(size_t)i] * (double)est[(size_t)i];
-            key[(size_t)i] = g2 >= thr ? (0x40000000u | (abs_bits(est[(size_t)i]) >> 1)) : prio[(size_t)i];
-        }
+    // line 4: Top_k = H + rand_l(NH), with l = k - |H|
+    std::vector<int32_t> top;
+    if ((int64_t)H.size() <= x->k) {
+        top = H;
+        const int64_t l = x->k - (int64_t)H.size();
+        // rand_l(NH): the l members of NH with the largest fill priority, ties to the smaller index
+        std::vector<int64_t> nh64(NH.begin(), NH.end());
+        std::vector<uint32_t> prio(NH.size());
+        if ((e = ssgd_oracle_fill_priority(fill_seed, (int64_t)NH.size(), nh64.data(), prio.data()))) return e;
+        std::vector<int64_t> order(NH.size());
+        for (size_t t = 0; t < NH.size(); ++t) order[t] = (int64_t)t;
+        std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+            if (prio[(size_t)a] != prio[(size_t)b]) return prio[(size_t)a] > prio[(size_t)b];
+            return NH[(size_t)a] < NH[(size_t)b];
+        });
+        for (int64_t t = 0; t < l; ++t) top.push_back(NH[(size_t)order[(size_t)t]]);
+    } else {
+        // more heavy coordinates than k (outside the paper's guarantee, which has |H| <= k): keep the k
+        // members of H with the largest |estimate| (fp32 bit pattern of the magnitude), ties to the smaller index
+        std::vector<int32_t> order = H;
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
+            const uint32_t ka = abs_bits(est[(size_t)a]), kb = abs_bits(est[(size_t)b]);
+            if (ka != kb) return ka > kb;
+            return a < b;
+        });
+        top.assign(order.begin(), order.begin() + x->k);
     }
-    std::vector<int32_t> order((size_t)x->d);
-    for (int64_t i = 0; i < x->d; ++i) order[(size_t)i] = (int32_t)i;
-    std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) {
-        if (key[(size_t)a] != key[(size_t)b]) return key[(size_t)a] > key[(size_t)b];
-        return a < b;
-    });
-    std::vector<int32_t> top(order.begin(), order.begin() + x->k);
     std::sort(top.begin(), top.end());
     // line 5
     std::vector<double> xs((size_t)x->k);

@@ -122,12 +122,12 @@ int ssgd_oracle_l2_estimate(const ssgd_oracle_ctx* ctx, const float* Tf, double*
 /* Lines 1-5 on an fp32 [r][c] table Tf:
  *   l2 = ssgd_oracle_l2_estimate;  est = ssgd_oracle_estimate;
  *   H  = { i : (double)est_i^2 >= l2/k }           (line 3, read with the square its proof uses)
- *   Top = the k first coordinates when heavy ones are put first and the others follow by fill priority:
- *         key(i) = 2^30 + floor(bits(|est_i|) / 2)  if i is in H,  else  priority(i)  (< 2^30);
- *         larger key first, ties to the smaller index.
- *         For |H| <= k that is H plus a random (k-|H|)-subset of NH (line 4).  |H| > k lies outside the
- *         paper's guarantee and its line 4; the same ordering then keeps the k heavy coordinates with
- *         the largest estimates (magnitudes compared without their last mantissa bit).
+ *   NH = the other coordinates
+ *   Top = H + rand_l(NH), l = k - |H|               (line 4): the l members of NH with the largest fill
+ *         priority, ties to the smaller index.
+ *         |H| > k lies outside the paper's guarantee and its line 4 (l would be negative); the reading taken
+ *         then is "the k members of H with the largest |est|" under the method's usual total order
+ *         (fp32 bit pattern of the magnitude, ties to the smaller index), and nothing from NH.
  *   out_val[t] = (float) sum over w = 0..W-1 of v_w[out_idx[t]]   (line 5, fp64 in worker order)
  * out_idx is ascending.  nheavy_out receives |H|.  The state is not modified. */
 int ssgd_oracle_heavymix(const ssgd_oracle_ctx* ctx, const float* Tf, const float* v, int64_t ld,

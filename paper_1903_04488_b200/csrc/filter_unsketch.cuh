@@ -61,7 +61,7 @@ struct FilterArgs {
 
 // ---- bit per bucket ------------------------------------------------------------------------------------------
 // One warp per 32 words (1024 buckets) of one row: 32 coalesced loads, a ballot each; lane k keeps ballot k.
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_bitmap_build(const FilterArgs F) {
     pdl_trigger();
     pdl_wait();
@@ -115,7 +115,7 @@ __device__ __forceinline__ float binomial_tail(int r, int need, float p) {
 
 // One thread per folded word: 32 folded bits, each the OR of 2^s consecutive bits of the full bitmap.  The last
 // block to finish turns the density of the folded bitmap into the decision between the two first-pass kernels.
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_bitmap_fold(const FilterArgs F) {
     __shared__ uint32_t s_last;
     pdl_trigger();

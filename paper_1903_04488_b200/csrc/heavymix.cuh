@@ -3,9 +3,14 @@
 //   line 1   l2 = median over rows j of sum_b S[j][b]^2          (k_row_sumsq: fp64 partial sums)
 //   line 2   est_i = median_j s_j(i) S[j][h_j(i)]                 (the same device code as k_unsketch)
 //   line 3   H = { i : est_i^2 >= l2 / k }                        (compared in fp64)
-//   line 4   Top_k = H + a random (k - |H|)-subset of the rest    (k_heavymix_keys writes one 31-bit key per
-//            coordinate: 2^30 + bits(|est_i|)/2 for heavy ones, else a 30-bit priority mixed from (seed, i);
-//            the exact radix select of select.cuh then takes the k largest keys, ties to the smaller index)
+//   line 4   Top_k = H + a random (k - |H|)-subset of the rest    (k_heavymix_keys writes one key per
+//            coordinate: 2^30 for heavy ones, else a 30-bit priority mixed from (seed, i) < 2^30; the exact
+//            radix select of select.cuh then takes the k largest keys, ties to the smaller index: all of H
+//            and the l = k - |H| other coordinates with the largest priorities)
+//            |H| > k (outside the paper's guarantee): the k members of H with the largest |est_i|, ties to
+//            the smaller index.  k_heavymix_rekey and a second selection, enqueued behind the first, run only
+//            in that case (they return at once otherwise): the key becomes the full 31-bit magnitude of a
+//            heavy coordinate's estimate and 0 for the others.
 //   line 5   exact values of Top_k, summed over the workers       (k_gather)
 #pragma once
 #include <stdint.h>
@@ -27,6 +32,7 @@ struct HeavymixArgs {
     HashParams hp; Bucketizer bk;
     HeavymixState* hm;
     float* keys;                // [d] selection keys stored as fp32 bit patterns, 16-byte aligned
+    float* est;                 // [d] the estimates, kept for k_heavymix_rekey, 16-byte aligned
     SelBuffers sb;              // H1 of the keys goes here
     uint32_t k;
     uint64_t fill_seed;
@@ -43,7 +49,7 @@ __device__ __forceinline__ uint32_t fill_priority30(uint64_t seed, uint32_t i) {
 }
 
 // sum of squares of every row; grid.y = row, grid.x strides over the columns
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_row_sumsq(const float* __restrict__ table, int64_t c, HeavymixState* __restrict__ hm) {
     __shared__ double s_part[8];
     const int j = blockIdx.y;
@@ -99,20 +105,24 @@ k_heavymix_keys(const HeavymixArgs A) {
                 rowv[e][j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[e] & P31)), hb[e]);
         }
         uint32_t kv[4];
+        float mv[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const float m = median_of<R>(rowv[e]);
             const bool heavy = (double)m * (double)m >= thr;
-            kv[e] = heavy ? (0x40000000u | (key_of(m) >> 1)) : fill_priority30(A.fill_seed, (uint32_t)(i0 + e));
+            mv[e] = m;
+            kv[e] = heavy ? 0x40000000u : fill_priority30(A.fill_seed, (uint32_t)(i0 + e));
             if (heavy && i0 + e < A.d) ++my_heavy;
         }
         if (i0 + 3 < A.d) {
             *reinterpret_cast<uint4*>(A.keys + i0) = make_uint4(kv[0], kv[1], kv[2], kv[3]);
+            *reinterpret_cast<float4*>(A.est + i0) = make_float4(mv[0], mv[1], mv[2], mv[3]);
 #pragma unroll
             for (int e = 0; e < 4; ++e) atomicAdd(&sh.hist[kv[e] >> H1_SHIFT], 1u);
         } else {
             for (int e = 0; e < 4 && i0 + e < A.d; ++e) {
                 A.keys[i0 + e] = __uint_as_float(kv[e]);
+                A.est[i0 + e] = mv[e];
                 atomicAdd(&sh.hist[kv[e] >> H1_SHIFT], 1u);
             }
         }
@@ -124,8 +134,41 @@ k_heavymix_keys(const HeavymixArgs A) {
     producer_epilogue(A.sb, A.k, sh);
 }
 
+// |H| > k only: keys[i] = magnitude bits of est_i for heavy coordinates, 0 for the others (a heavy coordinate's
+// estimate is non-zero unless l2 = 0, and then every coordinate is heavy), and their first histogram.
+static __global__ void __launch_bounds__(SEL_THREADS)
+k_heavymix_rekey(const HeavymixArgs A, int32_t r, SelBuffers sb2) {
+    __shared__ SelShared sh;
+    __shared__ double s_thr;
+    if (__ldcg(&A.hm->nheavy) <= A.k) return;
+    for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    if (threadIdx.x == 0) {
+        double rows[MAX_R];
+        for (int j = 0; j < r; ++j) rows[j] = A.hm->rowsum[j];
+        for (int p = 1; p < r; ++p) {
+            const double key = rows[p];
+            int q = p - 1;
+            while (q >= 0 && rows[q] > key) { rows[q + 1] = rows[q]; --q; }
+            rows[q + 1] = key;
+        }
+        s_thr = rows[r / 2] / (double)A.k;
+    }
+    __syncthreads();
+    const double thr = s_thr;
+    const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
+    for (int64_t i = (int64_t)blockIdx.x * SEL_THREADS + threadIdx.x; i < A.d; i += stride) {
+        const float m = A.est[i];
+        const uint32_t kv = (double)m * (double)m >= thr ? key_of(m) : 0u;
+        A.keys[i] = __uint_as_float(kv);
+        atomicAdd(&sh.hist[kv >> H1_SHIFT], 1u);
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(sh.hist, sb2.h1);
+    producer_epilogue(sb2, A.k, sh);
+}
+
 // l2 (median of the row sums) and |H| to caller-provided device words
-__global__ void k_heavymix_report(const HeavymixState* __restrict__ hm, int r, double* __restrict__ l2_out,
+static __global__ void k_heavymix_report(const HeavymixState* __restrict__ hm, int r, double* __restrict__ l2_out,
                                   int32_t* __restrict__ nheavy_out) {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     double rows[MAX_R];

@@ -1,0 +1,96 @@
+// launch_unsketch.cu -- instantiations and launches of the kernels that evaluate Algorithm 4's estimate for
+// every coordinate (Algorithm 3 line 9; Algorithm 1 line 2).
+#include "ctx.cuh"
+
+namespace ssgd {
+
+template <int R, bool POW2>
+int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
+    // a few blocks per SM: each block pays one histogram flush
+    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * SSGD_K3_GRID);
+    CU(launch_pdl(st, k_unsketch<R, POW2>, grid, K3_THREADS, 0, A), "launch k_unsketch");
+    LAUNCHED("k_unsketch");
+    return SSGD_OK;
+}
+
+int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_unsketch_t, x, A, st)
+}
+
+// The first pass over all coordinates: the bit-per-bucket filter when the (folded) bitmap fits an SM's shared
+// memory, else the early-exit kernel that reads the table.
+bool use_filter(const ssgd_ctx* x) {
+    return x->prune_mode != SSGD_PRUNE_EARLY_EXIT && x->bm_fold >= 0 &&
+           sizeof(SelShared) + FILTER_QUEUE_BYTES + (size_t)FILTER_MAX_WORDS * 4 <= (size_t)x->max_smem_optin;
+}
+
+template <int R, bool POW2>
+int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
+    CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, A),
+       "launch k_unsketch_sample");
+    LAUNCHED("k_unsketch_sample");
+    const int pruned_grid = grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID);
+    if (use_filter(x)) {
+        FilterArgs F;
+        F.A = A;
+        F.bm_full = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_full);
+        F.bm_fold = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_fold);
+        F.stride_full = x->bm_stride_full; F.stride_fold = x->bm_stride_fold; F.fold = x->bm_fold; F.r = x->r;
+        const int64_t build_tasks = (int64_t)x->r * ((x->bm_stride_full + 31) / 32);
+        CU(launch_pdl(st, k_bitmap_build, grid_for(build_tasks, SEL_WARPS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, F),
+           "launch k_bitmap_build");
+        LAUNCHED("k_bitmap_build");
+        if (F.fold) {
+            CU(launch_pdl(st, k_bitmap_fold, grid_for((int64_t)x->r * F.stride_fold, SEL_THREADS, (int64_t)x->sm_count * 8),
+                          SEL_THREADS, 0, F), "launch k_bitmap_fold");
+            LAUNCHED("k_bitmap_fold");
+        }
+        auto kern = F.fold ? k_unsketch_filter<R, POW2, true> : k_unsketch_filter<R, POW2, false>;
+        const size_t smem = (size_t)x->r * (F.fold ? F.stride_fold : F.stride_full) * 4 + FILTER_QUEUE_BYTES;
+        if (!x->filter_ready) {
+            CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)((size_t)FILTER_MAX_WORDS * 4 + FILTER_QUEUE_BYTES)), "smem attribute");
+            x->filter_ready = true;
+        }
+        CU(launch_pdl(st, kern, grid_for(A.d, FILTER_THREADS, (int64_t)x->sm_count), FILTER_THREADS, smem, F),
+           "launch k_unsketch_filter");
+        LAUNCHED("k_unsketch_filter");
+        if (F.fold) {                                    // runs only if the folded bitmap turned out too dense
+            SparseArgs G = A;
+            G.gated = 1;
+            // plain stream order, no programmatic launch: measured on B200, blocks of this kernel that become
+            // resident while the declining filter kernel drains cost 4 ms (d = 9e7)
+            k_unsketch_pruned<R, POW2><<<pruned_grid, SEL_THREADS, 0, st>>>(G);
+            LAUNCHED("k_unsketch_pruned");
+        }
+    } else {
+        CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, A), "launch k_unsketch_pruned");
+        LAUNCHED("k_unsketch_pruned");
+    }
+    SparseArgs B = A;
+    B.rerun = 1;                                         // returns at once unless the first pass kept too few
+    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, B), "launch k_unsketch_pruned (unpruned rerun)");
+    LAUNCHED("k_unsketch_pruned");
+    return SSGD_OK;
+}
+
+int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_sparse_t, x, A, st)
+}
+
+template <int R, bool POW2>
+int launch_heavymix_keys_t(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
+    const int64_t groups = (A.d + 3) / 4;
+    k_heavymix_keys<R, POW2><<<grid_for(groups, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, st>>>(A);
+    LAUNCHED("k_heavymix_keys");
+    return SSGD_OK;
+}
+
+int launch_heavymix_keys(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
+    DISPATCH_R(launch_heavymix_keys_t, x, A, st)
+}
+
+}  // namespace ssgd

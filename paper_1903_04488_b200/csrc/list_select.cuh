@@ -28,7 +28,7 @@ constexpr int MAP_CHUNK_WORDS = SEL_THREADS * 8;       // map words per block in
 #ifdef __CUDACC__
 
 // ---- histogram pass over the list; its last block publishes T and Q --------------------------------------
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_list_hist(SparseBuffers sp) {
     __shared__ SelShared sh;
     pdl_trigger();
@@ -66,7 +66,7 @@ k_list_hist(SparseBuffers sp) {
 // Every list item is a distinct coordinate, so the marks a chunk of the maps receives can be counted here, one
 // atomic per marked item on the chunk's counter (zeroed with the maps); the last block turns the counts into
 // exclusive offsets for k_map_emit.
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_list_mark(SparseBuffers sp, int64_t nchunks) {
     __shared__ SelShared sh;
     // chunk counters are hot addresses (a few hundred of them for 1e5 marks): count in shared memory first
@@ -134,7 +134,7 @@ struct EmitSecondRound {
     int64_t pending_words;
 };
 
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_map_emit(SparseBuffers sp, int64_t nwords, int64_t nchunks, uint32_t m, int32_t* __restrict__ cand_idx,
            EmitSecondRound E) {
     __shared__ SelShared sh;

@@ -54,11 +54,16 @@ struct SelBuffers {
     uint32_t* chunk_gt;  // [nchunks] counts, then exclusive offsets
     uint32_t* chunk_eq;  // [nchunks]
     uint32_t* h19;       // [H19_BINS] zeroed, or NULL: with it, k_sel_pass23 replaces k_sel_pass2 + k_sel_pass3
+    // optional gate: if not NULL, the selection's kernels do nothing unless *gate > gate_above (a selection that is
+    // enqueued unconditionally but needed only in a case the device decides)
+    const uint32_t* gate;
+    uint32_t gate_above;
 };
 
 #ifdef __CUDACC__
 
 __device__ __forceinline__ uint32_t key_of(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+__device__ __forceinline__ bool sel_gated_off(const SelBuffers& sb) { return sb.gate && __ldcg(sb.gate) <= sb.gate_above; }
 
 // Histogram passes load SEL_BATCH items per thread before touching shared memory, so that a pass costs a few
 // L2 round trips instead of one per item (the shared-memory atomics keep the compiler from hoisting loads).
@@ -145,7 +150,7 @@ __device__ __forceinline__ void flush_hist(const uint32_t* s_hist, uint32_t* __r
 }
 
 // ---- pass 2: H2 over items whose top digit equals the threshold digit -----------------------------
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ SelShared sh;
     pdl_trigger();
@@ -171,7 +176,7 @@ k_sel_pass2(const float* __restrict__ val, int64_t n, SelBuffers sb) {
 }
 
 // ---- pass 3: H3 over items matching the 23-bit prefix; its last block publishes T and Q -----------
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ SelShared sh;
     pdl_trigger();
@@ -204,12 +209,13 @@ k_sel_pass3(const float* __restrict__ val, int64_t n, SelBuffers sb) {
 // the first digit in a 2^19-bin table in global memory (few items: the first digit has already cut the input
 // down to one bin in 4096).  The last block finds the second digit in H2 and the third among the 256 bins of the
 // big table under it: the exact threshold key T and the tie quota Q.
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_sel_pass23(const float* __restrict__ val, int64_t n, SelBuffers sb) {
     __shared__ SelShared sh;
     pdl_trigger();
     for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
+    if (sel_gated_off(sb)) return;
     const uint32_t d1 = sb.state->d1;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
@@ -319,6 +325,7 @@ k_sel_count(const float* __restrict__ val, int64_t n, SelBuffers sb, int64_t nch
     __shared__ SelShared sh;
     pdl_trigger();
     pdl_wait();
+    if (sel_gated_off(sb)) return;
     const uint32_t T = sb.state->thr_key;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {
@@ -345,6 +352,7 @@ __device__ __forceinline__ void sel_emit_chunks(const float* __restrict__ val, i
     __shared__ uint32_t s_wg[SEL_WARPS], s_we[SEL_WARPS];
     pdl_trigger();
     pdl_wait();
+    if (sel_gated_off(sb)) return;
     const uint32_t T = sb.state->thr_key, Q = sb.state->quota_eq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int64_t chunk = blockIdx.x; chunk < nchunks; chunk += gridDim.x) {

@@ -7,7 +7,6 @@
 //                       dense), k_gather (line 10), k_emit_candidates / k_emit_final, k_zero and
 //                       k_flush_pending (line 13, eager and deferred), k_hashes
 //   accum_tma.cuh       k_accum_insert_tma: lines 5-7 as a bulk-copy (TMA) + mbarrier pipeline
-//   accum_ws.cuh        k_accum_insert_ws: the same pipeline with separate stream and sketch warps
 //   filter_unsketch.cuh k_bitmap_build, k_bitmap_fold, k_unsketch_filter: line 9 decided per coordinate on a
 //                       one-bit-per-bucket copy of the table in shared memory
 //   sparse_select.cuh   k_unsketch_sample, k_unsketch_pruned: the sampled threshold; line 9 with early exit on
@@ -17,6 +16,8 @@
 //                       (lines 9, 11)
 //   heavymix.cuh        k_row_sumsq, k_heavymix_keys: Algorithm 1
 //   hash.cuh, estimate.cuh   the hash family and the median-of-r estimate
+// The kernels instantiated per (rows, power-of-two columns) are launched from launch_accum.cu and
+// launch_unsketch.cu; ctx.cuh holds what the units share.
 // HBM-bound work is the accumulate+insert kernel (20 bytes per worker-coordinate); nothing here is a dense
 // contraction, so there are no tensor-core instructions.
 #include <cuda_bf16.h>
@@ -32,65 +33,14 @@
 #include <new>
 #include <string>
 
-#include "../../include/ssgd.h"
-#include "hash.cuh"
-#include "select.cuh"
-#include "accum_tma.cuh"
-#include "accum_ws.cuh"
-#include "estimate.cuh"
-#include "sparse_select.cuh"
-#include "filter_unsketch.cuh"
+#include "ctx.cuh"
 #include "list_select.cuh"
-#include "heavymix.cuh"
-#include "step_kernels.cuh"
 
 
 // ==================================================================================================
 // host side: context, argument checks, launch plans
 // ==================================================================================================
 using namespace ssgd;
-
-struct ssgd_ctx {
-    int64_t d, c, k;
-    int32_t r, W;
-    uint64_t seed;
-    HashParams hp;
-    Bucketizer bk;
-    bool pow2;
-    int32_t insert_mode;
-    // binding
-    float* u; float* v; int64_t ld;
-    char* ws; size_t ws_bytes; int64_t ncand_max;
-    // workspace layout (byte offsets)
-    size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
-    size_t off_sp_hist, off_sp_state, off_maps, off_map_chunks, off_list_idx, off_list_est;   // early-exit path
-    size_t map_bytes;
-    int64_t list_cap, nchunk_map;
-    size_t off_bm_full, off_bm_fold;                       // bit-per-bucket filter (filter_unsketch.cuh)
-    int32_t bm_stride_full, bm_stride_fold, bm_fold;       // bm_fold < 0: the bitmap cannot be folded into shared memory
-    bool filter_ready;                                     // shared-memory attribute of the filter kernel set
-    uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
-    size_t off_pending;     // d-bit map of the deferred zero-out; survives from step to step
-    int32_t zero_mode;      // SSGD_ZERO_DEFERRED / SSGD_ZERO_EAGER
-    bool pending_dirty;     // a deferred ssgd_step has run since the last flush: u, v may await their zero-out
-    size_t off_hm;
-    int32_t prune_mode;
-    size_t persist_bytes;
-    size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel   // > 0: launches that touch the table carry an L2 access-policy window of this size
-    size_t off_xsum;        // per-coordinate sums over the workers of the new v, written by ssgd_step's accumulate kernel
-    size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
-    int64_t nchunk_c, nchunk_f;
-    // device facts
-    int device; int sm_count; int max_smem_optin;
-    int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
-    int ws_blocks_per_sm;   // same for the warp-specialised kernel
-    int64_t launches;
-    // optional per-stage timing of ssgd_step (CUDA events on the caller's stream)
-    bool timing;
-    cudaEvent_t* ev;        // [TIMING_SLOTS][SSGD_NSTAGES + 1]
-    int32_t ev_steps;       // steps recorded since the last collection
-    std::string last_error;
-};
 
 namespace {
 
@@ -171,26 +121,6 @@ SelBuffers sel_buffers(ssgd_ctx* x, bool final_stage) {
     return sb;
 }
 
-inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-int cuda_fail(ssgd_ctx* x, cudaError_t e, const char* what) {
-    x->last_error = std::string(what) + ": " + cudaGetErrorString(e);
-    return SSGD_ECUDA;
-}
-
-#define CU(call, what)                                                   \
-    do {                                                                 \
-        cudaError_t e_ = (call);                                         \
-        if (e_ != cudaSuccess) return cuda_fail(x, e_, what);            \
-    } while (0)
-
-#define LAUNCHED(what)                                                   \
-    do {                                                                 \
-        x->launches++;                                                   \
-        cudaError_t e_ = cudaGetLastError();                             \
-        if (e_ != cudaSuccess) return cuda_fail(x, e_, what);            \
-    } while (0)
-
 int ensure_device(ssgd_ctx* x) {
     if (x->device >= 0) return SSGD_OK;
     int dev = 0;
@@ -199,189 +129,6 @@ int ensure_device(ssgd_ctx* x) {
     CU(cudaDeviceGetAttribute(&x->max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev), "smem optin");
     x->device = dev;
     return SSGD_OK;
-}
-
-// Launch with programmatic stream serialization: the kernel may become resident while its predecessor
-// drains; it orders itself with pdl_wait().  SSGD_NO_PDL=1 in the environment turns the attribute off.
-bool pdl_enabled() {
-    static const bool on = [] { const char* e = std::getenv("SSGD_NO_PDL"); return !(e && e[0] == '1'); }();
-    return on;
-}
-
-// An L2 access-policy window for one launch: accesses inside [base, base+bytes) are kept (persisting),
-// everything else the kernel touches is treated as streaming.
-struct L2Window { const void* base; size_t bytes; };
-
-template <typename... P, typename... A>
-cudaError_t launch_pdl_w(cudaStream_t st, L2Window win, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3((unsigned)block);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute at[2];
-    int n = 0;
-    if (pdl_enabled()) {
-        at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[n].val.programmaticStreamSerializationAllowed = 1;
-        ++n;
-    }
-    if (win.base && win.bytes) {
-        at[n].id = cudaLaunchAttributeAccessPolicyWindow;
-        at[n].val.accessPolicyWindow.base_ptr = const_cast<void*>(win.base);
-        at[n].val.accessPolicyWindow.num_bytes = win.bytes;
-        at[n].val.accessPolicyWindow.hitRatio = 1.0f;
-        at[n].val.accessPolicyWindow.hitProp = cudaAccessPropertyPersisting;
-        at[n].val.accessPolicyWindow.missProp = cudaAccessPropertyStreaming;
-        ++n;
-    }
-    cfg.attrs = at;
-    cfg.numAttrs = n;
-    return cudaLaunchKernelEx(&cfg, kern, P(args)...);
-}
-
-template <typename... P, typename... A>
-cudaError_t launch_pdl(cudaStream_t st, void (*kern)(P...), int grid, int block, size_t smem, A... args) {
-    return launch_pdl_w(st, L2Window{nullptr, 0}, kern, grid, block, smem, args...);
-}
-
-inline int grid_for(int64_t items, int threads, int64_t cap) {
-    int64_t b = (items + threads - 1) / threads;
-    if (b < 1) b = 1;
-    if (b > cap) b = cap;
-    return (int)b;
-}
-
-// ---- K1 dispatch over (R, POW2, MODE) ------------------------------------------------------------
-template <int R, bool POW2, int MODE>
-int launch_accum_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
-    const int64_t groups = (A.d + 3) / 4;
-    if (MODE == INS_MERGED_SMEM) {
-        const size_t smem = (size_t)R * A.c * 4;
-        CU(cudaFuncSetAttribute(k_accum_insert<R, POW2, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)smem), "smem attribute");
-        const int grid = grid_for(groups, K1_THREADS, x->sm_count);
-        k_accum_insert<R, POW2, MODE><<<grid, K1_THREADS, smem, st>>>(A);
-    } else {
-        const int grid = grid_for(groups, K1_THREADS, (int64_t)1 << 30);
-        bool few = false;
-        if constexpr (MODE == INS_MERGED_GLOBAL) {
-            if (A.W <= K1_UNROLL_FEW) {
-                few = true;
-                CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, k_accum_insert<R, POW2, MODE, K1_UNROLL_FEW>, grid,
-                                K1_THREADS, 0, A), "launch k_accum_insert");
-            }
-        }
-        if (!few)
-            CU(launch_pdl_w(st, L2Window{MODE == INS_MERGED_GLOBAL ? A.table : nullptr, x->persist_bytes},
-                            k_accum_insert<R, POW2, MODE>, grid, K1_THREADS, 0, A), "launch k_accum_insert");
-    }
-    LAUNCHED("k_accum_insert");
-    return SSGD_OK;
-}
-
-template <int R, bool POW2>
-int launch_accum_m(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
-    switch (mode) {
-        case INS_MERGED_GLOBAL: return launch_accum_t<R, POW2, INS_MERGED_GLOBAL>(x, A, st);
-        case INS_PER_WORKER: return launch_accum_t<R, POW2, INS_PER_WORKER>(x, A, st);
-        default: return launch_accum_t<R, POW2, INS_MERGED_SMEM>(x, A, st);
-    }
-}
-
-// -DSSGD_TUNE_ONLY_R5 instantiates the r = 5, power-of-two-c kernels only (quick builds while tuning)
-#ifdef SSGD_TUNE_ONLY_R5
-#define DISPATCH_R(fn, ...)                                                       \
-    if (x->r == 5 && x->pow2) return fn<5, true>(__VA_ARGS__);                    \
-    return SSGD_EINVAL;
-#else
-#define DISPATCH_R(fn, ...)                                                       \
-    switch (x->r) {                                                               \
-        case 1: return x->pow2 ? fn<1, true>(__VA_ARGS__) : fn<1, false>(__VA_ARGS__);    \
-        case 3: return x->pow2 ? fn<3, true>(__VA_ARGS__) : fn<3, false>(__VA_ARGS__);    \
-        case 5: return x->pow2 ? fn<5, true>(__VA_ARGS__) : fn<5, false>(__VA_ARGS__);    \
-        case 7: return x->pow2 ? fn<7, true>(__VA_ARGS__) : fn<7, false>(__VA_ARGS__);    \
-        case 9: return x->pow2 ? fn<9, true>(__VA_ARGS__) : fn<9, false>(__VA_ARGS__);    \
-        case 11: return x->pow2 ? fn<11, true>(__VA_ARGS__) : fn<11, false>(__VA_ARGS__); \
-        case 13: return x->pow2 ? fn<13, true>(__VA_ARGS__) : fn<13, false>(__VA_ARGS__); \
-        case 15: return x->pow2 ? fn<15, true>(__VA_ARGS__) : fn<15, false>(__VA_ARGS__); \
-        default: return SSGD_EINVAL;                                              \
-    }
-#endif
-
-int launch_accum(ssgd_ctx* x, const AccumArgs& A, int mode, cudaStream_t st) {
-    DISPATCH_R(launch_accum_m, x, A, mode, st)
-}
-
-template <int R, bool POW2>
-int launch_accum_tma_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
-    auto kern = k_accum_insert_tma<R, POW2>;
-    const size_t smem = sizeof(KtShared);
-    if (x->kt_blocks_per_sm == 0) {
-        CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "smem attribute");
-        int nb = 0;
-        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, KT_THREADS, smem), "occupancy query");
-        x->kt_blocks_per_sm = nb < 1 ? 1 : nb;
-    }
-    const int64_t ntiles = ((A.d & ~(int64_t)3) + KT_TC - 1) / KT_TC;
-    const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->kt_blocks_per_sm);
-    CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, kern, grid, KT_THREADS, smem, A,
-                    reinterpret_cast<int32_t*>(x->ws + x->off_err)), "launch k_accum_insert_tma");
-    LAUNCHED("k_accum_insert_tma");
-    return SSGD_OK;
-}
-
-int launch_accum_tma(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
-    DISPATCH_R(launch_accum_tma_t, x, A, st)
-}
-
-template <int R, bool POW2>
-int launch_insert_rows_t(ssgd_ctx* x, const float* xsum, float* table, int lo, int hi, cudaStream_t st) {
-    const int64_t groups = (x->d + 3) / 4;
-    CU(launch_pdl(st, k_insert_rows<R, POW2>, grid_for(groups, 256, (int64_t)x->sm_count * 8), 256, 0, xsum, x->d, table, x->c,
-                  x->hp, x->bk, lo, hi), "launch k_insert_rows");
-    LAUNCHED("k_insert_rows");
-    return SSGD_OK;
-}
-
-int launch_insert_rows(ssgd_ctx* x, const float* xsum, float* table, int lo, int hi, cudaStream_t st) {
-    DISPATCH_R(launch_insert_rows_t, x, xsum, table, lo, hi, st)
-}
-
-template <int R, bool POW2>
-int launch_accum_ws_t(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
-    auto kern = k_accum_insert_ws<R, POW2>;
-    const size_t smem = sizeof(WsShared);
-    if (x->ws_blocks_per_sm == 0) {
-        CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem), "smem attribute");
-        int nb = 0;
-        CU(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kern, WS_THREADS, smem), "occupancy query");
-        x->ws_blocks_per_sm = nb < 1 ? 1 : nb;
-    }
-    const int64_t ntiles = ((A.d & ~(int64_t)3) + WS_TC - 1) / WS_TC;
-    const int grid = grid_for(ntiles, 1, (int64_t)x->sm_count * x->ws_blocks_per_sm);
-    CU(launch_pdl_w(st, L2Window{A.table, x->persist_bytes}, kern, grid, WS_THREADS, smem, A,
-                    reinterpret_cast<int32_t*>(x->ws + x->off_err)), "launch k_accum_insert_ws");
-    LAUNCHED("k_accum_insert_ws");
-    return SSGD_OK;
-}
-
-int launch_accum_ws(ssgd_ctx* x, const AccumArgs& A, cudaStream_t st) {
-    DISPATCH_R(launch_accum_ws_t, x, A, st)
-}
-
-template <int R, bool POW2>
-int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
-    const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
-    // a few blocks per SM: each block pays one histogram flush
-    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * SSGD_K3_GRID);
-    CU(launch_pdl(st, k_unsketch<R, POW2>, grid, K3_THREADS, 0, A), "launch k_unsketch");
-    LAUNCHED("k_unsketch");
-    return SSGD_OK;
-}
-
-int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
-    DISPATCH_R(launch_unsketch_t, x, A, st)
 }
 
 // Radix-select passes after the producer filled H1: leaves thresholds in sb.state and exclusive
@@ -471,68 +218,6 @@ bool use_sparse(const ssgd_ctx* x, int64_t ncand) {
     return x->bm_fold == 0 || (x->r >= 5 && x->r <= 9);
 }
 
-// The first pass over all coordinates: the bit-per-bucket filter when the (folded) bitmap fits an SM's shared
-// memory, else the early-exit kernel that reads the table.
-bool use_filter(const ssgd_ctx* x) {
-    return x->prune_mode != SSGD_PRUNE_EARLY_EXIT && x->bm_fold >= 0 &&
-           sizeof(SelShared) + FILTER_QUEUE_BYTES + (size_t)FILTER_MAX_WORDS * 4 <= (size_t)x->max_smem_optin;
-}
-
-template <int R, bool POW2>
-int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
-    const int64_t groups = (A.d + 3) / 4;
-    const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
-    CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, A),
-       "launch k_unsketch_sample");
-    LAUNCHED("k_unsketch_sample");
-    const int pruned_grid = grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID);
-    if (use_filter(x)) {
-        FilterArgs F;
-        F.A = A;
-        F.bm_full = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_full);
-        F.bm_fold = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_fold);
-        F.stride_full = x->bm_stride_full; F.stride_fold = x->bm_stride_fold; F.fold = x->bm_fold; F.r = x->r;
-        const int64_t build_tasks = (int64_t)x->r * ((x->bm_stride_full + 31) / 32);
-        CU(launch_pdl(st, k_bitmap_build, grid_for(build_tasks, SEL_WARPS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, F),
-           "launch k_bitmap_build");
-        LAUNCHED("k_bitmap_build");
-        if (F.fold) {
-            CU(launch_pdl(st, k_bitmap_fold, grid_for((int64_t)x->r * F.stride_fold, SEL_THREADS, (int64_t)x->sm_count * 8),
-                          SEL_THREADS, 0, F), "launch k_bitmap_fold");
-            LAUNCHED("k_bitmap_fold");
-        }
-        auto kern = F.fold ? k_unsketch_filter<R, POW2, true> : k_unsketch_filter<R, POW2, false>;
-        const size_t smem = (size_t)x->r * (F.fold ? F.stride_fold : F.stride_full) * 4 + FILTER_QUEUE_BYTES;
-        if (!x->filter_ready) {
-            CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    (int)((size_t)FILTER_MAX_WORDS * 4 + FILTER_QUEUE_BYTES)), "smem attribute");
-            x->filter_ready = true;
-        }
-        CU(launch_pdl(st, kern, grid_for(A.d, FILTER_THREADS, (int64_t)x->sm_count), FILTER_THREADS, smem, F),
-           "launch k_unsketch_filter");
-        LAUNCHED("k_unsketch_filter");
-        if (F.fold) {                                    // runs only if the folded bitmap turned out too dense
-            SparseArgs G = A;
-            G.gated = 1;
-            // plain stream order, no programmatic launch: measured on B200, blocks of this kernel that become
-            // resident while the declining filter kernel drains cost 4 ms (d = 9e7)
-            k_unsketch_pruned<R, POW2><<<pruned_grid, SEL_THREADS, 0, st>>>(G);
-            LAUNCHED("k_unsketch_pruned");
-        }
-    } else {
-        CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, A), "launch k_unsketch_pruned");
-        LAUNCHED("k_unsketch_pruned");
-    }
-    SparseArgs B = A;
-    B.rerun = 1;                                         // returns at once unless the first pass kept too few
-    CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, B), "launch k_unsketch_pruned (unpruned rerun)");
-    LAUNCHED("k_unsketch_pruned");
-    return SSGD_OK;
-}
-
-int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
-    DISPATCH_R(launch_sparse_t, x, A, st)
-}
 
 // Line 9 with early exit: sample -> pruned unsketch (-> unpruned rerun if the sample misjudged) -> selection on
 // the survivor list (list_select.cuh).
@@ -630,24 +315,11 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
     if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
     if (x->insert_mode == SSGD_INSERT_TMA) return INS_MERGED_TMA;
-    if (x->insert_mode == SSGD_INSERT_WS) return INS_MERGED_WS;
     // measured on B200: the bulk-copy pipeline wins once a tile's walk over the workers is long
     // (W = 128: 5.73 vs 5.43 TB/s), plain loads win for short walks (W = 16: 4.93 vs 4.83 TB/s)
     // measured at C2's d (plain / bulk-copy, TB/s): W = 32 5.98 / 5.36; 96 5.79 / 5.64; 128 5.72 / 5.69; 192 5.53 / 5.71;
     // 256 5.43 / 5.70 -- the plain kernel's threads loop over the workers 16 at a time, and loop less well than they start
     return x->W > 128 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
-}
-
-template <int R, bool POW2>
-int launch_heavymix_keys_t(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
-    const int64_t groups = (A.d + 3) / 4;
-    k_heavymix_keys<R, POW2><<<grid_for(groups, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, st>>>(A);
-    LAUNCHED("k_heavymix_keys");
-    return SSGD_OK;
-}
-
-int launch_heavymix_keys(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st) {
-    DISPATCH_R(launch_heavymix_keys_t, x, A, st)
 }
 
 }  // namespace
@@ -670,7 +342,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->pow2 = (c & (c - 1)) == 0;
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
-    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0; x->ws_blocks_per_sm = 0;
+    x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
     x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
@@ -756,7 +428,7 @@ int ssgd_step_used_fallback(ssgd_ctx* x, void* stream, int32_t* out) {
 }
 
 int ssgd_set_insert_mode(ssgd_ctx* x, int32_t mode) {
-    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_WS) return SSGD_EINVAL;
+    if (!x || mode < SSGD_INSERT_AUTO || mode > SSGD_INSERT_TMA) return SSGD_EINVAL;
     x->insert_mode = mode;
     return SSGD_OK;
 }
@@ -889,8 +561,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     A.xsum = reinterpret_cast<float*>(x->ws + x->off_xsum);   // the second round reads these instead of W values of v
     if (split) A.rows_here = rows_fit;
     if ((e = mark(x, 0, st))) return e;
-    if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st)
-             : mode == INS_MERGED_WS ? launch_accum_ws(x, A, st) : launch_accum(x, A, mode, st))) return e;
+    if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st) : launch_accum(x, A, mode, st))) return e;
     if (split)
         for (int lo = rows_fit; lo < x->r; lo += rows_fit)
             if ((e = launch_insert_rows(x, A.xsum, merged, lo, lo + rows_fit < x->r ? lo + rows_fit : x->r, st))) return e;
@@ -967,6 +638,7 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     A.table = merged; A.c = x->c; A.d = x->d; A.r = x->r; A.hp = x->hp; A.bk = x->bk;
     A.hm = reinterpret_cast<HeavymixState*>(x->ws + x->off_hm);
     A.keys = reinterpret_cast<float*>(x->ws + x->off_est);
+    A.est = reinterpret_cast<float*>(x->ws + x->off_list_est);   // the survivor list's room: d floats
     A.sb = sel_buffers(x, false);
     A.k = (uint32_t)x->k;
     A.fill_seed = fill_seed;
@@ -977,6 +649,18 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     if ((e = launch_select(x, A.keys, x->d, A.sb, x->nchunk_c, st, false))) return e;
     CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)A.keys,
                   x->d, A.sb, out_idx, (float*)nullptr, (uint32_t)x->k, x->nchunk_c), "launch k_emit_candidates");
+    LAUNCHED("k_emit_candidates");
+    // |H| > k (decided on the device): a second selection among the heavy coordinates on their full magnitudes
+    // overwrites out_idx; its kernels return at once otherwise.  It uses the final stage's histograms and state
+    // and, once the first selection is done with them, the candidate stage's chunk counters.
+    SelBuffers sb2 = sel_buffers(x, true);
+    sb2.chunk_gt = A.sb.chunk_gt; sb2.chunk_eq = A.sb.chunk_eq;
+    sb2.gate = &A.hm->nheavy; sb2.gate_above = (uint32_t)x->k;
+    k_heavymix_rekey<<<grid_for(x->d, SEL_THREADS * 4, (int64_t)x->sm_count * 8), SEL_THREADS, 0, st>>>(A, x->r, sb2);
+    LAUNCHED("k_heavymix_rekey");
+    if ((e = launch_select(x, A.keys, x->d, sb2, x->nchunk_c, st, false))) return e;
+    CU(launch_pdl(st, k_emit_candidates, grid_for(x->nchunk_c, 1, (int64_t)x->sm_count * 8), SEL_THREADS, 0, (const float*)A.keys,
+                  x->d, sb2, out_idx, (float*)nullptr, (uint32_t)x->k, x->nchunk_c), "launch k_emit_candidates");
     LAUNCHED("k_emit_candidates");
     // line 5: exact values of the chosen coordinates, summed over the workers
     SelBuffers sf = sel_buffers(x, true);

@@ -35,7 +35,7 @@ namespace ssgd {
 // pipeline of accum_tma.cuh; this form serves the per-worker tables of ssgd_sketch_accumulate and the
 // shared-memory table variant.
 // ------------------------------------------------------------------------------------------------
-enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3, INS_MERGED_WS = 4 };
+enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
 
 #ifndef SSGD_K1_UNROLL
 #define SSGD_K1_UNROLL 16
@@ -222,7 +222,7 @@ k_insert_rows(const float* __restrict__ xsum, int64_t d, float* __restrict__ tab
 // ------------------------------------------------------------------------------------------------
 // K2: merge of the per-worker tables, worker order
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_merge(const float* __restrict__ tables, float* __restrict__ merged, int64_t rc, int32_t W) {
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
     const int64_t t0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -267,14 +267,14 @@ __device__ __forceinline__ float dequant16(uint16_t h, int fmt) {
     return fmt == 0 ? __half2float(__ushort_as_half(h)) : __bfloat162float(__ushort_as_bfloat16(h));
 }
 
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_quantize16(const float* __restrict__ x, uint16_t* __restrict__ q, int64_t n, int fmt) {
     const int64_t stride = (int64_t)gridDim.x * 256;
     for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < n; t += stride) q[t] = quant16(__ldcs(x + t), fmt);
 }
 
 // merged[t] = sum over w = 0..W-1 (that order, fp32) of the decoded q[w][t]
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_merge16(const uint16_t* __restrict__ q, float* __restrict__ merged, int64_t n, int32_t W, int fmt) {
     const int64_t stride = (int64_t)gridDim.x * 256;
     for (int64_t t = (int64_t)blockIdx.x * 256 + threadIdx.x; t < n; t += stride) {
@@ -344,7 +344,7 @@ k_unsketch(const UnsketchArgs A) {
 // ------------------------------------------------------------------------------------------------
 // candidate emit (line 9, second half)
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(SEL_THREADS)
+static __global__ void __launch_bounds__(SEL_THREADS)
 k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32_t* __restrict__ cand_idx,
                   float* __restrict__ cand_est, uint32_t cap, int64_t nchunks) {
     sel_emit_chunks<SEL_ITEMS>(est, d, sb, nchunks, [&](uint32_t slot, int64_t i) {
@@ -362,7 +362,7 @@ k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32
 #endif
 constexpr int GATHER_UNROLL = SSGD_GATHER_UNROLL;   // scattered loads in flight per thread
 
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ v, int64_t ld, int32_t W,
          int64_t d, float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag,
          uint32_t* __restrict__ pending_clear, int64_t pending_words) {
@@ -406,7 +406,7 @@ k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restric
 // Line 10 inside ssgd_step: the accumulate kernel has already summed every coordinate's new v over the workers
 // (fp64, worker order, rounded once) on its way to the sketch, so the second round's exact sum of a candidate is
 // one read of that array instead of W scattered reads of v.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_gather_sums(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ xsum, int64_t d,
               float* __restrict__ xs, SelBuffers sb, uint32_t want, int32_t* __restrict__ errflag,
               uint32_t* __restrict__ pending_clear, int64_t pending_words) {
@@ -452,7 +452,7 @@ k_emit_final(const float* __restrict__ xs, int64_t ncand, SelBuffers sb, const i
 // The deferred form of line 13: the chosen coordinates are marked in a d-bit map, and the next step's
 // accumulate kernel, which reads every u and v anyway, treats marked coordinates as zero.  This kernel applies
 // the map to memory for callers that read u or v in between: one thread per map word.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_flush_pending(uint32_t* __restrict__ pending, int64_t nwords, float* __restrict__ u, float* __restrict__ v,
                 int64_t ld, int32_t W, int64_t d) {
     pdl_trigger();
@@ -471,7 +471,7 @@ k_flush_pending(uint32_t* __restrict__ pending, int64_t nwords, float* __restric
     }
 }
 
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
 k_zero(const int32_t* __restrict__ out_idx, int64_t k, float* __restrict__ u, float* __restrict__ v,
        int64_t ld, int32_t W, int64_t d) {
     pdl_trigger();

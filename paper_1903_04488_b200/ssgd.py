@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libssgd.so")
 
 OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_NCAND = 262144
-INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA, INSERT_WS = 0, 1, 2, 3, 4
+INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT = 0, 1, 2, 3
 ZERO_DEFERRED, ZERO_EAGER = 0, 1
 FMT_F16, FMT_BF16 = 0, 1

@@ -82,3 +82,41 @@ def test_heavymix_on_the_step_table(cuda_device):
     assert (out_idx.cpu().numpy() == want["out_idx"]).all()
     assert (out_val.cpu().numpy() == want["out_val"]).all()
     assert set(st.planted_idx.cpu().tolist()) <= set(want["out_idx"].tolist())
+
+
+@pytest.mark.parametrize("d,k", [(200, 20), (200, 150), (100_003, 777), (100_003, 60_000)])
+def test_heavymix_more_heavy_than_k_compares_full_magnitudes(cuda_device, d, k):
+    """|H| > k (outside the paper's guarantee): one row, four buckets holding +-1.0 and +-(the next fp32 above
+    1.0), so every coordinate is heavy and the magnitudes differ in the last mantissa bit only.  The k kept are
+    the k largest under the full fp32 magnitude, ties to the smaller index -- the oracle's explicit branch."""
+    dev = cuda_device
+    one = np.float32(1.0)
+    up = np.nextafter(one, np.float32(2.0))
+    Tf = np.array([[one, up, -one, -up]], np.float32)
+    eng = S.Ssgd(d, 1, 4, k, 2, 21)
+    orc = Oracle(d, 1, 4, k, 2, 21)
+    ld = (d + 3) // 4 * 4
+    gen = torch.Generator(device=dev).manual_seed(d + k)
+    v = torch.zeros((2, ld), device=dev)
+    v[:, :d] = torch.randn((2, d), generator=gen, device=dev)
+    u = torch.zeros_like(v)
+    eng.bind(u, v, k)
+    out_idx = torch.full((k,), -1, dtype=torch.int32, device=dev)
+    out_val = torch.empty(k, device=dev)
+    nheavy = torch.zeros(1, dtype=torch.int32, device=dev)
+    v_h = v.cpu().numpy()
+    for seed in (3, 4):
+        want = orc.heavymix(Tf, v_h, seed)
+        eng.heavymix(torch.tensor(Tf, device=dev), seed, out_idx, out_val, None, nheavy)
+        assert eng.status() == S.OK
+        assert nheavy.item() == want["nheavy"] == d
+        assert (out_idx.cpu().numpy() == want["out_idx"]).all()
+        assert (out_val.cpu().numpy().view(np.uint32) == want["out_val"].view(np.uint32)).all()
+    assert want["out_idx"].tolist() != list(range(k))       # a key without the last mantissa bit would give this
+    # the same context, a table with |H| <= k next: the gated second selection must stay out of the way
+    Tf2 = np.array([[50.0, 0.25, -0.25, 0.125]], np.float32)
+    want = orc.heavymix(Tf2, v_h, 9)
+    if want["nheavy"] <= k:
+        eng.heavymix(torch.tensor(Tf2, device=dev), 9, out_idx, out_val, None, nheavy)
+        assert eng.status() == S.OK and nheavy.item() == want["nheavy"]
+        assert (out_idx.cpu().numpy() == want["out_idx"]).all()

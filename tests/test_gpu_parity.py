@@ -159,7 +159,7 @@ STEP_CASES = [
 
 
 @pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
-@pytest.mark.parametrize("mode", [S.INSERT_WS, S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
+@pytest.mark.parametrize("mode", [S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
 def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
     if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
@@ -457,7 +457,7 @@ def test_stored_small_case_is_reproduced_exactly(cuda_device):
     want = json.load(open(os.path.join(here, "golden", "oracle_small_case.json")))
     sh = want["shape"]
     dev = cuda_device
-    for mode in (S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_SMEM):
+    for mode in (S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_SMEM):
         eng = S.Ssgd(sh["d"], sh["r"], sh["c"], sh["k"], sh["W"], sh["seed"])
         assert eng.get_hash_params().tolist() == want["hash_params"]
         ld = (sh["d"] + 3) // 4 * 4
@@ -535,7 +535,7 @@ def _random_case(seed):
     ncand = int(rng.integers(1, d + 1))
     k = int(rng.integers(1, ncand + 1))
     prune = int(rng.choice([S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_AUTO]))
-    mode = int(rng.choice([S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_AUTO]))
+    mode = int(rng.choice([S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_AUTO]))
     zero = int(rng.choice([S.ZERO_DEFERRED, S.ZERO_EAGER]))
     cfg = base.scaled(name=f"rnd{seed}", d=d, W=W, r=r, c=c, ncand=ncand, k=k, base_seed=1000 + seed)
     return cfg, prune, mode, zero
@@ -557,7 +557,7 @@ def test_random_shapes_lockstep(cuda_device, seed):
 # ------------------------------------------------------------------------------------------------
 # Algorithm 3 line 13, deferred into the next step's streaming kernel
 # ------------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("mode", [S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_WS, S.INSERT_SMEM])
+@pytest.mark.parametrize("mode", [S.INSERT_GLOBAL, S.INSERT_TMA, S.INSERT_SMEM])
 def test_deferred_zero_equals_eager_zero(cuda_device, mode):
     """Two engines on the same inputs, one zeroing at once and one deferring: identical outputs every step, the
     deferring one's memory still holds the old values at the chosen coordinates until its next step or a flush,

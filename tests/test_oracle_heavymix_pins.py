@@ -109,6 +109,52 @@ def test_heavymix_more_heavy_than_k_keeps_the_largest():
     assert out["out_val"].tolist() == in0[:k].astype(np.float32).tolist()
 
 
+def test_heavymix_last_mantissa_bit_decides_when_more_than_k_are_heavy():
+    """|H| > k with heavy estimates that differ only in the last mantissa bit.  One row, four buckets holding
+    +-1.0 and +-(the next fp32 above 1.0): every coordinate reads one of them, l2/k is about 4/k < 1, so all d
+    coordinates are heavy.  The k kept must be the k largest under the FULL fp32 magnitude, ties to the smaller
+    index (numpy.lexsort restatement) -- a key that drops the last mantissa bit would see d-way ties and return
+    the first k indices instead."""
+    one = np.float32(1.0)
+    up = np.nextafter(one, np.float32(2.0))
+    d = 200
+    Tf = np.array([[one, up, -one, -up]], np.float32)
+    v = (10.0 + np.arange(d, dtype=np.float32)).reshape(1, d)
+    for k in (20, 150):                                   # fewer than, and more than, the coordinates reading `up`
+        o = Oracle(d, 1, 4, k, 1, 21)
+        h, _ = o.hashes(np.arange(d))
+        est = o.estimate(Tf)
+        is_up = np.isin(h[0], (1, 3))
+        assert (np.abs(est) == np.where(is_up, up, one)).all() and 20 < is_up.sum() < 150
+        out = o.heavymix(Tf, v, fill_seed=5)
+        assert out["nheavy"] == d
+        bits = np.abs(est).view(np.uint32).astype(np.int64)
+        order = np.lexsort((np.arange(d), -bits))         # magnitude bits descending, then index ascending
+        want = np.sort(order[:k])
+        assert out["out_idx"].tolist() == want.tolist()
+        assert out["out_idx"].tolist() != list(range(k))  # what a coarser key would give
+        if k == 20:
+            assert is_up[out["out_idx"]].all()
+        else:
+            assert is_up[out["out_idx"]].sum() == is_up.sum()
+        assert (out["out_val"] == v[0, out["out_idx"]]).all()
+
+
+def test_heavymix_more_heavy_than_k_never_takes_from_nh():
+    """|H| > k: nothing from NH may appear, whatever its fill priority.  One row, two buckets (10, 1): coordinates
+    in bucket 0 read 10 (heavy), the others read 1 (not heavy)."""
+    d, k = 300, 9
+    o = Oracle(d, 1, 2, k, 1, 11)
+    Tf = np.array([[10.0, 1.0]], np.float32)
+    v = np.ones((1, d), np.float32)
+    h, _ = o.hashes(np.arange(d))
+    heavy = np.flatnonzero(h[0] == 0)
+    for seed in range(20):
+        out = o.heavymix(Tf, v, fill_seed=seed)
+        assert out["nheavy"] == heavy.size > k
+        assert out["out_idx"].tolist() == heavy[:k].tolist()
+
+
 def test_fill_is_uniform_over_the_non_heavy_coordinates():
     d, k = 400, 40
     o = Oracle(d, 1, 512, k, 1, 0)
