@@ -56,6 +56,7 @@ extern "C" {
 #define SSGD_EDEVICE    -6  /* a kernel recorded an error: bad index in a caller's list, or a wait gave up */
 #define SSGD_ENOMEM     -7  /* host allocation failed                                                  */
 #define SSGD_ETOOBIG    -8  /* size beyond the fixed capacity of ssgd_exact_topk_static                */
+#define SSGD_EPENDING   -9  /* a deferred zero-out has not been applied yet: ssgd_flush first (or ssgd_unbind) */
 
 #define SSGD_MAX_R 15
 
@@ -84,6 +85,11 @@ typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory 
 /* Algorithm 4 init(r, c) plus the shape of Algorithm 3: d coordinates, r rows (odd, 1..15), c columns,
  * k final sparsity, W workers; 1 <= d < 2^31-1, 1 <= c < 2^31-1, 1 <= k <= d, W >= 1.  Host only. */
 int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int32_t W, uint64_t seed);
+/* Frees the host object.  While a deferred zero-out of the last ssgd_step is still pending (see
+ * ssgd_set_zero_mode) the bound u and v do not hold Algorithm 3 line 13's zeros yet and the marks live only in
+ * the workspace, so the call refuses with SSGD_EPENDING and leaves the context alive: call ssgd_flush first, or
+ * ssgd_unbind to give the marks up on purpose.  (It does not write the zeros itself because it cannot know
+ * that the caller's buffers still exist.) */
 int ssgd_destroy(ssgd_ctx* ctx);
 
 /* The 4r hash parameters, row j at out4r[4j..4j+3] = a_j, b_j, a'_j, b'_j (host memory). */
@@ -103,6 +109,8 @@ int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
  * coordinates: call ssgd_flush before reading u or v yourself.  The library's own entry points that read u or v
  * (ssgd_sketch_accumulate, ssgd_exact_topk, ssgd_heavymix) flush first; ssgd_exact_topk_static has no context
  * and cannot.  Every result (chosen coordinates, values, the state after a flush) is identical in both modes.
+ * The pending marks are state of the method that lives in the workspace: to checkpoint, call ssgd_flush and
+ * save u and v; ssgd_bind and ssgd_destroy refuse (SSGD_EPENDING) while marks are pending.
  * EAGER: ssgd_step writes the zeros before it returns control to the stream's next operation. */
 #define SSGD_ZERO_DEFERRED 0
 #define SSGD_ZERO_EAGER    1
@@ -132,9 +140,14 @@ int ssgd_workspace_bytes(const ssgd_ctx* ctx, int64_t ncand_max, size_t* out_byt
 
 /* Attach the caller-owned worker state u, v ([W][ld] fp32, device; Algorithm 3 line 1 wants them
  * zero before the first step) and the caller-owned workspace (device, 256-byte aligned, at least
- * ssgd_workspace_bytes(ncand_max)).  The buffers must stay valid while the context uses them. */
+ * ssgd_workspace_bytes(ncand_max)).  The buffers must stay valid while the context uses them.  Rebinding a
+ * context whose last step's zero-out is still pending is refused with SSGD_EPENDING (see ssgd_destroy). */
 int ssgd_bind(ssgd_ctx* ctx, float* u, float* v, int64_t ld, void* workspace, size_t workspace_bytes,
               int64_t ncand_max);
+/* Detaches u, v and the workspace.  A pending deferred zero-out is DISCARDED (the previously bound u and v keep
+ * their old values at the last step's k coordinates): the explicit way out of SSGD_EPENDING for a caller who no
+ * longer wants that state.  Touches no device memory. */
+int ssgd_unbind(ssgd_ctx* ctx);
 
 /* Algorithm 3 lines 5-7 (Algorithm 4 update): updates the bound u, v from g ([W][ld_g] fp32, device,
  * read only) and writes each worker's own sketch to tables[w] ([W][r][c] fp32, device; zeroed by the

@@ -349,6 +349,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
 }
 
 int ssgd_destroy(ssgd_ctx* ctx) {
+    if (ctx && ctx->pending_dirty) return SSGD_EPENDING;   // Algorithm 3 line 13 of the last step exists only as marks
     if (ctx && ctx->ev) {
         for (int i = 0; i < TIMING_SLOTS * EV_PER_STEP; ++i) cudaEventDestroy(ctx->ev[i]);
         delete[] ctx->ev;
@@ -447,6 +448,7 @@ int ssgd_bind(ssgd_ctx* x, float* u, float* v, int64_t ld, void* workspace, size
     if (ncand_max < x->k || ncand_max > x->d) return SSGD_EINVAL;
     if (!aligned16(u) || !aligned16(v) || (ld & 3)) return SSGD_EALIGN;
     if (reinterpret_cast<uintptr_t>(workspace) % ALIGN) return SSGD_EALIGN;
+    if (x->pending_dirty) return SSGD_EPENDING;
     layout(x, ncand_max);
     if (workspace_bytes < x->total_bytes) return SSGD_EWORKSPACE;
     x->u = u; x->v = v; x->ld = ld;
@@ -455,6 +457,13 @@ int ssgd_bind(ssgd_ctx* x, float* u, float* v, int64_t ld, void* workspace, size
     if (e) return e;
     CU(cudaMemset(x->ws + x->off_err, 0, 16), "clear error flag");
     CU(cudaMemset(x->ws + x->off_pending, 0, x->map_bytes), "clear pending map");   // nothing awaits its zero-out
+    x->pending_dirty = false;
+    return SSGD_OK;
+}
+
+int ssgd_unbind(ssgd_ctx* x) {
+    if (!x) return SSGD_EINVAL;
+    x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->pending_dirty = false;
     return SSGD_OK;
 }
@@ -827,6 +836,7 @@ const char* ssgd_strerror(int code) {
         case SSGD_EDEVICE: return "a kernel reported an error (index out of range, or a bounded wait gave up)";
         case SSGD_ENOMEM: return "out of host memory";
         case SSGD_ETOOBIG: return "size exceeds the fixed capacity of the built-in scratch";
+        case SSGD_EPENDING: return "a deferred zero-out is pending: call ssgd_flush first (or ssgd_unbind to discard it)";
         default: return "unknown error";
     }
 }

@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libssgd.so")
 
-OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG = 0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG, EPENDING = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT = 0, 1, 2, 3
@@ -39,6 +39,7 @@ SIGNATURES = {
     "ssgd_flush": [_vp, _vp],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
+    "ssgd_unbind": [_vp],
     "ssgd_sketch_accumulate": [_vp, _vp, _i64, _f32, _vp, _vp],
     "ssgd_sketch_merge": [_vp, _vp, _vp, _vp],
     "ssgd_sketch_quantize16": [_vp, _vp, _i32, _vp, _vp],
@@ -127,7 +128,15 @@ class Ssgd:
 
     def __del__(self):
         h, self._h = getattr(self, "_h", None), None
-        if h:
+        if h and self._lib.ssgd_destroy(h) == EPENDING:
+            # the object goes away with a deferred zero-out pending: the bound tensors are still referenced
+            # here, so apply it to them; if that is no longer possible (interpreter shutdown), give it up
+            try:
+                code = self._lib.ssgd_flush(h, _stream())
+            except Exception:
+                code = ECUDA
+            if code != OK:
+                self._lib.ssgd_unbind(h)
             self._lib.ssgd_destroy(h)
 
     def _chk(self, code: int, what: str):
@@ -213,6 +222,11 @@ class Ssgd:
         self._keep = (u, v, workspace)
         self.ncand_max = ncand_max
         return workspace
+
+    def unbind(self) -> None:
+        """Detaches u, v and the workspace; a pending deferred zero-out is discarded."""
+        self._chk(self._lib.ssgd_unbind(self._h), "ssgd_unbind")
+        self._keep = None
 
     # ---- stage calls (asynchronous on the current stream) ------------------------------------
     def sketch_accumulate(self, g: torch.Tensor, rho: float, tables: torch.Tensor) -> None:

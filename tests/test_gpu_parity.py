@@ -158,14 +158,24 @@ STEP_CASES = [
 ]
 
 
-@pytest.mark.parametrize("cfg,steps", STEP_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
-@pytest.mark.parametrize("mode", [S.INSERT_TMA, S.INSERT_GLOBAL, S.INSERT_SMEM])
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
+def _lockstep_combinations():
+    """Every insert variant with the dense candidate path, and every candidate path with the plain-load insert
+    (the candidate path does not depend on the insert variant); the shared-memory insert only where the table fits."""
+    names = {S.INSERT_TMA: "tma", S.INSERT_GLOBAL: "global", S.INSERT_SMEM: "smem",
+             S.PRUNE_ON: "filter", S.PRUNE_EARLY_EXIT: "early_exit", S.PRUNE_OFF: "dense"}
+    out = []
+    for cfg, steps in STEP_CASES:
+        base = f"{cfg.name}-d{cfg.d}-W{cfg.W}-r{cfg.r}-c{cfg.c}"
+        combos = [(S.INSERT_GLOBAL, p) for p in (S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF)] + [(S.INSERT_TMA, S.PRUNE_OFF)]
+        if cfg.r * cfg.c * 4 <= 200 * 1024:
+            combos.append((S.INSERT_SMEM, S.PRUNE_OFF))
+        for mode, prune in combos:
+            out.append(pytest.param(cfg, steps, mode, prune, id=f"{base}-{names[mode]}-{names[prune]}"))
+    return out
+
+
+@pytest.mark.parametrize("cfg,steps,mode,prune", _lockstep_combinations())
 def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
-    if mode == S.INSERT_SMEM and cfg.r * cfg.c * 4 > 200 * 1024:
-        pytest.skip("table does not fit the shared-memory variant")
-    if prune != S.PRUNE_OFF and mode != S.INSERT_GLOBAL:
-        pytest.skip("the candidate path does not depend on the insert variant: one combination suffices")
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_insert_mode(mode)
     eng.set_prune_mode(prune)
@@ -433,6 +443,14 @@ def test_full_size_C5_worker_sweep(cuda_device, W):
     if free < need:
         pytest.skip(f"needs {need >> 30} GiB of device memory")
     run_full(cfg, cuda_device, 1, True)
+
+
+@pytest.mark.parametrize("name", ["P1", "P2", "P3"])
+def test_full_size_paper_sketch_shapes(cuda_device, name):
+    """The paper's own sketch shapes (Table 1 footnotes) at full size, one step in lock step with the oracle:
+    15 x 180,000 with 1.6e6 candidates (dense candidate path, r = 15, real modulo), 5 x 1,000,000 with 3.6e6
+    candidates (bucket bitmap folded 4x), 5 x 180,000 at d = 7.3e7 with 2.6e6 candidates."""
+    run_full(wl.CONFIGS[name], cuda_device, 1, True)
 
 
 def test_full_size_many_coordinates_few_workers(cuda_device):

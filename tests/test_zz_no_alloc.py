@@ -1,4 +1,4 @@
-"""The workspace-free second round + top-k (ssgd_exact_topk_static) against ssgd_exact_topk.
+"""The workspace-free second round + top-k (ssgd_exact_topk_static) against ssgd_exact_topk and the CPU oracle.
 
 Some users of this library are not allowed to allocate device memory: a gradient-compression hook
 that runs inside a trainer whose own allocator holds all of the GPU's memory gets buffers handed in
@@ -7,16 +7,19 @@ They cannot give ssgd_bind a workspace, so ssgd_exact_topk_static keeps its scra
 inside the library.  That array is shared by every call and keeps the previous call's contents, which
 is why this test calls the entry point twice in a row, on different inputs, and wants both results to
 match the workspace-based entry point exactly (the work is integer selection on identically computed
-sums, so the comparison is bit for bit, as in the other parity tests).
+sums, so the comparison is bit for bit, as in the other parity tests) -- and, because the two entry points
+share kernels, the oracle's own second round and final top-k (Algorithm 3 lines 10-11) as well.
 
 Collected last on purpose (file name): if it fails, a run that stops at the first failure has already
 run every other test.  It does not depend on them: it passes alone in a fresh process too.
 """
 import ctypes as C
 
+import numpy as np
 import pytest
 import torch
 
+from oracle import Oracle
 from paper_1903_04488_b200 import ssgd as S
 from paper_1903_04488_b200 import workloads as wl
 
@@ -55,6 +58,41 @@ def test_static_entry_point_matches_workspace_entry_point_twice(cuda_device):
         assert torch.equal(out_idx, want_idx)
         assert torch.equal(out_val.view(torch.int32), want_val.view(torch.int32))
         assert torch.equal(v, v_before)          # this entry point never writes the state
+        # Algorithm 3 lines 10-11 as the oracle states them, on the same v and candidates
+        orc = Oracle(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+        cand_h = cand.cpu().numpy()
+        xs = orc.second_round(v.cpu().numpy(), cand_h)
+        o_idx, o_val = orc.final_topk(cand_h, xs)
+        order = np.argsort(o_idx)
+        assert (out_idx.cpu().numpy() == o_idx[order]).all()
+        assert (out_val.cpu().numpy().view(np.uint32) == o_val[order].view(np.uint32)).all()
+
+
+def test_static_entry_point_counts_an_out_of_range_candidate_as_zero(cuda_device):
+    """A candidate outside [0, d) is never dereferenced: its sum counts as 0, the rest is unchanged."""
+    dev = cuda_device
+    cfg = wl.C2.scaled(d=50_001, W=3, c=1024, ncand=600, k=100)
+    v = wl.gradients(wl.Structure(cfg, dev), 0)
+    cand = torch.arange(0, 3 * cfg.ncand, 3, dtype=torch.int32, device=dev)
+    bad = cand.clone()
+    bad[7] = cfg.d + 123
+    bad[8] = -5
+    out = []
+    for c in (cand, bad):
+        oi = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+        ov = torch.empty(cfg.k, device=dev)
+        S.exact_topk_static(v, cfg.d, c, cfg.k, oi, ov)
+        torch.cuda.synchronize()
+        out.append((oi.cpu().numpy(), ov.cpu().numpy()))
+    orc = Oracle(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+    xs = orc.second_round(v.cpu().numpy(), cand.cpu().numpy())
+    xs_bad = xs.copy()
+    xs_bad[[7, 8]] = 0.0
+    for (gi, gv), x, c in zip(out, (xs, xs_bad), (cand, bad)):
+        o_idx, o_val = orc.final_topk(c.cpu().numpy(), x)
+        pos = {int(i): n for n, i in enumerate(c.cpu().numpy())}
+        order = np.argsort([pos[int(i)] for i in o_idx])     # outputs come in cand_idx order
+        assert (gi == o_idx[order]).all() and (gv.view(np.uint32) == o_val[order].view(np.uint32)).all()
 
 
 def test_static_entry_point_rejects_what_it_cannot_hold(cuda_device):
