@@ -79,6 +79,12 @@ extern "C" {
 #define SSGD_PRUNE_OFF  1
 #define SSGD_PRUNE_ON   2
 #define SSGD_PRUNE_EARLY_EXIT 3
+/* FUSED: lines 9-13 run as ONE cooperative kernel (dense estimates, exact radix select behind grid barriers, the
+ * second round, the final top-k and line 13 by the last block), for problems so small that a chain of short
+ * launches costs more than the work: needs d <= 2^22 and ncand <= 16384 (SSGD_EINVAL from ssgd_step otherwise).  If
+ * the r x c table fits the shared memory of a cluster of up to 8 thread blocks, the estimates read it from there.
+ * AUTO takes this path for d <= 2^21 when it applies.  The results are those of the other modes. */
+#define SSGD_PRUNE_FUSED 4
 
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
 
@@ -115,6 +121,14 @@ int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
 #define SSGD_ZERO_DEFERRED 0
 #define SSGD_ZERO_EAGER    1
 int ssgd_set_zero_mode(ssgd_ctx* ctx, int32_t mode);
+/* Limit, in nanoseconds (>= 1000; default 2e9), of every wait inside a kernel: the grid barriers of the FUSED tail
+ * and the pipeline barriers of the bulk-copy insert kernel.  A wait that runs out makes its kernel record an
+ * error and return; ssgd_status then reports SSGD_EDEVICE once, results of that step are undefined, and the
+ * context stays usable. */
+int ssgd_set_wait_limit_ns(ssgd_ctx* ctx, int64_t ns);
+/* Test hook: thread block (block_plus_one - 1) of those kernels leaves without ever arriving at its barriers, so
+ * that the others' waits run out (nothing hangs, nothing faults); 0 switches the hook off. */
+int ssgd_test_withhold_block(ssgd_ctx* ctx, int32_t block_plus_one);
 /* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Cheap when
  * nothing is pending (one pass over d/8 bytes). */
 int ssgd_flush(ssgd_ctx* ctx, void* stream);
@@ -154,6 +168,16 @@ int ssgd_unbind(ssgd_ctx* ctx);
  * call, then filled with reductions, so bucket sums are order-dependent in the last bits). */
 int ssgd_sketch_accumulate(ssgd_ctx* ctx, const float* g, int64_t ld_g, float rho, float* tables,
                            void* stream);
+
+/* How ssgd_sketch_accumulate walks the W x d worker-coordinates.  COORDINATE_MAJOR: one launch, a thread owns a
+ * group of coordinates and visits every worker (hashes computed once per coordinate; reductions scatter over all
+ * W tables at once).  WORKER_MAJOR: one launch per worker, so that only that worker's r x c table receives
+ * reductions and stays L2-resident meanwhile (hashes recomputed per worker).  AUTO: WORKER_MAJOR once the W
+ * tables together exceed 32 MiB.  The results are the same up to the order of the reductions. */
+#define SSGD_SCHED_AUTO             0
+#define SSGD_SCHED_COORDINATE_MAJOR 1
+#define SSGD_SCHED_WORKER_MAJOR     2
+int ssgd_set_accumulate_schedule(ssgd_ctx* ctx, int32_t mode);
 
 /* Algorithm 3 line 8 (mergeability, Section 3): merged[j][b] = sum over w = 0..W-1, in that order,
  * of tables[w][j][b].  merged is [r][c] fp32, device. */

@@ -11,9 +11,10 @@
 // per coordinate into the L2-resident merged table (sum_w S(v_w) = S(sum_w v_w), Section 3).
 // Several CTAs share an SM, so one CTA's reduction phase overlaps the others' streaming.
 //
-// Every mbarrier wait is bounded: after KT_WAIT_NS nanoseconds the waiter records ERR_TIMEOUT in the
-// error word, raises the CTA's abort flag and leaves; the producer then waits (bounded again) for the
-// copies it still has in flight before the CTA exits.
+// Every mbarrier wait is bounded: after `wait_ns` nanoseconds (an argument; ssgd_set_wait_limit_ns) the waiter
+// records ERR_TIMEOUT in the error word, raises the CTA's abort flag and leaves; whatever happened, the producer
+// waits (bounded again) for the copies it still has in flight before it leaves, so that none lands in a CTA
+// that is gone.
 #pragma once
 #include <stdint.h>
 
@@ -39,6 +40,8 @@ struct AccumArgs {
     // d-bit map of coordinates whose zero-out (Algorithm 3 line 13) is still pending from the previous step: their
     // u and v are read as +0.  NULL: nothing is pending.
     const uint32_t* pending;
+    uint64_t wait_ns;    // limit of every wait inside the kernel (bulk-copy pipeline only)
+    int32_t withhold;    // test hook (bulk-copy pipeline only): the producer of CTA (withhold - 1) issues nothing
 };
 
 #ifndef SSGD_KT_STAGES
@@ -49,7 +52,6 @@ constexpr int KT_CONSUMERS = KT_CONSUMER_WARPS * 32;
 constexpr int KT_THREADS = KT_CONSUMERS + 32;       // + one producer warp
 constexpr int KT_TC = KT_CONSUMERS * 4;             // coordinates per tile: one float4 per consumer thread
 constexpr int KT_STAGES = SSGD_KT_STAGES;
-constexpr uint64_t KT_WAIT_NS = 2000000000ull;      // a wait gives up after two seconds
 
 struct alignas(128) KtSlot { float g[KT_TC]; float u[KT_TC]; float v[KT_TC]; };
 struct KtShared {
@@ -102,14 +104,14 @@ __device__ __forceinline__ uint64_t global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait; false if it gave up (KT_WAIT_NS elapsed) or the CTA is aborting.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort) {
+// Bounded wait; false if it gave up (wait_ns elapsed) or the CTA is aborting.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort, uint64_t wait_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0) {
-            if (*abort || global_ns() - t0 > KT_WAIT_NS) return false;
+            if (*abort || global_ns() - t0 > wait_ns) return false;
             __nanosleep(64);
         }
     }
@@ -150,28 +152,30 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
             const uint64_t pol = policy_evict_first();
             uint32_t n = 0;
             bool ok = true;
-            for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
+            const bool withheld = A.withhold && (int)blockIdx.x == A.withhold - 1;
+            for (int64_t tile = blockIdx.x; tile < ntiles && ok && !withheld; tile += gridDim.x) {
                 const int64_t i0 = tile * KT_TC;
                 const uint32_t bytes = (uint32_t)((d_main - i0 < KT_TC ? d_main - i0 : KT_TC) * 4);
                 for (int w = 0; w < A.W; ++w, ++n) {
                     const int s = n % KT_STAGES;
-                    if (n >= KT_STAGES && !mbar_wait(&S.empty[s], ((n / KT_STAGES) - 1) & 1, &S.abort)) { ok = false; break; }
+                    if (n >= KT_STAGES && !mbar_wait(&S.empty[s], ((n / KT_STAGES) - 1) & 1, &S.abort, A.wait_ns)) { ok = false; break; }
                     mbar_expect_tx(&S.full[s], 3 * bytes);
                     bulk_load(S.slot[s].g, A.g + (int64_t)w * A.ld_g + i0, bytes, &S.full[s], pol);
                     bulk_load(S.slot[s].u, A.u + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
                     bulk_load(S.slot[s].v, A.v + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
                 }
             }
-            if (!ok) {
-                // give up: report, tell the consumers, and let the copies already issued land before exit
+            if (!ok) {                                     // give up: report and tell the consumers
                 atomicExch(errflag, ERR_TIMEOUT);
                 S.abort = 1;
-                const uint32_t first = n > KT_STAGES ? n - KT_STAGES : 0;
-                for (uint32_t m = first; m < n; ++m) {
-                    uint64_t* bar = &S.full[m % KT_STAGES];
-                    const uint64_t t0 = global_ns();
-                    while (!mbar_try_wait(bar, (m / KT_STAGES) & 1) && global_ns() - t0 < KT_WAIT_NS) __nanosleep(64);
-                }
+            }
+            // the copies of the last stages issued must have landed before this CTA may go away, whether the
+            // consumers took them or gave up (returns at once for stages that completed long ago)
+            const uint32_t first = n > KT_STAGES ? n - KT_STAGES : 0;
+            for (uint32_t m = first; m < n; ++m) {
+                uint64_t* bar = &S.full[m % KT_STAGES];
+                const uint64_t t0 = global_ns();
+                while (!mbar_try_wait(bar, (m / KT_STAGES) & 1) && global_ns() - t0 < A.wait_ns) __nanosleep(64);
             }
         }
     } else {
@@ -185,7 +189,7 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
             const uint32_t pend = active ? pending_bits4(A.pending, i0) : 0u;
             for (int w = 0; w < A.W; ++w, ++n) {
                 const int s = n % KT_STAGES;
-                if (!mbar_wait(&S.full[s], (n / KT_STAGES) & 1, &S.abort)) { ok = false; break; }
+                if (!mbar_wait(&S.full[s], (n / KT_STAGES) & 1, &S.abort, A.wait_ns)) { ok = false; break; }
                 if (active) {
                     const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[4 * tid]);
                     float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * tid]);

@@ -4,6 +4,7 @@
 //   launch_accum.cu     Algorithm 3 lines 5-7 (k_accum_insert, k_accum_insert_tma, k_insert_rows)
 //   launch_unsketch.cu  Algorithm 3 line 9 (k_unsketch, k_unsketch_sample, k_unsketch_filter, k_unsketch_pruned)
 //                       and Algorithm 1's key kernel
+//   launch_small.cu     Algorithm 3 lines 9-13 in one cooperative kernel (k_small_tail)
 //   ssgd.cu             the C ABI, workspace layout, the selections and everything else
 #pragma once
 #include <cuda_runtime.h>
@@ -21,6 +22,7 @@
 #include "filter_unsketch.cuh"
 #include "heavymix.cuh"
 #include "step_kernels.cuh"
+#include "small_tail.cuh"
 
 struct ssgd_ctx {
     int64_t d, c, k;
@@ -35,6 +37,7 @@ struct ssgd_ctx {
     char* ws; size_t ws_bytes; int64_t ncand_max;
     // workspace layout (byte offsets)
     size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
+    size_t off_h19_c, off_h19_f, off_small;
     size_t off_sp_hist, off_sp_state, off_maps, off_map_chunks, off_list_idx, off_list_est;   // early-exit path
     size_t map_bytes;
     int64_t list_cap, nchunk_map;
@@ -44,6 +47,7 @@ struct ssgd_ctx {
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
     size_t off_pending;     // d-bit map of the deferred zero-out; survives from step to step
     int32_t zero_mode;      // SSGD_ZERO_DEFERRED / SSGD_ZERO_EAGER
+    int32_t sched_mode;     // SSGD_SCHED_*: how ssgd_sketch_accumulate walks workers and coordinates
     bool pending_dirty;     // a deferred ssgd_step has run since the last flush: u, v may await their zero-out
     size_t off_hm;
     int32_t prune_mode;
@@ -55,6 +59,9 @@ struct ssgd_ctx {
     // device facts
     int device; int sm_count; int max_smem_optin;
     int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
+    int small_grid, small_cs; size_t small_smem;   // launch shape of the one-kernel tail (small_grid 0 = not queried yet)
+    uint64_t wait_ns;       // limit of every device-side wait (grid barriers, mbarriers)
+    int32_t withhold;       // test hook: this CTA (1-based; 0 = none) never arrives, so the others' waits run out
     int64_t launches;
     // optional per-stage timing of ssgd_step (CUDA events on the caller's stream)
     bool timing;
@@ -159,5 +166,8 @@ int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st);
 bool use_filter(const ssgd_ctx* x);
 int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st);
 int launch_heavymix_keys(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st);
+// defined in launch_small.cu
+bool small_tail_applicable(const ssgd_ctx* x, int64_t ncand);
+int launch_small_tail(ssgd_ctx* x, SmallArgs& A, cudaStream_t st);
 
 }  // namespace ssgd

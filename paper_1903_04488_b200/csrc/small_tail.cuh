@@ -1,0 +1,410 @@
+// small_tail.cuh -- Algorithm 3 lines 9-13 in ONE kernel, for problems so small that a chain of short launches
+// costs more than the work itself (d up to a few million coordinates, at most SMALL_MAX_NCAND candidates).
+//
+// The grid is co-resident (one CTA per SM, launched cooperatively) and its CTAs meet at three grid-wide barriers:
+//
+//   phase 1   every CTA estimates its share of the coordinates (Algorithm 4 estimate: median of the r signed
+//             buckets), stores est[i] and counts the top 12 bits of |est| in a shared-memory histogram -> H1.
+//             If the r x c table fits the shared memory of a thread-block cluster (2, 4 or 8 CTAs), each CTA first
+//             copies its column slice of every row into shared memory and the r lookups per coordinate are
+//             distributed-shared-memory loads instead of scattered reads of L2: the dense unsketch is bound by
+//             the rate of scattered 32-byte sectors (about one per clock per SM), shared memory is not.
+//   barrier   H1 complete: every CTA finds the first threshold digit d1 for itself
+//   phase 2   histogram H2 of the next 11 key bits among the items inside d1
+//   barrier   -> second digit d2
+//   phase 3   histogram H3 of the last 8 key bits among the items matching the 23-bit prefix
+//   barrier   -> threshold key T and tie quota Q
+//   phase 4   every CTA marks its coordinates above T in a d-bit map A, those equal to T in map B.  The CTA that
+//             draws the last ticket goes on alone (nobody waits for it):
+//   phase 5   ordered walk of the two maps -> cand_idx ascending, ties at T to the smallest coordinates
+//             (line 9); xs[m] = the accumulate kernel's sum over the workers at cand_idx[m] (line 10); exact
+//             top-k of |xs| in shared memory, 12 + 11 + 8 bits, ordered emit of out_idx / out_val (line 11);
+//             line 13 as marks in the pending map (deferred) or as zeros written to u and v (eager, small k*W).
+//
+// Every wait at a barrier is bounded: after `wait_ns` the waiting CTA records ERR_TIMEOUT in the error word,
+// raises the abort flag so that the others stop waiting too, and returns.  All use of other CTAs' shared memory
+// lies before the first barrier and is closed by a cluster barrier, so a CTA that gives up leaves nobody reading
+// memory that is gone.
+#pragma once
+#include <stdint.h>
+
+#include "accum_tma.cuh"
+#include "estimate.cuh"
+#include "hash.cuh"
+#include "select.cuh"
+
+namespace ssgd {
+
+constexpr int ST_THREADS = 512;
+constexpr int ST_WARPS = ST_THREADS / 32;
+constexpr int64_t SMALL_MAX_NCAND = 16384;               // candidates the last CTA holds in shared memory
+constexpr int64_t SMALL_MAX_D = (int64_t)1 << 22;        // coordinates (the last CTA walks two d-bit maps)
+constexpr size_t SMALL_TABLE_SMEM_MAX = 200 * 1024;      // table slice per CTA (next to a 16 KiB histogram)
+
+struct SmallState {          // zeroed before the step
+    uint32_t bar;            // arrivals at the grid barriers (monotonic: barrier n completes at n * gridDim.x)
+    uint32_t abort;          // a wait gave up
+    uint32_t ticket;         // CTAs that finished phase 4
+    uint32_t pad[13];
+};
+
+struct SmallArgs {
+    const float* table; int64_t c; int64_t d;
+    HashParams hp; Bucketizer bk;
+    float* est;              // [d], 16-byte aligned
+    uint32_t* h1; uint32_t* h2; uint32_t* h3;   // global histograms of the candidate selection, zeroed
+    SmallState* st;
+    uint32_t* map_a; uint32_t* map_b;           // [ceil(d/32)] words each, zeroed; 16-byte aligned
+    const float* xsum;       // [d] per-coordinate sums over the workers of the new v
+    int32_t* cand_idx; float* xs;               // [ncand] (kept for inspection)
+    uint32_t ncand, k;
+    int32_t* out_idx; float* out_val;           // [k]
+    uint32_t* pending;       // the pending map of a deferred line 13: emptied in phase 1 (the accumulate kernel has
+    int64_t pending_words;   // consumed it), marked again in phase 5 if mark_pending != 0
+    int32_t mark_pending;
+    float* u; float* v; int64_t ld; int32_t W;  // eager line 13 written here when zero_inline != 0
+    int32_t zero_inline;
+    int32_t use_smem;        // 1: table slices in the cluster's shared memory
+    int32_t col_shift;       // use_smem: columns [rank << col_shift, (rank + 1) << col_shift) of every row live in CTA `rank`
+    uint64_t wait_ns;        // limit of a barrier wait
+    int32_t withhold;        // test hook: CTA (withhold - 1) leaves before the first barrier, so the others' wait runs out
+    int32_t* errflag;
+};
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// fp32 at byte offset `off` of the dynamic shared memory of CTA `rank` of this cluster
+__device__ __forceinline__ float dsmem_load(uint32_t local_base, uint32_t off, uint32_t rank) {
+    uint32_t remote;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_base + off), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// n-th (1-based) grid barrier.  False, in every thread of the CTA, if the wait ran out or another CTA gave up.
+__device__ __forceinline__ bool small_grid_barrier(const SmallArgs& A, uint32_t nth, uint32_t* s_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t ok = 1;
+        __threadfence();
+        atomicAdd(&A.st->bar, 1u);
+        const uint32_t target = nth * gridDim.x;
+        const uint64_t t0 = global_ns();
+        for (uint32_t it = 1; ld_acquire_u32(&A.st->bar) < target; ++it) {
+            if ((it & 15u) == 0 && (ld_acquire_u32(&A.st->abort) != 0u || global_ns() - t0 > A.wait_ns)) { ok = 0; break; }
+        }
+        if (!ok) { atomicExch(&A.st->abort, 1u); atomicExch(A.errflag, ERR_TIMEOUT); }
+        __threadfence();
+        *s_flag = ok;
+    }
+    __syncthreads();
+    return *s_flag != 0;
+}
+
+// Largest bin D of a shared-memory histogram with count(bins > D) < want <= count(bins >= D); rem = want - count(bins > D).
+// All ST_THREADS threads call.  1 <= want <= total count.
+template <int NBINS>
+__device__ __forceinline__ void smem_find_from_top(const uint32_t* hist, uint32_t want, uint32_t* s_warp, uint32_t* s_found,
+                                                   uint32_t& digit, uint32_t& rem) {
+    constexpr int NT = NBINS < ST_THREADS ? NBINS : ST_THREADS;   // searching threads
+    constexpr int PER = NBINS / NT;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    if (t == 0) { s_found[0] = 0; s_found[1] = 1; }
+    uint32_t sum = 0, incl = 0;
+    if (t < NT) {
+#pragma unroll
+        for (int s = 0; s < PER; ++s) sum += hist[t * PER + s];
+    }
+    incl = sum;                                            // sum over the lanes >= lane of this warp
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t o = __shfl_down_sync(0xFFFFFFFFu, incl, off);
+        if (lane + off < 32) incl += o;
+    }
+    if (lane == 0) s_warp[warp] = incl;
+    __syncthreads();
+    if (t < NT) {
+        uint32_t above = incl - sum;
+        for (int w2 = warp + 1; w2 < ST_WARPS; ++w2) above += s_warp[w2];
+        if (above < want && want <= above + sum) {
+            uint32_t acc = above;
+            for (int b = t * PER + PER - 1; b >= t * PER; --b) {
+                const uint32_t h = hist[b];
+                if (acc + h >= want) { s_found[0] = (uint32_t)b; s_found[1] = want - acc; break; }
+                acc += h;
+            }
+        }
+    }
+    __syncthreads();
+    digit = s_found[0];
+    rem = s_found[1];
+    __syncthreads();
+}
+
+// Exclusive block-wide scan of two counters per thread (ST_THREADS threads).
+__device__ __forceinline__ void block_excl_scan2(uint32_t a, uint32_t b, uint32_t* s_a, uint32_t* s_b, uint32_t& ea, uint32_t& eb) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t ia = a, ib = b;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t oa = __shfl_up_sync(0xFFFFFFFFu, ia, off), ob = __shfl_up_sync(0xFFFFFFFFu, ib, off);
+        if (lane >= off) { ia += oa; ib += ob; }
+    }
+    __syncthreads();
+    if (lane == 31) { s_a[warp] = ia; s_b[warp] = ib; }
+    __syncthreads();
+    ea = ia - a; eb = ib - b;
+    for (int w = 0; w < warp; ++w) { ea += s_a[w]; eb += s_b[w]; }
+    __syncthreads();
+}
+
+template <int R, bool POW2>
+__global__ void __launch_bounds__(ST_THREADS, 1)
+k_small_tail(const SmallArgs A) {
+    extern __shared__ __align__(16) unsigned char st_dyn[];   // table slice, later the candidates and their sums
+    __shared__ SelShared sh;
+    __shared__ uint32_t s_flag, s_warp_a[ST_WARPS], s_warp_b[ST_WARPS], s_found[2];
+    const int tid = threadIdx.x;
+    const int64_t groups = (A.d + 3) >> 2;
+    const int64_t gstride = (int64_t)gridDim.x * ST_THREADS;
+    const int64_t gtid = (int64_t)blockIdx.x * ST_THREADS + tid;
+    const uint32_t crank = A.use_smem ? cluster_ctarank() : 0u;
+    const uint32_t dyn_base = (uint32_t)__cvta_generic_to_shared(st_dyn);
+    const uint32_t cols = 1u << A.col_shift;               // columns of a row held by one CTA
+
+    // ---------------- phase 1: table slice -> shared memory; estimates, H1 ----------------
+    for (int b = tid; b < H1_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    if (A.pending)
+        for (int64_t t = gtid; t < A.pending_words; t += gstride) A.pending[t] = 0u;   // consumed by the accumulate kernel
+    if (A.use_smem) {
+        float* slice = reinterpret_cast<float*>(st_dyn);
+        const int64_t c0 = (int64_t)crank << A.col_shift;
+        const int64_t n = c0 < A.c ? (A.c - c0 < (int64_t)cols ? A.c - c0 : (int64_t)cols) : 0;   // my columns of a row
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const float* src = A.table + (int64_t)j * A.c + c0;
+            float* dst = slice + (int64_t)j * cols;
+            for (int64_t b0 = tid; b0 < n; b0 += ST_THREADS * 8) {
+                float t[8];
+#pragma unroll
+                for (int s = 0; s < 8; ++s) t[s] = b0 + s * ST_THREADS < n ? __ldcg(src + b0 + s * ST_THREADS) : 0.f;
+#pragma unroll
+                for (int s = 0; s < 8; ++s) if (b0 + s * ST_THREADS < n) dst[b0 + s * ST_THREADS] = t[s];
+            }
+        }
+        cluster_sync_all();                                // every slice of the cluster is in place
+    } else {
+        __syncthreads();
+    }
+    for (int64_t q = gtid; q < groups; q += gstride) {
+        const int64_t i0 = q << 2;
+        float rowv[4][R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            uint32_t hb[4];
+            row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const uint32_t b = hb[e] & P31;
+                float t;
+                if (A.use_smem) t = dsmem_load(dyn_base, ((uint32_t)j * cols + (b & (cols - 1u))) * 4u, b >> A.col_shift);
+                else t = table_load(A.table + (int64_t)j * A.c + b);
+                rowv[e][j] = apply_sign(t, hb[e]);
+            }
+        }
+        float m[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m[e] = median_of<R>(rowv[e]);
+        if (i0 + 3 < A.d) {
+            *reinterpret_cast<float4*>(A.est + i0) = make_float4(m[0], m[1], m[2], m[3]);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) atomicAdd(&sh.hist[key_of(m[e]) >> H1_SHIFT], 1u);
+        } else {
+            for (int e = 0; e < 4 && i0 + e < A.d; ++e) {
+                A.est[i0 + e] = m[e];
+                atomicAdd(&sh.hist[key_of(m[e]) >> H1_SHIFT], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(sh.hist, A.h1);
+    if (A.use_smem) cluster_sync_all();                    // nobody reads this CTA's slice any more
+    if (A.withhold && (int)blockIdx.x == A.withhold - 1) return;
+    if (!small_grid_barrier(A, 1, &s_flag)) return;
+
+    // keys of this thread's coordinates, re-read from est (L2) in each of the later phases
+    auto for_my_keys = [&](auto&& f) {
+        for (int64_t q = gtid; q < groups; q += gstride) {
+            const int64_t i0 = q << 2;
+            uint32_t key[4];
+            if (i0 + 3 < A.d) {
+                const float4 t = __ldcg(reinterpret_cast<const float4*>(A.est + i0));
+                key[0] = key_of(t.x); key[1] = key_of(t.y); key[2] = key_of(t.z); key[3] = key_of(t.w);
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) key[e] = i0 + e < A.d ? key_of(__ldcg(A.est + i0 + e)) : NO_ITEM;
+            }
+            f(i0, key);
+        }
+    };
+
+    // ---------------- phase 2: second digit ----------------
+    uint32_t d1, rem1, d2, rem2, d3, rem3;
+    block_find_from_top<H1_BINS>(A.h1, A.ncand, sh, d1, rem1);
+    for (int b = tid; b < H2_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    for_my_keys([&](int64_t, const uint32_t (&key)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (key[e] != NO_ITEM && (key[e] >> H1_SHIFT) == d1) atomicAdd(&sh.hist[(key[e] >> H2_SHIFT) & (H2_BINS - 1)], 1u);
+    });
+    __syncthreads();
+    flush_hist<H2_BINS>(sh.hist, A.h2);
+    if (!small_grid_barrier(A, 2, &s_flag)) return;
+
+    // ---------------- phase 3: third digit ----------------
+    block_find_from_top<H2_BINS>(A.h2, rem1, sh, d2, rem2);
+    const uint32_t prefix = (d1 << H2_BITS) | d2;
+    for (int b = tid; b < H3_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    for_my_keys([&](int64_t, const uint32_t (&key)[4]) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            if (key[e] != NO_ITEM && (key[e] >> H2_SHIFT) == prefix) atomicAdd(&sh.hist[key[e] & (H3_BINS - 1)], 1u);
+    });
+    __syncthreads();
+    flush_hist<H3_BINS>(sh.hist, A.h3);
+    if (!small_grid_barrier(A, 3, &s_flag)) return;
+
+    // ---------------- phase 4: marks ----------------
+    block_find_from_top<H3_BINS>(A.h3, rem2, sh, d3, rem3);
+    const uint32_t T = (d1 << H1_SHIFT) | (d2 << H2_SHIFT) | d3, Q = rem3;
+    for_my_keys([&](int64_t i0, const uint32_t (&key)[4]) {
+        uint32_t gt = 0, eq = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            if (key[e] == NO_ITEM) continue;
+            gt |= (key[e] > T ? 1u : 0u) << e;
+            eq |= (key[e] == T ? 1u : 0u) << e;
+        }
+        const int sh4 = (int)(i0 & 31);                    // a group of four never straddles a map word
+        if (gt) atomicOr(A.map_a + (i0 >> 5), gt << sh4);
+        if (eq) atomicOr(A.map_b + (i0 >> 5), eq << sh4);
+    });
+    if (!block_is_last(&A.st->ticket, sh)) return;
+
+    // ---------------- phase 5 (one CTA): candidates, second round, final top-k, line 13 ----------------
+    int32_t* cand_s = reinterpret_cast<int32_t*>(st_dyn);
+    float* xs_s = reinterpret_cast<float*>(st_dyn) + A.ncand;
+    const int64_t nwords = (A.d + 31) >> 5;
+    const int64_t per = ((nwords + ST_THREADS - 1) / ST_THREADS + 3) & ~(int64_t)3;   // words per thread, a multiple of 4
+    const int64_t w_lo = (int64_t)tid * per, w_hi = w_lo + per < nwords ? w_lo + per : nwords;
+    uint32_t ca = 0, cb = 0;
+    for (int64_t w = w_lo; w < w_hi; w += 4) {
+        if (w + 3 < nwords) {
+            const uint4 a = __ldcg(reinterpret_cast<const uint4*>(A.map_a + w)), b = __ldcg(reinterpret_cast<const uint4*>(A.map_b + w));
+            ca += __popc(a.x) + __popc(a.y) + __popc(a.z) + __popc(a.w);
+            cb += __popc(b.x) + __popc(b.y) + __popc(b.z) + __popc(b.w);
+        } else {
+            for (int64_t t = w; t < w_hi; ++t) { ca += __popc(__ldcg(A.map_a + t)); cb += __popc(__ldcg(A.map_b + t)); }
+        }
+    }
+    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) cand_s[m] = 0;     // consistent histograms fill every slot
+    uint32_t run_a, run_b;
+    block_excl_scan2(ca, cb, s_warp_a, s_warp_b, run_a, run_b);
+    if (ca | cb) {
+        for (int64_t w = w_lo; w < w_hi; ++w) {
+            const uint32_t wa = __ldcg(A.map_a + w), wb = __ldcg(A.map_b + w);
+            uint32_t bits = wa | wb;
+            while (bits) {
+                const int bit = __ffs(bits) - 1;
+                bits &= bits - 1;
+                uint32_t slot = 0xFFFFFFFFu;
+                if ((wa >> bit) & 1u) { slot = run_a + (run_b < Q ? run_b : Q); ++run_a; }
+                else { if (run_b < Q) slot = run_a + run_b; ++run_b; }
+                if (slot < A.ncand) {
+                    const int32_t coord = (int32_t)((w << 5) + bit);
+                    cand_s[slot] = coord;
+                    A.cand_idx[slot] = coord;
+                }
+            }
+        }
+    }
+    for (int b = tid; b < H1_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    // line 10: one read per candidate of the sums the accumulate kernel left
+    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) {
+        const uint32_t i = (uint32_t)cand_s[m];
+        const float x = (int64_t)i < A.d ? __ldcg(A.xsum + i) : 0.0f;
+        xs_s[m] = x;
+        A.xs[m] = x;
+        atomicAdd(&sh.hist[key_of(x) >> H1_SHIFT], 1u);
+    }
+    __syncthreads();
+    // line 11: exact top-k of |xs| among the candidates, all in shared memory
+    uint32_t e1, r1, e2, r2, e3, r3;
+    smem_find_from_top<H1_BINS>(sh.hist, A.k, s_warp_a, s_found, e1, r1);
+    for (int b = tid; b < H2_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) {
+        const uint32_t key = key_of(xs_s[m]);
+        if ((key >> H1_SHIFT) == e1) atomicAdd(&sh.hist[(key >> H2_SHIFT) & (H2_BINS - 1)], 1u);
+    }
+    __syncthreads();
+    smem_find_from_top<H2_BINS>(sh.hist, r1, s_warp_a, s_found, e2, r2);
+    const uint32_t prefix2 = (e1 << H2_BITS) | e2;
+    for (int b = tid; b < H3_BINS; b += ST_THREADS) sh.hist[b] = 0;
+    __syncthreads();
+    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) {
+        const uint32_t key = key_of(xs_s[m]);
+        if ((key >> H2_SHIFT) == prefix2) atomicAdd(&sh.hist[key & (H3_BINS - 1)], 1u);
+    }
+    __syncthreads();
+    smem_find_from_top<H3_BINS>(sh.hist, r2, s_warp_a, s_found, e3, r3);
+    const uint32_t T2 = (e1 << H1_SHIFT) | (e2 << H2_SHIFT) | e3, Q2 = r3;
+    // ordered emit: thread t owns the candidates [t * per2, (t + 1) * per2)
+    const uint32_t per2 = (A.ncand + ST_THREADS - 1) / ST_THREADS;
+    const uint32_t m_lo = tid * per2 < A.ncand ? tid * per2 : A.ncand;
+    const uint32_t m_hi = m_lo + per2 < A.ncand ? m_lo + per2 : A.ncand;
+    uint32_t cg = 0, ce = 0;
+    for (uint32_t m = m_lo; m < m_hi; ++m) {
+        const uint32_t key = key_of(xs_s[m]);
+        cg += key > T2 ? 1u : 0u;
+        ce += key == T2 ? 1u : 0u;
+    }
+    uint32_t g_before, e_before;
+    block_excl_scan2(cg, ce, s_warp_a, s_warp_b, g_before, e_before);
+    for (uint32_t m = m_lo; m < m_hi; ++m) {
+        const float x = xs_s[m];
+        const uint32_t key = key_of(x);
+        uint32_t slot = 0xFFFFFFFFu;
+        if (key > T2) { slot = g_before + (e_before < Q2 ? e_before : Q2); ++g_before; }
+        else if (key == T2) { if (e_before < Q2) slot = g_before + e_before; ++e_before; }
+        if (slot < A.k) {
+            const int32_t i = cand_s[m];
+            A.out_idx[slot] = i;
+            A.out_val[slot] = x;
+            if (A.mark_pending) atomicOr(A.pending + (i >> 5), 1u << (i & 31));  // deferred line 13
+            if (A.zero_inline)
+                for (int64_t w = 0; w < A.W; ++w) { A.u[w * A.ld + i] = 0.0f; A.v[w * A.ld + i] = 0.0f; }
+        }
+    }
+}
+
+#endif  // __CUDACC__
+}  // namespace ssgd

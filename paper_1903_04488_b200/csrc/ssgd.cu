@@ -46,6 +46,10 @@ namespace {
 
 constexpr size_t ALIGN = 256;
 constexpr int TIMING_SLOTS = 256;
+// ssgd_sketch_accumulate goes through the workers one launch at a time once all W tables together exceed this
+constexpr size_t WORKER_MAJOR_MIN_BYTES = (size_t)32 << 20;
+constexpr int64_t SMALL_AUTO_MAX_D = (int64_t)1 << 21;      // AUTO takes the one-kernel tail up to this many coordinates
+constexpr int64_t SMALL_INLINE_ZERO_MAX = 65536;            // eager line 13 inside the tail kernel up to this many k*W
 constexpr int EV_PER_STEP = SSGD_NSTAGES + 1;
 inline size_t up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
@@ -69,15 +73,21 @@ void derive_params(uint64_t seed, int32_t r, HashParams& hp) {
 
 void layout(ssgd_ctx* x, int64_t ncand_max) {
     size_t o = 0;
+    // the head, cleared at the start of every step.  What the one-kernel tail of small problems needs comes first
+    // (table, the two coordinate maps, its barrier state, H1-H3 and state of the candidate selection), so that its
+    // memset stops at off_h19_c
     x->off_table = o;   o += up((size_t)x->r * x->c * 4);
-    x->off_hist_c = o;  o += up((size_t)(SEL_HIST_WORDS + H19_BINS) * 4);
+    x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
+    x->off_maps = o;    o += 2 * x->map_bytes;
+    x->off_small = o;   o += up(sizeof(SmallState));
+    x->off_hist_c = o;  o += up((size_t)SEL_HIST_WORDS * 4);
     x->off_state_c = o; o += up(sizeof(SelState));
-    x->off_hist_f = o;  o += up((size_t)(SEL_HIST_WORDS + H19_BINS) * 4);
+    x->off_h19_c = o;   o += up((size_t)H19_BINS * 4);
+    x->off_hist_f = o;  o += up((size_t)SEL_HIST_WORDS * 4);
+    x->off_h19_f = o;   o += up((size_t)H19_BINS * 4);
     x->off_state_f = o; o += up(sizeof(SelState));
     x->off_sp_hist = o; o += up((size_t)(2 * H1_BINS + H2_BINS) * 4);   // its 2^19-bin table is the candidate selection's
     x->off_sp_state = o; o += up(sizeof(SparseState));
-    x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
-    x->off_maps = o;    o += 2 * x->map_bytes;
     x->nchunk_map = ((x->d + 31) / 32 + MAP_CHUNK_WORDS - 1) / MAP_CHUNK_WORDS;
     x->off_map_chunks = o; o += up((size_t)x->nchunk_map * 8);   // marks per chunk of map words: counted from zero
     x->off_hm = o;      o += up(sizeof(HeavymixState));
@@ -113,7 +123,8 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
 SelBuffers sel_buffers(ssgd_ctx* x, bool final_stage) {
     SelBuffers sb{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_hist_f : x->off_hist_c));
-    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS; sb.h19 = h + SEL_HIST_WORDS;
+    sb.h1 = h; sb.h2 = h + H1_BINS; sb.h3 = h + H1_BINS + H2_BINS;
+    sb.h19 = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_h19_f : x->off_h19_c));
     sb.state = reinterpret_cast<SelState*>(x->ws + (final_stage ? x->off_state_f : x->off_state_c));
     uint32_t* ch = reinterpret_cast<uint32_t*>(x->ws + (final_stage ? x->off_chunk_f : x->off_chunk_c));
     const int64_t nch = final_stage ? x->nchunk_f : x->nchunk_c;
@@ -194,7 +205,7 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
     SparseBuffers sp{};
     uint32_t* h = reinterpret_cast<uint32_t*>(x->ws + x->off_sp_hist);
     sp.h1_sample = h; sp.h1 = h + H1_BINS; sp.h2 = h + 2 * H1_BINS;
-    sp.h19 = reinterpret_cast<uint32_t*>(x->ws + x->off_hist_c) + SEL_HIST_WORDS;   // never used by both in one step
+    sp.h19 = reinterpret_cast<uint32_t*>(x->ws + x->off_h19_c);   // never used by both in one step
     sp.state = reinterpret_cast<SparseState*>(x->ws + x->off_sp_state);
     sp.list_idx = reinterpret_cast<int32_t*>(x->ws + x->off_list_idx);
     sp.list_est = reinterpret_cast<float*>(x->ws + x->off_list_est);
@@ -204,6 +215,13 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
     sp.chunk_a = reinterpret_cast<uint32_t*>(x->ws + x->off_map_chunks);
     sp.chunk_b = sp.chunk_a + x->nchunk_map;
     return sp;
+}
+
+// Whether ssgd_step runs lines 9-13 as the one cooperative kernel of small_tail.cuh.  AUTO: up to 2^21 coordinates
+// (measured on B200 against the chain of short launches).
+bool use_small(const ssgd_ctx* x, int64_t ncand) {
+    if (x->prune_mode == SSGD_PRUNE_FUSED) return small_tail_applicable(x, ncand);
+    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D;
 }
 
 // Whether ssgd_step takes the pruned first pass + selection on the survivor list (filter_unsketch.cuh,
@@ -343,7 +361,8 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
+    x->small_grid = 0; x->small_cs = 0; x->small_smem = 0; x->wait_ns = 2000000000ull; x->withhold = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -410,8 +429,14 @@ int ssgd_set_insert_split(ssgd_ctx* x, int64_t bytes) {
     return SSGD_OK;
 }
 
+int ssgd_set_accumulate_schedule(ssgd_ctx* x, int32_t mode) {
+    if (!x || mode < SSGD_SCHED_AUTO || mode > SSGD_SCHED_WORKER_MAJOR) return SSGD_EINVAL;
+    x->sched_mode = mode;
+    return SSGD_OK;
+}
+
 int ssgd_set_prune_mode(ssgd_ctx* x, int32_t mode) {
-    if (!x || mode < SSGD_PRUNE_AUTO || mode > SSGD_PRUNE_EARLY_EXIT) return SSGD_EINVAL;
+    if (!x || mode < SSGD_PRUNE_AUTO || mode > SSGD_PRUNE_FUSED) return SSGD_EINVAL;
     x->prune_mode = mode;
     return SSGD_OK;
 }
@@ -481,7 +506,22 @@ int ssgd_sketch_accumulate(ssgd_ctx* x, const float* g, int64_t ld_g, float rho,
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr; A.pending = nullptr;
-    return launch_accum(x, A, INS_PER_WORKER, st);
+    A.wait_ns = x->wait_ns; A.withhold = 0;
+    const size_t all_tables = (size_t)x->W * x->r * x->c * 4;
+    const bool worker_major = x->sched_mode == SSGD_SCHED_WORKER_MAJOR ||
+                              (x->sched_mode == SSGD_SCHED_AUTO && x->W > 1 && all_tables > WORKER_MAJOR_MIN_BYTES);
+    if (!worker_major) return launch_accum(x, A, INS_PER_WORKER, st);
+    // one worker per launch: its g, u, v stream past once and the reductions go to its own r x c table only, which
+    // stays L2-resident for the whole launch (a single worker's sketch is the merged-table kernel with W = 1)
+    const int64_t rc = (int64_t)x->r * x->c;
+    for (int w = 0; w < x->W; ++w) {
+        AccumArgs B = A;
+        B.W = 1;
+        B.g = g + (int64_t)w * ld_g; B.u = x->u + (int64_t)w * x->ld; B.v = x->v + (int64_t)w * x->ld;
+        B.table = tables + (int64_t)w * rc;
+        if ((e = launch_accum(x, B, INS_MERGED_GLOBAL, st))) return e;
+    }
+    return SSGD_OK;
 }
 
 int ssgd_sketch_merge(ssgd_ctx* x, const float* tables, float* merged, void* stream) {
@@ -555,14 +595,17 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     const int mode = resolve_insert_mode(x);
     if (mode < 0) return SSGD_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool small = use_small(x, ncand);
+    if (x->prune_mode == SSGD_PRUNE_FUSED && !small) return SSGD_EINVAL;
     // table, histograms, selection state: one memset (the error flag is sticky until ssgd_status)
-    CU(cudaMemsetAsync(x->ws, 0, x->off_err, st), "memset workspace head");
+    CU(cudaMemsetAsync(x->ws, 0, small ? x->off_h19_c : x->off_err, st), "memset workspace head");
     x->launches++;
     float* merged = reinterpret_cast<float*>(x->ws + x->off_table);
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
     A.pending = pending_map(x);      // the previous step's deferred zero-out, applied while u and v stream past
+    A.wait_ns = x->wait_ns; A.withhold = x->withhold;
     // a table that cannot stay in L2 next to the stream is inserted a slice of rows at a time
     const size_t row_bytes = (size_t)x->c * 4;
     const int rows_fit = (int)(x->split_bytes / row_bytes);
@@ -577,6 +620,36 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);
+    if (small) {
+        // lines 9-13 in one cooperative kernel
+        SmallArgs T{};
+        T.table = merged; T.c = x->c; T.d = x->d; T.hp = x->hp; T.bk = x->bk; T.est = est;
+        SelBuffers sb = sel_buffers(x, false);
+        T.h1 = sb.h1; T.h2 = sb.h2; T.h3 = sb.h3;
+        T.st = reinterpret_cast<SmallState*>(x->ws + x->off_small);
+        T.map_a = reinterpret_cast<uint32_t*>(x->ws + x->off_maps);
+        T.map_b = reinterpret_cast<uint32_t*>(x->ws + x->off_maps + x->map_bytes);
+        T.xsum = A.xsum; T.cand_idx = cand; T.xs = reinterpret_cast<float*>(x->ws + x->off_xs);
+        T.ncand = (uint32_t)ncand; T.k = (uint32_t)x->k; T.out_idx = out_idx; T.out_val = out_val;
+        const bool deferred = x->zero_mode == SSGD_ZERO_DEFERRED;
+        T.pending = pending_map(x); T.pending_words = (x->d + 31) / 32; T.mark_pending = deferred ? 1 : 0;
+        T.u = x->u; T.v = x->v; T.ld = x->ld; T.W = x->W;
+        T.zero_inline = (!deferred && x->k * (int64_t)x->W <= SMALL_INLINE_ZERO_MAX) ? 1 : 0;
+        T.wait_ns = x->wait_ns; T.withhold = x->withhold;
+        T.errflag = reinterpret_cast<int32_t*>(x->ws + x->off_err);
+        if ((e = launch_small_tail(x, T, st))) return e;
+        if ((e = mark(x, 2, st)) || (e = mark(x, 3, st))) return e;
+        if (deferred) {
+            x->pending_dirty = true;
+        } else if (!T.zero_inline) {
+            CU(launch_pdl(st, k_zero, grid_for(x->k * (int64_t)x->W, 256, (int64_t)x->sm_count * 16), 256, 0, (const int32_t*)out_idx,
+                          x->k, x->u, x->v, x->ld, x->W, x->d), "launch k_zero");
+            LAUNCHED("k_zero");
+        }
+        if ((e = mark(x, 4, st))) return e;
+        if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
+        return SSGD_OK;
+    }
     const bool sparse = use_sparse(x, ncand);
     if (sparse) {
         if ((e = unsketch_select_sparse(x, merged, ncand, cand, st, A.xsum))) return e;
@@ -587,6 +660,18 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED, A.xsum, sparse))) return e;
     if ((e = mark(x, 4, st))) return e;
     if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
+    return SSGD_OK;
+}
+
+int ssgd_set_wait_limit_ns(ssgd_ctx* x, int64_t ns) {
+    if (!x || ns < 1000) return SSGD_EINVAL;
+    x->wait_ns = (uint64_t)ns;
+    return SSGD_OK;
+}
+
+int ssgd_test_withhold_block(ssgd_ctx* x, int32_t block_plus_one) {
+    if (!x || block_plus_one < 0) return SSGD_EINVAL;
+    x->withhold = block_plus_one;
     return SSGD_OK;
 }
 

@@ -17,8 +17,9 @@ LIB_PATH = os.path.join(_HERE, "libssgd.so")
 OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG, EPENDING = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
-PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT = 0, 1, 2, 3
+PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT, PRUNE_FUSED = 0, 1, 2, 3, 4
 ZERO_DEFERRED, ZERO_EAGER = 0, 1
+SCHED_AUTO, SCHED_COORDINATE_MAJOR, SCHED_WORKER_MAJOR = 0, 1, 2
 FMT_F16, FMT_BF16 = 0, 1
 MAX_R = 15
 
@@ -31,11 +32,14 @@ SIGNATURES = {
     "ssgd_set_hash_params": [_vp, _vp],
     "ssgd_set_insert_mode": [_vp, _i32],
     "ssgd_set_prune_mode": [_vp, _i32],
+    "ssgd_set_accumulate_schedule": [_vp, _i32],
     "ssgd_set_insert_split": [_vp, _i64],
     "ssgd_set_prune_sample_rank": [_vp, _i64],
     "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_set_zero_mode": [_vp, _i32],
+    "ssgd_set_wait_limit_ns": [_vp, _i64],
+    "ssgd_test_withhold_block": [_vp, _i32],
     "ssgd_flush": [_vp, _vp],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
     "ssgd_bind": [_vp, _vp, _vp, _i64, _vp, _sz, _i64],
@@ -160,6 +164,9 @@ class Ssgd:
     def set_prune_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_prune_mode(self._h, mode), "ssgd_set_prune_mode")
 
+    def set_accumulate_schedule(self, mode: int) -> None:
+        self._chk(self._lib.ssgd_set_accumulate_schedule(self._h, mode), "ssgd_set_accumulate_schedule")
+
     def set_prune_sample_rank(self, rank: int) -> None:
         self._chk(self._lib.ssgd_set_prune_sample_rank(self._h, rank), "ssgd_set_prune_sample_rank")
 
@@ -168,6 +175,12 @@ class Ssgd:
 
     def set_table_persistence(self, enable: bool) -> None:
         self._chk(self._lib.ssgd_set_table_persistence(self._h, 1 if enable else 0), "ssgd_set_table_persistence")
+
+    def set_wait_limit_ns(self, ns: int) -> None:
+        self._chk(self._lib.ssgd_set_wait_limit_ns(self._h, ns), "ssgd_set_wait_limit_ns")
+
+    def test_withhold_block(self, block_plus_one: int) -> None:
+        self._chk(self._lib.ssgd_test_withhold_block(self._h, block_plus_one), "ssgd_test_withhold_block")
 
     def set_zero_mode(self, mode: int) -> None:
         self._chk(self._lib.ssgd_set_zero_mode(self._h, mode), "ssgd_set_zero_mode")

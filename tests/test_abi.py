@@ -97,7 +97,8 @@ def test_unbound_context_refuses_to_run(lib):
 def test_mode_setters_check_their_argument(lib):
     eng = S.Ssgd(100, 5, 16, 10, 2, 1)
     for fn, good, bad in ((lib.ssgd_set_zero_mode, (S.ZERO_DEFERRED, S.ZERO_EAGER), (-1, 2)),
-                          (lib.ssgd_set_prune_mode, (S.PRUNE_AUTO, S.PRUNE_OFF, S.PRUNE_ON, S.PRUNE_EARLY_EXIT), (-1, 4)),
+                          (lib.ssgd_set_prune_mode, (S.PRUNE_AUTO, S.PRUNE_OFF, S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_FUSED), (-1, 5)),
+                          (lib.ssgd_set_accumulate_schedule, (S.SCHED_AUTO, S.SCHED_COORDINATE_MAJOR, S.SCHED_WORKER_MAJOR), (-1, 3)),
                           (lib.ssgd_set_insert_mode, (S.INSERT_AUTO, S.INSERT_GLOBAL, S.INSERT_SMEM, S.INSERT_TMA),
                            (-1, 4))):
         for m in good:

@@ -79,10 +79,12 @@ STAGE_CASES = [
 ]
 
 
+@pytest.mark.parametrize("sched", [S.SCHED_COORDINATE_MAJOR, S.SCHED_WORKER_MAJOR], ids=["coordinate_major", "worker_major"])
 @pytest.mark.parametrize("cfg", STAGE_CASES, ids=lambda c: f"{c.name}-d{c.d}-W{c.W}-r{c.r}-c{c.c}")
-def test_stage_calls_against_oracle(cuda_device, cfg):
+def test_stage_calls_against_oracle(cuda_device, cfg, sched):
     dev = cuda_device
     eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+    eng.set_accumulate_schedule(sched)
     orc = Oracle(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
     u, v = random_state(cfg, dev, 7)
     eng.bind(u, v, cfg.ncand)
@@ -162,13 +164,15 @@ def _lockstep_combinations():
     """Every insert variant with the dense candidate path, and every candidate path with the plain-load insert
     (the candidate path does not depend on the insert variant); the shared-memory insert only where the table fits."""
     names = {S.INSERT_TMA: "tma", S.INSERT_GLOBAL: "global", S.INSERT_SMEM: "smem",
-             S.PRUNE_ON: "filter", S.PRUNE_EARLY_EXIT: "early_exit", S.PRUNE_OFF: "dense"}
+             S.PRUNE_ON: "filter", S.PRUNE_EARLY_EXIT: "early_exit", S.PRUNE_OFF: "dense", S.PRUNE_FUSED: "fused"}
     out = []
     for cfg, steps in STEP_CASES:
         base = f"{cfg.name}-d{cfg.d}-W{cfg.W}-r{cfg.r}-c{cfg.c}"
         combos = [(S.INSERT_GLOBAL, p) for p in (S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF)] + [(S.INSERT_TMA, S.PRUNE_OFF)]
         if cfg.r * cfg.c * 4 <= 200 * 1024:
             combos.append((S.INSERT_SMEM, S.PRUNE_OFF))
+        if cfg.ncand <= 16384:
+            combos.append((S.INSERT_GLOBAL, S.PRUNE_FUSED))     # lines 9-13 in one cooperative kernel
         for mode, prune in combos:
             out.append(pytest.param(cfg, steps, mode, prune, id=f"{base}-{names[mode]}-{names[prune]}"))
     return out
@@ -189,7 +193,7 @@ def test_step_lockstep(cuda_device, cfg, steps, mode, prune):
         assert all(r["final_sym_diff_vs_unadopted"] == 0 for r in report)
 
 
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_FUSED])
 def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     cfg = wl.C2.scaled(d=10_001, W=3, c=256, ncand=700, k=300)
     eng, orc, u, v = make(cfg, cuda_device)
@@ -198,7 +202,7 @@ def test_all_zero_gradient_ties_break_by_index(cuda_device, prune):
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     assert idx.tolist() == list(range(cfg.k)) and (val == 0).all()
-    if prune != S.PRUNE_OFF:
+    if prune not in (S.PRUNE_OFF, S.PRUNE_FUSED):
         fell_back, survivors, bin_lo = eng.step_used_fallback()
         assert not fell_back and bin_lo == 0 and survivors == cfg.d   # nothing can be pruned; d ties ranked by index
 
@@ -238,7 +242,7 @@ def test_misjudged_threshold_reruns_without_pruning(cuda_device, prune):
     assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
 
 
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF])
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_FUSED])
 def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
     cfg = wl.C2.scaled(d=40_000, W=2, r=1, c=40_000, ncand=1000, k=400)
@@ -254,6 +258,100 @@ def test_heavy_ties_at_the_threshold(cuda_device, prune):
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     big = set(range(11, 500, 13))
     assert big <= set(idx.tolist())
+
+
+# ------------------------------------------------------------------------------------------------
+# lines 9-13 as one cooperative kernel (small problems)
+# ------------------------------------------------------------------------------------------------
+FUSED_CASES = [
+    # (configuration, steps, zero mode): table in one CTA's shared memory, in a cluster of 2, 4, 8, and too large for any
+    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 160 KiB: one CTA; zeros written in the kernel
+    (wl.C1.scaled(d=524_288, c=16_384, ncand=2000, k=1000), 2, S.ZERO_EAGER),             # C1's sketch: cluster of 2
+    (wl.C3.scaled(d=200_003, W=6, c=32_768, ncand=2000, k=1000), 3, S.ZERO_DEFERRED),     # cluster of 4
+    (wl.C4.scaled(d=270_002, W=3, c=65_536, ncand=1500, k=700), 3, S.ZERO_DEFERRED),      # cluster of 8
+    (wl.C2.scaled(d=250_001, W=2, c=200_000, ncand=16_384, k=16_384), 2, S.ZERO_DEFERRED),  # table read from L2; largest ncand; k = ncand
+    (wl.C2.scaled(d=150_002, W=17, r=3, c=999, ncand=9000, k=5000), 2, S.ZERO_EAGER),     # k*W too large for in-kernel zeros
+    (wl.C3.scaled(d=2_100_003, W=2, r=7, c=4001, ncand=5000, k=100), 2, S.ZERO_DEFERRED), # d above 2^21, real modulo
+    (wl.C2.scaled(d=7, W=3, r=5, c=16, ncand=7, k=3), 2, S.ZERO_EAGER),                   # fewer coordinates than threads
+]
+
+
+@pytest.mark.parametrize("cfg,steps,zero", FUSED_CASES, ids=lambda x: f"{x.name}-d{x.d}-W{x.W}-r{x.r}-c{x.c}" if hasattr(x, "name") else str(x))
+def test_fused_tail_lockstep(cuda_device, cfg, steps, zero):
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_FUSED)
+    eng.set_zero_mode(zero)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    n0 = eng.launch_count()
+    for t in range(steps):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o, flush=(t == steps - 1))
+    # memset + accumulate + tail (+ k_zero when k*W is too large for the tail) per step; check_step adds the dense
+    # stage call (5 launches) and the last one a flush
+    per_step = 3 + (1 if zero == S.ZERO_EAGER and cfg.k * cfg.W > 65536 else 0)
+    assert eng.launch_count() - n0 == steps * (per_step + 5) + 1
+
+
+def test_fused_tail_is_refused_where_it_does_not_apply(cuda_device):
+    cfg = wl.C2.scaled(d=400_000, W=2, c=4096, ncand=20_000, k=100)       # more candidates than the last block holds
+    eng, _, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_FUSED)
+    g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=cuda_device)
+    ov = torch.empty(cfg.k, device=cuda_device)
+    with pytest.raises(S.SsgdError) as e:
+        eng.step(g, cfg.rho, cfg.ncand, oi, ov)
+    assert e.value.code == S.EINVAL
+    eng.set_prune_mode(S.PRUNE_AUTO)                                      # AUTO takes another path
+    eng.step(g, cfg.rho, cfg.ncand, oi, ov)
+    assert eng.status() == S.OK
+
+
+def test_a_grid_barrier_wait_that_runs_out_is_reported_and_nothing_hangs(cuda_device):
+    """One block of the cooperative tail is withheld (it returns before the first grid barrier), so the others'
+    bounded waits run out after the configured limit: the kernel returns, ssgd_status reports SSGD_EDEVICE once,
+    and the next step on the same context is correct again."""
+    cfg = wl.C2.scaled(d=300_001, W=3, c=8192, ncand=3000, k=1500)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_FUSED)
+    eng.set_zero_mode(S.ZERO_EAGER)
+    st = wl.Structure(cfg, cuda_device)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=cuda_device)
+    ov = torch.empty(cfg.k, device=cuda_device)
+    eng.set_wait_limit_ns(200_000)                                        # 0.2 ms
+    eng.test_withhold_block(1)
+    eng.step(wl.gradients(st, 0), cfg.rho, cfg.ncand, oi, ov)
+    assert eng.status() == S.EDEVICE
+    assert eng.status() == S.OK
+    eng.test_withhold_block(0)
+    eng.set_wait_limit_ns(2_000_000_000)
+    u.zero_(); v.zero_()
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    check_step(orc, eng, wl.gradients(st, 1), cfg.rho, cfg.ncand, u_o, v_o)
+
+
+def test_a_pipeline_wait_that_runs_out_is_reported_and_nothing_hangs(cuda_device):
+    """The bulk-copy accumulate kernel's bounded waits: the producer of one CTA is withheld (it issues no copy, so
+    nothing is in flight), its consumers' waits run out after the configured limit, the CTA returns, the other
+    CTAs finish normally; ssgd_status reports SSGD_EDEVICE once and the context stays usable."""
+    cfg = wl.C2.scaled(d=400_003, W=5, c=4096, ncand=2000, k=1000)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_insert_mode(S.INSERT_TMA)
+    eng.set_prune_mode(S.PRUNE_OFF)
+    st = wl.Structure(cfg, cuda_device)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=cuda_device)
+    ov = torch.empty(cfg.k, device=cuda_device)
+    eng.set_wait_limit_ns(200_000)
+    eng.test_withhold_block(1)
+    eng.step(wl.gradients(st, 0), cfg.rho, cfg.ncand, oi, ov)
+    assert eng.status() == S.EDEVICE
+    assert eng.status() == S.OK
+    eng.test_withhold_block(0)
+    eng.set_wait_limit_ns(2_000_000_000)
+    eng.flush()
+    u.zero_(); v.zero_()
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    check_step(orc, eng, wl.gradients(st, 1), cfg.rho, cfg.ncand, u_o, v_o)
 
 
 def test_row_split_insert(cuda_device):
