@@ -81,9 +81,8 @@ extern "C" {
 #define SSGD_PRUNE_EARLY_EXIT 3
 /* FUSED: lines 9-13 run as ONE cooperative kernel (dense estimates, exact radix select behind grid barriers, the
  * second round, the final top-k and line 13 by the last block), for problems so small that a chain of short
- * launches costs more than the work: needs d <= 2^22 and ncand <= 16384 (SSGD_EINVAL from ssgd_step otherwise).  If
- * the r x c table fits the shared memory of a cluster of up to 8 thread blocks, the estimates read it from there.
- * AUTO takes this path for d <= 2^21 when it applies.  The results are those of the other modes. */
+ * launches costs more than the work: needs d <= 2^22 and ncand <= 16384 (SSGD_EINVAL from ssgd_step otherwise).
+ * AUTO takes this path for d <= 2^21 and ncand <= 4096.  The results are those of the other modes. */
 #define SSGD_PRUNE_FUSED 4
 
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
@@ -104,10 +103,6 @@ int ssgd_get_hash_params(const ssgd_ctx* ctx, uint32_t* out4r);
 int ssgd_set_hash_params(ssgd_ctx* ctx, const uint32_t* in4r);
 int ssgd_set_insert_mode(ssgd_ctx* ctx, int32_t mode);
 int ssgd_set_prune_mode(ssgd_ctx* ctx, int32_t mode);
-/* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
- * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
- * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
- * which leaves tables up to that size untouched). */
 /* When ssgd_step applies Algorithm 3 line 13 (u, v <- 0 at the k chosen coordinates).
  * DEFERRED (default): ssgd_step only marks the chosen coordinates in a d-bit map inside the workspace; the NEXT
  * ssgd_step reads marked coordinates of u and v as +0 inside the kernel that streams all of u and v anyway, so
@@ -132,6 +127,10 @@ int ssgd_test_withhold_block(ssgd_ctx* ctx, int32_t block_plus_one);
 /* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Cheap when
  * nothing is pending (one pass over d/8 bytes). */
 int ssgd_flush(ssgd_ctx* ctx, void* stream);
+/* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
+ * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
+ * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
+ * which leaves tables up to that size untouched). */
 int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
 /* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
  * (cudaLimitPersistingL2CacheSize of this process's CUDA context is raised to the table size, capped by the
@@ -144,6 +143,12 @@ int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
  * pruned), out[3] = 1 if a folded bucket bitmap was too dense and the first pass read the table instead,
  * out[4] = set bits of the folded bitmap (0 if the bitmap is not folded). */
 int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out5);
+/* Diagnostics of the last ssgd_step that took the FUSED tail (waits for the stream): nanoseconds since the tail
+ * kernel's first thread block started, at 12 points -- [0] start, [1] table copied to shared memory (if it is),
+ * [2] its estimates done, [3]-[5] past the three grid barriers (all of thread block 0); of the block that finishes
+ * the step alone: [6] it knows it is the last, [11] mark counts scanned, [7] candidates emitted, [8] second round
+ * done, [9] final threshold known, [10] end.  -1 where no stamp was taken. */
+int ssgd_tail_trace(ssgd_ctx* ctx, void* stream, int64_t* out12);
 /* For tests and diagnostics: the rank (from the top) in the sample's histogram that sets the prune threshold;
  * 0 = derive it from ncand (mean + 6 sigma + 16).  A rank of 1 puts the threshold at the largest sampled
  * estimate, which forces the unpruned rerun. */

@@ -44,14 +44,11 @@ struct AccumArgs {
     int32_t withhold;    // test hook (bulk-copy pipeline only): the producer of CTA (withhold - 1) issues nothing
 };
 
-#ifndef SSGD_KT_STAGES
-#define SSGD_KT_STAGES 6
-#endif
 constexpr int KT_CONSUMER_WARPS = 8;
 constexpr int KT_CONSUMERS = KT_CONSUMER_WARPS * 32;
 constexpr int KT_THREADS = KT_CONSUMERS + 32;       // + one producer warp
 constexpr int KT_TC = KT_CONSUMERS * 4;             // coordinates per tile: one float4 per consumer thread
-constexpr int KT_STAGES = SSGD_KT_STAGES;
+constexpr int KT_STAGES = 6;                        // ring slots of 12 KiB each
 
 struct alignas(128) KtSlot { float g[KT_TC]; float u[KT_TC]; float v[KT_TC]; };
 struct KtShared {

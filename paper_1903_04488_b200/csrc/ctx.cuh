@@ -51,15 +51,15 @@ struct ssgd_ctx {
     bool pending_dirty;     // a deferred ssgd_step has run since the last flush: u, v may await their zero-out
     size_t off_hm;
     int32_t prune_mode;
-    size_t persist_bytes;
-    size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel   // > 0: launches that touch the table carry an L2 access-policy window of this size
+    size_t persist_bytes;   // > 0: launches that touch the table carry an L2 access-policy window of this size
+    size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel
     size_t off_xsum;        // per-coordinate sums over the workers of the new v, written by ssgd_step's accumulate kernel
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;
     // device facts
     int device; int sm_count; int max_smem_optin;
     int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
-    int small_grid, small_cs; size_t small_smem;   // launch shape of the one-kernel tail (small_grid 0 = not queried yet)
+    int small_grid;         // CTAs of the one-kernel tail (0 = not queried yet)
     uint64_t wait_ns;       // limit of every device-side wait (grid barriers, mbarriers)
     int32_t withhold;       // test hook: this CTA (1-based; 0 = none) never arrives, so the others' waits run out
     int64_t launches;
@@ -93,11 +93,7 @@ inline int cuda_fail(ssgd_ctx* x, cudaError_t e, const char* what) {
     } while (0)
 
 // Launch with programmatic stream serialization: the kernel may become resident while its predecessor
-// drains; it orders itself with pdl_wait().  SSGD_NO_PDL=1 in the environment turns the attribute off.
-inline bool pdl_enabled() {
-    static const bool on = [] { const char* e = std::getenv("SSGD_NO_PDL"); return !(e && e[0] == '1'); }();
-    return on;
-}
+// drains; it orders itself with pdl_wait().
 
 // An L2 access-policy window for one launch: accesses inside [base, base+bytes) are kept (persisting),
 // everything else the kernel touches is treated as streaming.
@@ -112,11 +108,9 @@ cudaError_t launch_pdl_w(cudaStream_t st, L2Window win, void (*kern)(P...), int 
     cfg.stream = st;
     cudaLaunchAttribute at[2];
     int n = 0;
-    if (pdl_enabled()) {
-        at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[n].val.programmaticStreamSerializationAllowed = 1;
-        ++n;
-    }
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
     if (win.base && win.bytes) {
         at[n].id = cudaLaunchAttributeAccessPolicyWindow;
         at[n].val.accessPolicyWindow.base_ptr = const_cast<void*>(win.base);

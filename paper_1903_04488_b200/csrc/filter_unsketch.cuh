@@ -33,13 +33,8 @@ namespace ssgd {
 // Measured on B200 (C2; sample + bitmap + filter + the skipped rerun launch): 256 threads x 4 coordinates per
 // iteration 0.092 ms; 512 x 1, 2, 4: 0.073, 0.071, 0.073; 1024 x 1, 2: 0.070, 0.067.  With a folded bitmap the
 // kernel needs more than the 64 registers that 1024 threads leave it (d = 2e7, c = 2^20: 0.41 ms against 0.26 ms).
-#ifndef SSGD_FILTER_THREADS
-#define SSGD_FILTER_THREADS 512
-#endif
-#ifndef SSGD_FILTER_NC
-#define SSGD_FILTER_NC 2
-#endif
-constexpr int FILTER_THREADS = SSGD_FILTER_THREADS;
+constexpr int FILTER_THREADS = 512;
+constexpr int FILTER_NC = 2;                             // coordinates per loop iteration (independent lookups)
 constexpr int FILTER_WARPS = FILTER_THREADS / 32;
 constexpr int FILTER_QUEUE = 64;                         // entries per warp queue (at most 31 + 32 are ever held)
 constexpr int FILTER_MAX_WORDS = 49152;                  // 192 KiB of bitmap per SM (+ 16 KiB of queues + 16 KiB histogram)
@@ -109,9 +104,7 @@ __device__ __forceinline__ float binomial_tail(int r, int need, float p) {
 // 0.77 (same, ncand doubled) 2.79 / 2.89; 0.88 (d = 9e7, c = 1e6, 4 per bit) 4.82 / 4.91; 0.90 (d = 9e7, c = 2^22,
 // 16 per bit, ncand = 5e4) 7.49 / 7.85; 0.96 (d = 2e7, c = 2^20, ncand = 1.6e6) 2.65 / 2.60; 0.99 (d = 9e7, c = 2^22,
 // ncand = 2e5) 7.97 / 7.99; r = 15, 0.95 (d = 9e7, c = 180,000, 2 per bit) 16.7 / 12.5.
-#ifndef SSGD_FILTER_MAX_PASS
-#define SSGD_FILTER_MAX_PASS 0.93f
-#endif
+constexpr float FILTER_MAX_PASS = 0.93f;
 
 // One thread per folded word: 32 folded bits, each the OR of 2^s consecutive bits of the full bitmap.  The last
 // block to finish turns the density of the folded bitmap into the decision between the two first-pass kernels.
@@ -147,7 +140,7 @@ k_bitmap_fold(const FilterArgs F) {
     if (s_last && threadIdx.x == 0) {
         const float bits = (float)F.r * (float)((F.A.c + (1 << s) - 1) >> s);
         const float p = fminf(1.f, (float)__ldcg(&F.A.sp.state->fold_ones) / bits);
-        F.A.sp.state->use_table = binomial_tail(F.r, (F.r + 1) / 2, p) > SSGD_FILTER_MAX_PASS ? 1u : 0u;
+        F.A.sp.state->use_table = binomial_tail(F.r, (F.r + 1) / 2, p) > FILTER_MAX_PASS ? 1u : 0u;
     }
 }
 
@@ -263,7 +256,7 @@ k_unsketch_filter(const FilterArgs F) {
 
     // this thread's run of consecutive coordinates
     const uint32_t total_threads = gridDim.x * FILTER_THREADS;
-    constexpr int NC = SSGD_FILTER_NC;                   // coordinates per loop iteration (independent lookups)
+    constexpr int NC = FILTER_NC;
     const uint32_t per = (uint32_t)((A.d + total_threads - 1) / total_threads + NC - 1) / NC * NC;
     const uint32_t gtid = blockIdx.x * FILTER_THREADS + threadIdx.x;
     const uint64_t begin64 = (uint64_t)gtid * per;

@@ -8,7 +8,7 @@ template <int R, bool POW2>
 int launch_unsketch_t(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
     const int64_t groups = (A.d + K3_NC - 1) / K3_NC;
     // a few blocks per SM: each block pays one histogram flush
-    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * SSGD_K3_GRID);
+    const int grid = grid_for(groups, K3_THREADS, (int64_t)x->sm_count * K3_GRID);
     CU(launch_pdl(st, k_unsketch<R, POW2>, grid, K3_THREADS, 0, A), "launch k_unsketch");
     LAUNCHED("k_unsketch");
     return SSGD_OK;
@@ -32,7 +32,7 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
     CU(launch_pdl(st, k_unsketch_sample<R, POW2>, grid_for(windows, SEL_THREADS, (int64_t)x->sm_count * 4), SEL_THREADS, 0, A),
        "launch k_unsketch_sample");
     LAUNCHED("k_unsketch_sample");
-    const int pruned_grid = grid_for((A.d + SSGD_PRUNED_NC - 1) / SSGD_PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * SSGD_PRUNED_GRID);
+    const int pruned_grid = grid_for((A.d + PRUNED_NC - 1) / PRUNED_NC, SEL_THREADS, (int64_t)x->sm_count * PRUNED_GRID);
     if (use_filter(x)) {
         FilterArgs F;
         F.A = A;

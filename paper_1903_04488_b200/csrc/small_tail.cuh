@@ -5,10 +5,11 @@
 //
 //   phase 1   every CTA estimates its share of the coordinates (Algorithm 4 estimate: median of the r signed
 //             buckets), stores est[i] and counts the top 12 bits of |est| in a shared-memory histogram -> H1.
-//             If the r x c table fits the shared memory of a thread-block cluster (2, 4 or 8 CTAs), each CTA first
-//             copies its column slice of every row into shared memory and the r lookups per coordinate are
-//             distributed-shared-memory loads instead of scattered reads of L2: the dense unsketch is bound by
-//             the rate of scattered 32-byte sectors (about one per clock per SM), shared memory is not.
+//             If the whole r x c table fits one CTA's shared memory and the CTA has clearly more lookups to do
+//             than the table has entries, it copies the table first and looks up there (3.5 random 4-byte reads
+//             per clock per SM against 1.1 from L2, measured).  A table split over the shared memory of a
+//             thread-block cluster was measured and dropped: random reads of another CTA's shared memory run at
+//             0.7 per clock per SM in a cluster of 2 and 0.4 in clusters of 4 to 16 -- slower than L2.
 //   barrier   H1 complete: every CTA finds the first threshold digit d1 for itself
 //   phase 2   histogram H2 of the next 11 key bits among the items inside d1
 //   barrier   -> second digit d2
@@ -22,9 +23,7 @@
 //             line 13 as marks in the pending map (deferred) or as zeros written to u and v (eager, small k*W).
 //
 // Every wait at a barrier is bounded: after `wait_ns` the waiting CTA records ERR_TIMEOUT in the error word,
-// raises the abort flag so that the others stop waiting too, and returns.  All use of other CTAs' shared memory
-// lies before the first barrier and is closed by a cluster barrier, so a CTA that gives up leaves nobody reading
-// memory that is gone.
+// raises the abort flag so that the others stop waiting too, and returns.
 #pragma once
 #include <stdint.h>
 
@@ -45,7 +44,10 @@ struct SmallState {          // zeroed before the step
     uint32_t bar;            // arrivals at the grid barriers (monotonic: barrier n completes at n * gridDim.x)
     uint32_t abort;          // a wait gave up
     uint32_t ticket;         // CTAs that finished phase 4
-    uint32_t pad[13];
+    uint32_t pad;
+    uint64_t trace[12];      // globaltimer stamps of CTA 0 (slots 0-5) and of the last CTA (6-10), for diagnostics
+    // marks per stretch of map words (stretch w = the words warp w of the last CTA walks), counted in phase 4
+    uint32_t chunk_a[ST_WARPS], chunk_b[ST_WARPS];
 };
 
 struct SmallArgs {
@@ -64,8 +66,7 @@ struct SmallArgs {
     int32_t mark_pending;
     float* u; float* v; int64_t ld; int32_t W;  // eager line 13 written here when zero_inline != 0
     int32_t zero_inline;
-    int32_t use_smem;        // 1: table slices in the cluster's shared memory
-    int32_t col_shift;       // use_smem: columns [rank << col_shift, (rank + 1) << col_shift) of every row live in CTA `rank`
+    int32_t use_smem;        // 1: every CTA copies the table into its shared memory and looks up there
     uint64_t wait_ns;        // limit of a barrier wait
     int32_t withhold;        // test hook: CTA (withhold - 1) leaves before the first barrier, so the others' wait runs out
     int32_t* errflag;
@@ -73,23 +74,6 @@ struct SmallArgs {
 
 #ifdef __CUDACC__
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// fp32 at byte offset `off` of the dynamic shared memory of CTA `rank` of this cluster
-__device__ __forceinline__ float dsmem_load(uint32_t local_base, uint32_t off, uint32_t rank) {
-    uint32_t remote;
-    float v;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_base + off), "r"(rank));
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(remote) : "memory");
-    return v;
-}
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -183,34 +167,30 @@ k_small_tail(const SmallArgs A) {
     const int64_t groups = (A.d + 3) >> 2;
     const int64_t gstride = (int64_t)gridDim.x * ST_THREADS;
     const int64_t gtid = (int64_t)blockIdx.x * ST_THREADS + tid;
-    const uint32_t crank = A.use_smem ? cluster_ctarank() : 0u;
-    const uint32_t dyn_base = (uint32_t)__cvta_generic_to_shared(st_dyn);
-    const uint32_t cols = 1u << A.col_shift;               // columns of a row held by one CTA
+    const int64_t nwords = (A.d + 31) >> 5;                // words of a coordinate map
+    const int64_t per = ((nwords + ST_WARPS - 1) / ST_WARPS + 127) & ~(int64_t)127;   // map words per stretch: whole 512-byte rows
+    auto stamp = [&](int slot, bool mine) { if (mine && tid == 0) A.st->trace[slot] = global_ns(); };
+    const bool first_cta = blockIdx.x == 0;
+    stamp(0, first_cta);
 
     // ---------------- phase 1: table slice -> shared memory; estimates, H1 ----------------
     for (int b = tid; b < H1_BINS; b += ST_THREADS) sh.hist[b] = 0;
     if (A.pending)
         for (int64_t t = gtid; t < A.pending_words; t += gstride) A.pending[t] = 0u;   // consumed by the accumulate kernel
+    const float* slice = reinterpret_cast<const float*>(st_dyn);
     if (A.use_smem) {
-        float* slice = reinterpret_cast<float*>(st_dyn);
-        const int64_t c0 = (int64_t)crank << A.col_shift;
-        const int64_t n = c0 < A.c ? (A.c - c0 < (int64_t)cols ? A.c - c0 : (int64_t)cols) : 0;   // my columns of a row
+        float* dst = reinterpret_cast<float*>(st_dyn);
+        const int64_t n = (int64_t)R * A.c;
+        for (int64_t b0 = tid; b0 < n; b0 += ST_THREADS * 8) {
+            float t[8];
 #pragma unroll
-        for (int j = 0; j < R; ++j) {
-            const float* src = A.table + (int64_t)j * A.c + c0;
-            float* dst = slice + (int64_t)j * cols;
-            for (int64_t b0 = tid; b0 < n; b0 += ST_THREADS * 8) {
-                float t[8];
+            for (int s8 = 0; s8 < 8; ++s8) t[s8] = b0 + s8 * ST_THREADS < n ? __ldcg(A.table + b0 + s8 * ST_THREADS) : 0.f;
 #pragma unroll
-                for (int s = 0; s < 8; ++s) t[s] = b0 + s * ST_THREADS < n ? __ldcg(src + b0 + s * ST_THREADS) : 0.f;
-#pragma unroll
-                for (int s = 0; s < 8; ++s) if (b0 + s * ST_THREADS < n) dst[b0 + s * ST_THREADS] = t[s];
-            }
+            for (int s8 = 0; s8 < 8; ++s8) if (b0 + s8 * ST_THREADS < n) dst[b0 + s8 * ST_THREADS] = t[s8];
         }
-        cluster_sync_all();                                // every slice of the cluster is in place
-    } else {
-        __syncthreads();
     }
+    __syncthreads();
+    stamp(1, first_cta);
     for (int64_t q = gtid; q < groups; q += gstride) {
         const int64_t i0 = q << 2;
         float rowv[4][R];
@@ -220,11 +200,8 @@ k_small_tail(const SmallArgs A) {
             row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const uint32_t b = hb[e] & P31;
-                float t;
-                if (A.use_smem) t = dsmem_load(dyn_base, ((uint32_t)j * cols + (b & (cols - 1u))) * 4u, b >> A.col_shift);
-                else t = table_load(A.table + (int64_t)j * A.c + b);
-                rowv[e][j] = apply_sign(t, hb[e]);
+                const int64_t at = (int64_t)j * A.c + (hb[e] & P31);
+                rowv[e][j] = apply_sign(A.use_smem ? slice[at] : table_load(A.table + at), hb[e]);
             }
         }
         float m[4];
@@ -243,23 +220,34 @@ k_small_tail(const SmallArgs A) {
     }
     __syncthreads();
     flush_hist<H1_BINS>(sh.hist, A.h1);
-    if (A.use_smem) cluster_sync_all();                    // nobody reads this CTA's slice any more
     if (A.withhold && (int)blockIdx.x == A.withhold - 1) return;
+    stamp(2, first_cta);
     if (!small_grid_barrier(A, 1, &s_flag)) return;
+    stamp(3, first_cta);
 
-    // keys of this thread's coordinates, re-read from est (L2) in each of the later phases
+    // keys of this thread's coordinates, re-read from est (L2) in each of the later phases, four groups per round
+    // trip (the loads are unconditional so that they are all in flight before the first is used)
     auto for_my_keys = [&](auto&& f) {
-        for (int64_t q = gtid; q < groups; q += gstride) {
-            const int64_t i0 = q << 2;
-            uint32_t key[4];
-            if (i0 + 3 < A.d) {
-                const float4 t = __ldcg(reinterpret_cast<const float4*>(A.est + i0));
-                key[0] = key_of(t.x); key[1] = key_of(t.y); key[2] = key_of(t.z); key[3] = key_of(t.w);
-            } else {
+        for (int64_t q0 = gtid; q0 < groups; q0 += 4 * gstride) {
+            float4 t[4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) key[e] = i0 + e < A.d ? key_of(__ldcg(A.est + i0 + e)) : NO_ITEM;
+            for (int b = 0; b < 4; ++b) {
+                const int64_t i0 = (q0 + b * gstride) << 2;
+                t[b] = __ldcg(reinterpret_cast<const float4*>(A.est + (i0 + 3 < A.d ? i0 : 0)));
             }
-            f(i0, key);
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int64_t i0 = (q0 + b * gstride) << 2;
+                if (i0 >= A.d) continue;
+                uint32_t key[4];
+                if (i0 + 3 < A.d) {
+                    key[0] = key_of(t[b].x); key[1] = key_of(t[b].y); key[2] = key_of(t[b].z); key[3] = key_of(t[b].w);
+                } else {                                   // the ragged last group
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) key[e] = i0 + e < A.d ? key_of(__ldcg(A.est + i0 + e)) : NO_ITEM;
+                }
+                f(i0, key);
+            }
         }
     };
 
@@ -276,6 +264,7 @@ k_small_tail(const SmallArgs A) {
     __syncthreads();
     flush_hist<H2_BINS>(sh.hist, A.h2);
     if (!small_grid_barrier(A, 2, &s_flag)) return;
+    stamp(4, first_cta);
 
     // ---------------- phase 3: third digit ----------------
     block_find_from_top<H2_BINS>(A.h2, rem1, sh, d2, rem2);
@@ -290,6 +279,7 @@ k_small_tail(const SmallArgs A) {
     __syncthreads();
     flush_hist<H3_BINS>(sh.hist, A.h3);
     if (!small_grid_barrier(A, 3, &s_flag)) return;
+    stamp(5, first_cta);
 
     // ---------------- phase 4: marks ----------------
     block_find_from_top<H3_BINS>(A.h3, rem2, sh, d3, rem3);
@@ -303,50 +293,89 @@ k_small_tail(const SmallArgs A) {
             eq |= (key[e] == T ? 1u : 0u) << e;
         }
         const int sh4 = (int)(i0 & 31);                    // a group of four never straddles a map word
-        if (gt) atomicOr(A.map_a + (i0 >> 5), gt << sh4);
-        if (eq) atomicOr(A.map_b + (i0 >> 5), eq << sh4);
+        if (gt) { atomicOr(A.map_a + (i0 >> 5), gt << sh4); atomicAdd(&A.st->chunk_a[(i0 >> 5) / per], (uint32_t)__popc(gt)); }
+        if (eq) { atomicOr(A.map_b + (i0 >> 5), eq << sh4); atomicAdd(&A.st->chunk_b[(i0 >> 5) / per], (uint32_t)__popc(eq)); }
     });
     if (!block_is_last(&A.st->ticket, sh)) return;
 
     // ---------------- phase 5 (one CTA): candidates, second round, final top-k, line 13 ----------------
+    stamp(6, true);
     int32_t* cand_s = reinterpret_cast<int32_t*>(st_dyn);
     float* xs_s = reinterpret_cast<float*>(st_dyn) + A.ncand;
-    const int64_t nwords = (A.d + 31) >> 5;
-    const int64_t per = ((nwords + ST_THREADS - 1) / ST_THREADS + 3) & ~(int64_t)3;   // words per thread, a multiple of 4
-    const int64_t w_lo = (int64_t)tid * per, w_hi = w_lo + per < nwords ? w_lo + per : nwords;
-    uint32_t ca = 0, cb = 0;
-    for (int64_t w = w_lo; w < w_hi; w += 4) {
-        if (w + 3 < nwords) {
-            const uint4 a = __ldcg(reinterpret_cast<const uint4*>(A.map_a + w)), b = __ldcg(reinterpret_cast<const uint4*>(A.map_b + w));
-            ca += __popc(a.x) + __popc(a.y) + __popc(a.z) + __popc(a.w);
-            cb += __popc(b.x) + __popc(b.y) + __popc(b.z) + __popc(b.w);
-        } else {
-            for (int64_t t = w; t < w_hi; ++t) { ca += __popc(__ldcg(A.map_a + t)); cb += __popc(__ldcg(A.map_b + t)); }
+    // Warp w walks stretch w of the maps (how many marks each stretch holds was counted in phase 4), 128 words per
+    // step: lane l holds words 4l .. 4l+3 of the step, so that every load instruction reads 512 contiguous bytes
+    // Order inside a stretch is (step, lane, word, bit) = ascending coordinate.  Measured at d = 2^20 (2 x 128 KiB of
+    // maps, 2,000 marks): 13 us, of which 1.2 us are the loads -- the rest is instruction issue on this one SM (about
+    // 300 warp instructions per step and warp); the same loop not unrolled (batch in local memory) takes 20 us.
+    const int lane = tid & 31, warp = tid >> 5;
+    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) cand_s[m] = 0;     // consistent histograms fill every slot
+    uint32_t run_a = 0, run_b = 0, mine_a = 0, mine_b = 0;
+    {
+        const uint32_t ca = lane < ST_WARPS ? __ldcg(&A.st->chunk_a[lane]) : 0u;
+        const uint32_t cb = lane < ST_WARPS ? __ldcg(&A.st->chunk_b[lane]) : 0u;
+        for (int w = 0; w < ST_WARPS; ++w) {
+            const uint32_t ta = __shfl_sync(0xFFFFFFFFu, ca, w), tb = __shfl_sync(0xFFFFFFFFu, cb, w);
+            if (w < warp) { run_a += ta; run_b += tb; }
+            if (w == warp) { mine_a = ta; mine_b = tb; }
         }
     }
-    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) cand_s[m] = 0;     // consistent histograms fill every slot
-    uint32_t run_a, run_b;
-    block_excl_scan2(ca, cb, s_warp_a, s_warp_b, run_a, run_b);
-    if (ca | cb) {
-        for (int64_t w = w_lo; w < w_hi; ++w) {
-            const uint32_t wa = __ldcg(A.map_a + w), wb = __ldcg(A.map_b + w);
-            uint32_t bits = wa | wb;
-            while (bits) {
-                const int bit = __ffs(bits) - 1;
-                bits &= bits - 1;
-                uint32_t slot = 0xFFFFFFFFu;
-                if ((wa >> bit) & 1u) { slot = run_a + (run_b < Q ? run_b : Q); ++run_a; }
-                else { if (run_b < Q) slot = run_a + run_b; ++run_b; }
-                if (slot < A.ncand) {
-                    const int32_t coord = (int32_t)((w << 5) + bit);
-                    cand_s[slot] = coord;
-                    A.cand_idx[slot] = coord;
+    __syncthreads();                                       // cand_s is cleared before any warp fills its slots
+    stamp(11, true);
+    const int64_t w_lo = (int64_t)warp * per, w_hi = w_lo + per < nwords ? w_lo + per : nwords;
+    if (mine_a | mine_b) {                                 // warp-uniform
+        for (int64_t w0 = w_lo; w0 < w_hi; w0 += 8 * 128) {
+            // eight steps per round trip to L2.  The loads are unconditional: the maps are padded with zero words to
+            // a multiple of 64 and rows beyond the stretch's end are masked out below
+            uint4 a4[8], b4[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int64_t w = w0 + q * 128 + 4 * lane;
+                const int64_t wl = w < w_hi ? w : w_lo;
+                a4[q] = __ldcg(reinterpret_cast<const uint4*>(A.map_a + wl));
+                b4[q] = __ldcg(reinterpret_cast<const uint4*>(A.map_b + wl));
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int64_t w = w0 + q * 128 + 4 * lane;
+                uint32_t wa[4] = {a4[q].x, a4[q].y, a4[q].z, a4[q].w}, wb[4] = {b4[q].x, b4[q].y, b4[q].z, b4[q].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (w + e >= w_hi) { wa[e] = 0u; wb[e] = 0u; }
+                const uint32_t na = __popc(wa[0]) + __popc(wa[1]) + __popc(wa[2]) + __popc(wa[3]);
+                const uint32_t nb = __popc(wb[0]) + __popc(wb[1]) + __popc(wb[2]) + __popc(wb[3]);
+                if (__ballot_sync(0xFFFFFFFFu, (na | nb) != 0u) == 0u) continue;        // an empty step
+                uint32_t packed = na | (nb << 16), incl = packed;                        // at most 128 marks per lane
+#pragma unroll
+                for (int off = 1; off < 32; off <<= 1) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                    if (lane >= off) incl += o;
                 }
+                const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                uint32_t a = run_a + ((incl - packed) & 0xFFFFu), b = run_b + ((incl - packed) >> 16);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    uint32_t bits = wa[e] | wb[e];
+                    while (bits) {
+                        const int bit = __ffs(bits) - 1;
+                        bits &= bits - 1;
+                        uint32_t slot = 0xFFFFFFFFu;
+                        if ((wa[e] >> bit) & 1u) { slot = a + (b < Q ? b : Q); ++a; }
+                        else { if (b < Q) slot = a + b; ++b; }
+                        if (slot < A.ncand) {
+                            const int32_t coord = (int32_t)(((w + e) << 5) + bit);
+                            cand_s[slot] = coord;
+                            A.cand_idx[slot] = coord;
+                        }
+                    }
+                }
+                run_a += tot & 0xFFFFu;
+                run_b += tot >> 16;
             }
         }
     }
     for (int b = tid; b < H1_BINS; b += ST_THREADS) sh.hist[b] = 0;
     __syncthreads();
+    stamp(7, true);
     // line 10: one read per candidate of the sums the accumulate kernel left
     for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) {
         const uint32_t i = (uint32_t)cand_s[m];
@@ -356,6 +385,7 @@ k_small_tail(const SmallArgs A) {
         atomicAdd(&sh.hist[key_of(x) >> H1_SHIFT], 1u);
     }
     __syncthreads();
+    stamp(8, true);
     // line 11: exact top-k of |xs| among the candidates, all in shared memory
     uint32_t e1, r1, e2, r2, e3, r3;
     smem_find_from_top<H1_BINS>(sh.hist, A.k, s_warp_a, s_found, e1, r1);
@@ -377,6 +407,7 @@ k_small_tail(const SmallArgs A) {
     __syncthreads();
     smem_find_from_top<H3_BINS>(sh.hist, r2, s_warp_a, s_found, e3, r3);
     const uint32_t T2 = (e1 << H1_SHIFT) | (e2 << H2_SHIFT) | e3, Q2 = r3;
+    stamp(9, true);
     // ordered emit: thread t owns the candidates [t * per2, (t + 1) * per2)
     const uint32_t per2 = (A.ncand + ST_THREADS - 1) / ST_THREADS;
     const uint32_t m_lo = tid * per2 < A.ncand ? tid * per2 : A.ncand;
@@ -404,6 +435,8 @@ k_small_tail(const SmallArgs A) {
                 for (int64_t w = 0; w < A.W; ++w) { A.u[w * A.ld + i] = 0.0f; A.v[w * A.ld + i] = 0.0f; }
         }
     }
+    __syncthreads();
+    stamp(10, true);
 }
 
 #endif  // __CUDACC__

@@ -30,10 +30,7 @@
 namespace ssgd {
 
 // measured at C2/C3/C4: 1/32 0.210/0.345/1.524 ms (sample + early-exit kernel), 1/64 0.207, 1/128 0.205, 1/256 0.208/0.338/1.467
-#ifndef SSGD_SAMPLE_SHIFT
-#define SSGD_SAMPLE_SHIFT 6
-#endif
-constexpr int SPARSE_SAMPLE_SHIFT = SSGD_SAMPLE_SHIFT;   // one float4 group in 2^shift is sampled
+constexpr int SPARSE_SAMPLE_SHIFT = 6;   // one float4 group in 2^shift is sampled
 
 struct SparseState {                              // zeroed before the step
     uint32_t bin_lo;       // prune threshold: H1 bin index; 0 = nothing can be pruned
@@ -122,14 +119,9 @@ k_unsketch_sample(const SparseArgs A) {
 }
 
 // ---- every coordinate, with early exit; survivors appended to the list -----------------------------
-#ifndef SSGD_PRUNED_MINBLOCKS
-#define SSGD_PRUNED_MINBLOCKS 1
-#endif
-#ifndef SSGD_PRUNED_NC
-#define SSGD_PRUNED_NC 4
-#endif
+constexpr int PRUNED_NC = 4;                             // consecutive coordinates per thread
 template <int R, bool POW2>
-__global__ void __launch_bounds__(SEL_THREADS, SSGD_PRUNED_MINBLOCKS)
+__global__ void __launch_bounds__(SEL_THREADS)
 k_unsketch_pruned(const SparseArgs A) {
     __shared__ SelShared sh;
     constexpr int NEED = (R + 1) / 2;      // big row estimates a survivor must have
@@ -141,7 +133,7 @@ k_unsketch_pruned(const SparseArgs A) {
     const uint32_t bin_lo = A.rerun ? 0u : A.sp.state->bin_lo;
     __syncthreads();
     const int lane = threadIdx.x & 31;
-    constexpr int NC = SSGD_PRUNED_NC;                     // consecutive coordinates per thread
+    constexpr int NC = PRUNED_NC;
     const int64_t groups = (A.d + NC - 1) / NC;
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
     // warp-uniform trip count: the append below uses warp-wide shuffles

@@ -48,7 +48,11 @@ constexpr size_t ALIGN = 256;
 constexpr int TIMING_SLOTS = 256;
 // ssgd_sketch_accumulate goes through the workers one launch at a time once all W tables together exceed this
 constexpr size_t WORKER_MAJOR_MIN_BYTES = (size_t)32 << 20;
-constexpr int64_t SMALL_AUTO_MAX_D = (int64_t)1 << 21;      // AUTO takes the one-kernel tail up to this many coordinates
+// AUTO takes the one-kernel tail up to this many coordinates and candidates.  Measured on B200, whole step,
+// fused / chain of launches: d = 2^20, W = 4, ncand = 2000: 0.109 / 0.127 ms; d = 2^21, W = 4, ncand = 4000: 0.181 /
+// 0.210; d = 2e6, W = 16, ncand = 16000: 0.290 / 0.281 (the last block's serial part grows with ncand)
+constexpr int64_t SMALL_AUTO_MAX_D = (int64_t)1 << 21;
+constexpr int64_t SMALL_AUTO_MAX_NCAND = 4096;
 constexpr int64_t SMALL_INLINE_ZERO_MAX = 65536;            // eager line 13 inside the tail kernel up to this many k*W
 constexpr int EV_PER_STEP = SSGD_NSTAGES + 1;
 inline size_t up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
@@ -221,7 +225,8 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
 // (measured on B200 against the chain of short launches).
 bool use_small(const ssgd_ctx* x, int64_t ncand) {
     if (x->prune_mode == SSGD_PRUNE_FUSED) return small_tail_applicable(x, ncand);
-    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D;
+    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D &&
+           ncand <= SMALL_AUTO_MAX_NCAND;
 }
 
 // Whether ssgd_step takes the pruned first pass + selection on the survivor list (filter_unsketch.cuh,
@@ -361,8 +366,8 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
-    x->small_grid = 0; x->small_cs = 0; x->small_smem = 0; x->wait_ns = 2000000000ull; x->withhold = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SSGD_SPLIT_BYTES_DEFAULT;
+    x->small_grid = 0; x->wait_ns = 2000000000ull; x->withhold = 0;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
@@ -660,6 +665,17 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if ((e = gather_select_zero(x, cand, ncand, out_idx, out_val, st, x->zero_mode == SSGD_ZERO_DEFERRED, A.xsum, sparse))) return e;
     if ((e = mark(x, 4, st))) return e;
     if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
+    return SSGD_OK;
+}
+
+int ssgd_tail_trace(ssgd_ctx* x, void* stream, int64_t* out12) {
+    int e = check_bound(x);
+    if (e) return e;
+    if (!out12) return SSGD_EINVAL;
+    CU(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)), "stream synchronize");
+    SmallState s;
+    CU(cudaMemcpy(&s, x->ws + x->off_small, sizeof(s), cudaMemcpyDeviceToHost), "read tail state");
+    for (int t = 0; t < 12; ++t) out12[t] = s.trace[t] ? (int64_t)(s.trace[t] - s.trace[0]) : -1;
     return SSGD_OK;
 }
 

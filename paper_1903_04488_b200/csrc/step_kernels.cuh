@@ -12,48 +12,34 @@
 #include "hash.cuh"
 #include "select.cuh"
 
+namespace ssgd {
+
 // Table bytes one insert kernel may scatter into; larger tables are inserted in row slices.  Measured on B200
 // (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each): 1 row per kernel 6.43 ms, 2 rows 6.25, 3 rows 6.60,
 // 4 rows 6.89, all 5 rows in one kernel 7.80.
-#ifndef SSGD_SPLIT_BYTES_DEFAULT
-#define SSGD_SPLIT_BYTES_DEFAULT ((size_t)40 << 20)
-#endif
+constexpr size_t SPLIT_BYTES_DEFAULT = (size_t)40 << 20;
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
-#ifndef SSGD_PRUNED_GRID
-#define SSGD_PRUNED_GRID 4
-#endif
-#ifndef SSGD_K3_GRID
-#define SSGD_K3_GRID 4
-#endif
+constexpr int PRUNED_GRID = 4;
+constexpr int K3_GRID = 4;
 
-namespace ssgd {
 
 // ------------------------------------------------------------------------------------------------
-// K1 (plain-load form): momentum + error accumulation + sketch insert.  ssgd_step uses the bulk-copy
-// pipeline of accum_tma.cuh; this form serves the per-worker tables of ssgd_sketch_accumulate and the
+// K1 (plain-load form): momentum + error accumulation + sketch insert.  ssgd_step's default up to 128 workers
+// (the bulk-copy pipeline of accum_tma.cuh beyond); also the per-worker tables of ssgd_sketch_accumulate and the
 // shared-memory table variant.
 // ------------------------------------------------------------------------------------------------
 enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
 
-#ifndef SSGD_K1_UNROLL
-#define SSGD_K1_UNROLL 16
-#endif
-#ifndef SSGD_K1_MINBLOCKS
-#define SSGD_K1_MINBLOCKS 1
-#endif
 // Measured on B200 (C2, W = 16): 256 threads x 4 workers in flight 4.93 TB/s; 128 x 8 5.38; 128 x 16 5.58;
 // 64 x 16 5.56; forcing more resident blocks (fewer registers) or 32 workers in flight is slower.
 // The grid has one float4 group per thread on purpose: capping it at 2, 4, 8, 16, 40 blocks per SM (each
 // thread then loops over 74 ... 4 groups) took 0.887, 0.860, 0.814, 0.724, 0.654 ms against 0.635 ms, and
 // deferring a group's reductions until the next group's loads are issued recovered only part of that (0.805 ms
 // at 2 blocks per SM).
-#ifndef SSGD_K1_THREADS
-#define SSGD_K1_THREADS 128
-#endif
-constexpr int K1_THREADS = SSGD_K1_THREADS;
-constexpr int K1_UNROLL = SSGD_K1_UNROLL;  // workers in flight per thread: 3 x 16 B loads each
+constexpr int K1_THREADS = 128;
+constexpr int K1_UNROLL = 16;              // workers in flight per thread: 3 x 16 B loads each
 constexpr int K1_UNROLL_PW = 4;            // same, for the per-worker-table mode (it also holds 4r hashes)
 
 // UM: workers in flight per thread in the merged modes.  Measured on B200 with 4 workers (d = 7.3e7 / 9e7, r = 5):
@@ -61,7 +47,7 @@ constexpr int K1_UNROLL_PW = 4;            // same, for the per-worker-table mod
 // to cover the stream while the reductions issue); with 8 workers 4, 8 and 16 are equal.
 constexpr int K1_UNROLL_FEW = 4;
 template <int R, bool POW2, int MODE, int UM = K1_UNROLL>
-__global__ void __launch_bounds__(K1_THREADS, SSGD_K1_MINBLOCKS)
+__global__ void __launch_bounds__(K1_THREADS)
 k_accum_insert(const AccumArgs A) {
     extern __shared__ float s_table[];  // MODE == INS_MERGED_SMEM: [R][c]
     const int64_t rc = (int64_t)R * A.c;
@@ -357,10 +343,7 @@ k_emit_candidates(const float* __restrict__ est, int64_t d, SelBuffers sb, int32
 // ------------------------------------------------------------------------------------------------
 // K5: second round -- xs[m] = sum_w v_w[cand[m]] (fp64, w = 0..W-1), rounded once to fp32
 // ------------------------------------------------------------------------------------------------
-#ifndef SSGD_GATHER_UNROLL
-#define SSGD_GATHER_UNROLL 8
-#endif
-constexpr int GATHER_UNROLL = SSGD_GATHER_UNROLL;   // scattered loads in flight per thread
+constexpr int GATHER_UNROLL = 8;   // scattered loads in flight per thread
 
 static __global__ void __launch_bounds__(256)
 k_gather(const int32_t* __restrict__ cand, int64_t ncand, const float* __restrict__ v, int64_t ld, int32_t W,

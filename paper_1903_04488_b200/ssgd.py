@@ -39,6 +39,7 @@ SIGNATURES = {
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
     "ssgd_set_zero_mode": [_vp, _i32],
     "ssgd_set_wait_limit_ns": [_vp, _i64],
+    "ssgd_tail_trace": [_vp, _vp, C.POINTER(_i64)],
     "ssgd_test_withhold_block": [_vp, _i32],
     "ssgd_flush": [_vp, _vp],
     "ssgd_workspace_bytes": [_vp, _i64, C.POINTER(_sz)],
@@ -201,6 +202,12 @@ class Ssgd:
         out = (_i32 * 5)()
         self._chk(self._lib.ssgd_step_used_fallback(self._h, _stream(), out), "ssgd_step_used_fallback")
         return bool(out[3]), int(out[4])
+
+    def tail_trace(self):
+        """Nanosecond stamps of the last fused tail (see ssgd_tail_trace), -1 where none was taken."""
+        out = (_i64 * 12)()
+        self._chk(self._lib.ssgd_tail_trace(self._h, _stream(), out), "ssgd_tail_trace")
+        return list(out)
 
     def workspace_bytes(self, ncand_max: int) -> int:
         out = _sz()

@@ -264,11 +264,12 @@ def test_heavy_ties_at_the_threshold(cuda_device, prune):
 # lines 9-13 as one cooperative kernel (small problems)
 # ------------------------------------------------------------------------------------------------
 FUSED_CASES = [
-    # (configuration, steps, zero mode): table in one CTA's shared memory, in a cluster of 2, 4, 8, and too large for any
-    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 160 KiB: one CTA; zeros written in the kernel
-    (wl.C1.scaled(d=524_288, c=16_384, ncand=2000, k=1000), 2, S.ZERO_EAGER),             # C1's sketch: cluster of 2
-    (wl.C3.scaled(d=200_003, W=6, c=32_768, ncand=2000, k=1000), 3, S.ZERO_DEFERRED),     # cluster of 4
-    (wl.C4.scaled(d=270_002, W=3, c=65_536, ncand=1500, k=700), 3, S.ZERO_DEFERRED),      # cluster of 8
+    # (configuration, steps, zero mode): the table copied into shared memory (it fits and d >= 2 * c * 148), or read from L2
+    (wl.C2.scaled(d=700_001, W=2, c=2048, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 40 KiB table in shared memory; zeros written in the kernel
+    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 160 KiB table, too few lookups: L2
+    (wl.C1.scaled(d=524_288, c=16_384, ncand=2000, k=1000), 2, S.ZERO_EAGER),             # C1's sketch
+    (wl.C3.scaled(d=200_003, W=6, c=32_768, ncand=2000, k=1000), 3, S.ZERO_DEFERRED),
+    (wl.C4.scaled(d=270_002, W=3, c=65_536, ncand=1500, k=700), 3, S.ZERO_DEFERRED),
     (wl.C2.scaled(d=250_001, W=2, c=200_000, ncand=16_384, k=16_384), 2, S.ZERO_DEFERRED),  # table read from L2; largest ncand; k = ncand
     (wl.C2.scaled(d=150_002, W=17, r=3, c=999, ncand=9000, k=5000), 2, S.ZERO_EAGER),     # k*W too large for in-kernel zeros
     (wl.C3.scaled(d=2_100_003, W=2, r=7, c=4001, ncand=5000, k=100), 2, S.ZERO_DEFERRED), # d above 2^21, real modulo
