@@ -5,9 +5,9 @@
 //
 //   phase 1   every CTA estimates its share of the coordinates (Algorithm 4 estimate: median of the r signed
 //             buckets), stores est[i] and counts the top 12 bits of |est| in a shared-memory histogram -> H1.
-//             If the whole r x c table fits one CTA's shared memory and the CTA has clearly more lookups to do
-//             than the table has entries, it copies the table first and looks up there (3.5 random 4-byte reads
-//             per clock per SM against 1.1 from L2, measured).  A table split over the shared memory of a
+//             As many rows of the table as fit one CTA's shared memory are copied there first and looked up there
+//             (3.5 random 4-byte reads per clock per SM against 1.1 from L2, measured), provided the CTA has
+//             enough lookups to do for the copy to pay; the other rows are read from L2.  A table split over the shared memory of a
 //             thread-block cluster was measured and dropped: random reads of another CTA's shared memory run at
 //             0.7 per clock per SM in a cluster of 2 and 0.4 in clusters of 4 to 16 -- slower than L2.
 //   barrier   H1 complete: every CTA finds the first threshold digit d1 for itself
@@ -66,7 +66,7 @@ struct SmallArgs {
     int32_t mark_pending;
     float* u; float* v; int64_t ld; int32_t W;  // eager line 13 written here when zero_inline != 0
     int32_t zero_inline;
-    int32_t use_smem;        // 1: every CTA copies the table into its shared memory and looks up there
+    int32_t rows_smem;       // every CTA copies rows [0, rows_smem) of the table into its shared memory and looks up there
     uint64_t wait_ns;        // limit of a barrier wait
     int32_t withhold;        // test hook: CTA (withhold - 1) leaves before the first barrier, so the others' wait runs out
     int32_t* errflag;
@@ -178,15 +178,33 @@ k_small_tail(const SmallArgs A) {
     if (A.pending)
         for (int64_t t = gtid; t < A.pending_words; t += gstride) A.pending[t] = 0u;   // consumed by the accumulate kernel
     const float* slice = reinterpret_cast<const float*>(st_dyn);
-    if (A.use_smem) {
-        float* dst = reinterpret_cast<float*>(st_dyn);
-        const int64_t n = (int64_t)R * A.c;
-        for (int64_t b0 = tid; b0 < n; b0 += ST_THREADS * 8) {
-            float t[8];
+    if (A.rows_smem > 0) {
+        const int64_t n = (int64_t)A.rows_smem * A.c;      // the first rows are one contiguous piece of the table
+        if ((A.c & 3) == 0) {
+            float4* dst = reinterpret_cast<float4*>(st_dyn);
+            const float4* src = reinterpret_cast<const float4*>(A.table);
+            for (int64_t b0 = tid; b0 < (n >> 2); b0 += ST_THREADS * 8) {
+                float4 t[8];
 #pragma unroll
-            for (int s8 = 0; s8 < 8; ++s8) t[s8] = b0 + s8 * ST_THREADS < n ? __ldcg(A.table + b0 + s8 * ST_THREADS) : 0.f;
+                for (int s8 = 0; s8 < 8; ++s8) {
+                    const int64_t at = b0 + s8 * ST_THREADS;
+                    t[s8] = __ldcg(src + (at < (n >> 2) ? at : 0));
+                }
 #pragma unroll
-            for (int s8 = 0; s8 < 8; ++s8) if (b0 + s8 * ST_THREADS < n) dst[b0 + s8 * ST_THREADS] = t[s8];
+                for (int s8 = 0; s8 < 8; ++s8) if (b0 + s8 * ST_THREADS < (n >> 2)) dst[b0 + s8 * ST_THREADS] = t[s8];
+            }
+        } else {
+            float* dst = reinterpret_cast<float*>(st_dyn);
+            for (int64_t b0 = tid; b0 < n; b0 += ST_THREADS * 8) {
+                float t[8];
+#pragma unroll
+                for (int s8 = 0; s8 < 8; ++s8) {
+                    const int64_t at = b0 + s8 * ST_THREADS;
+                    t[s8] = __ldcg(A.table + (at < n ? at : 0));
+                }
+#pragma unroll
+                for (int s8 = 0; s8 < 8; ++s8) if (b0 + s8 * ST_THREADS < n) dst[b0 + s8 * ST_THREADS] = t[s8];
+            }
         }
     }
     __syncthreads();
@@ -201,7 +219,7 @@ k_small_tail(const SmallArgs A) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const int64_t at = (int64_t)j * A.c + (hb[e] & P31);
-                rowv[e][j] = apply_sign(A.use_smem ? slice[at] : table_load(A.table + at), hb[e]);
+                rowv[e][j] = apply_sign(j < A.rows_smem ? slice[at] : table_load(A.table + at), hb[e]);
             }
         }
         float m[4];

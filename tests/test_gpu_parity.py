@@ -264,10 +264,11 @@ def test_heavy_ties_at_the_threshold(cuda_device, prune):
 # lines 9-13 as one cooperative kernel (small problems)
 # ------------------------------------------------------------------------------------------------
 FUSED_CASES = [
-    # (configuration, steps, zero mode): the table copied into shared memory (it fits and d >= 2 * c * 148), or read from L2
+    # (configuration, steps, zero mode): all rows of the table copied into shared memory, some of them, or none
     (wl.C2.scaled(d=700_001, W=2, c=2048, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 40 KiB table in shared memory; zeros written in the kernel
     (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), 3, S.ZERO_EAGER),          # 160 KiB table, too few lookups: L2
-    (wl.C1.scaled(d=524_288, c=16_384, ncand=2000, k=1000), 2, S.ZERO_EAGER),             # C1's sketch
+    (wl.C1.scaled(d=800_000, c=16_384, ncand=2000, k=1000), 2, S.ZERO_EAGER),             # C1's sketch: 3 of 5 rows in shared memory
+    (wl.C2.scaled(d=900_002, W=2, r=7, c=9_999, ncand=2000, k=1000), 2, S.ZERO_DEFERRED), # 5 of 7 rows, c not a multiple of 4
     (wl.C3.scaled(d=200_003, W=6, c=32_768, ncand=2000, k=1000), 3, S.ZERO_DEFERRED),
     (wl.C4.scaled(d=270_002, W=3, c=65_536, ncand=1500, k=700), 3, S.ZERO_DEFERRED),
     (wl.C2.scaled(d=250_001, W=2, c=200_000, ncand=16_384, k=16_384), 2, S.ZERO_DEFERRED),  # table read from L2; largest ncand; k = ncand
