@@ -701,6 +701,7 @@ int ssgd_flush(ssgd_ctx* x, void* stream) {
     int e = check_bound(x);
     if (e) return e;
     if ((e = ensure_device(x))) return e;
+    if (!x->pending_dirty) return SSGD_OK;                 // no deferred step since the last flush: nothing is marked
     return flush_pending(x, static_cast<cudaStream_t>(stream));
 }
 
