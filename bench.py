@@ -42,13 +42,14 @@ FALLBACK_HBM_GBS = 6650.0          # earlier measurement on this machine, used only
 ORACLE_COORDS_PER_S = 4.0e6        # conservative single-thread estimate used to size oracle samples
 HEADLINE = "C5_W256"
 SWEEP = ("C1", "C2", "C3", "C4", "C5_W8", "C5_W32", "C5_W128", "C5_W256")
+PAPER_SHAPES = ("P1", "P2", "P3")  # the paper's own sketch shapes (Table 1 footnotes), timed after the sweep
 L2_FLUSH_BYTES = 512 << 20         # written between repetitions of configurations whose working set fits in L2
 COLD_SETS = 8                      # independent (g, u, v, workspace) sets rotated through for such configurations
 # DRAM bytes per launch of the accumulate+insert kernel from ncu captures (dram__bytes_read.sum +
 # dram__bytes_write.sum on a small case, scaled in proportion to W*d), keyed by kernel: bytes per worker-coordinate
 NCU_TRAFFIC_BYTES_PER_UNIT = {
     "k_accum_insert": 1906.1e6 / (16 * 6_000_002),       # profiles/k_accum_insert_C2_d6M.md
-    "k_accum_insert_tma": None,
+    "k_accum_insert_tma": 5.12498e9 / (256 * 1_000_002),  # profiles/k_accum_insert_tma_C5_W256_d1M.md
 }
 
 
@@ -295,7 +296,7 @@ def step_bytes(cfg) -> float:
 
 
 def dominant_kernel(cfg) -> str:
-    return "k_accum_insert_tma" if cfg.W > 128 else "k_accum_insert"
+    return "k_accum_insert_tma" if cfg.W >= 64 else "k_accum_insert"
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -510,6 +511,11 @@ def run_ours(args):
                 per_config[name] = {"skipped": f"needs more device memory than the {f >> 30} GiB free"}
                 continue
             per_config[name] = measure_config(c, dev, args, gpu_index, reps)
+        for name in PAPER_SHAPES:
+            c = wl.CONFIGS[name]
+            f, _ = torch.cuda.mem_get_info()
+            if f >= (c.steps + 2) * c.W * c.ld * 4 + (4 << 30):
+                per_config[name] = measure_config(c, dev, args, gpu_index, reps)
         if args.faithful_c2:
             fargs = argparse.Namespace(**dict(vars(args), mode="faithful"))
             per_config["C2_faithful"] = measure_config(wl.CONFIGS["C2"], dev, fargs, gpu_index, reps)

@@ -61,7 +61,7 @@ extern "C" {
 #define SSGD_MAX_R 15
 
 /* Insert variants of ssgd_step (ssgd_set_insert_mode) */
-#define SSGD_INSERT_AUTO   0  /* SSGD_INSERT_TMA when W > 128, else SSGD_INSERT_GLOBAL (measured)            */
+#define SSGD_INSERT_AUTO   0  /* SSGD_INSERT_TMA when W >= 64, else SSGD_INSERT_GLOBAL (measured)            */
 #define SSGD_INSERT_GLOBAL 1  /* plain 128-bit loads; reductions straight into the L2-resident table    */
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */

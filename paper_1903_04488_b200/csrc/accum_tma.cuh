@@ -1,6 +1,6 @@
 // accum_tma.cuh -- the streaming form of Algorithm 3 lines 5-7 used by ssgd_step on sm_100a.
 //
-// One persistent CTA owns tiles of KT_TC consecutive coordinates.  For a tile it walks the W workers;
+// Persistent CTAs (one per SM) own tiles of KT_TC consecutive coordinates.  For a tile it walks the W workers;
 // each (tile, worker) is one pipeline stage: three bulk asynchronous copies (cp.async.bulk, the TMA
 // engine) bring that worker's g, u and v slices into a ring of shared-memory slots, completion is
 // signalled on an mbarrier.  A dedicated producer warp keeps the ring full, so the bytes in flight do
@@ -9,7 +9,7 @@
 // write u', v' straight back to global memory (coalesced 128-bit stores) and release the slot.
 // After the last worker each consumer thread hashes its four coordinates and issues the r reductions
 // per coordinate into the L2-resident merged table (sum_w S(v_w) = S(sum_w v_w), Section 3).
-// Several CTAs share an SM, so one CTA's reduction phase overlaps the others' streaming.
+// The producer runs ahead into the next tile while the consumers issue a tile's reductions.
 //
 // Every mbarrier wait is bounded: after `wait_ns` nanoseconds (an argument; ssgd_set_wait_limit_ns) the waiter
 // records ERR_TIMEOUT in the error word, raises the CTA's abort flag and leaves; whatever happened, the producer
@@ -47,8 +47,15 @@ struct AccumArgs {
 constexpr int KT_CONSUMER_WARPS = 8;
 constexpr int KT_CONSUMERS = KT_CONSUMER_WARPS * 32;
 constexpr int KT_THREADS = KT_CONSUMERS + 32;       // + one producer warp
-constexpr int KT_TC = KT_CONSUMERS * 4;             // coordinates per tile: one float4 per consumer thread
-constexpr int KT_STAGES = 6;                        // ring slots of 12 KiB each
+// Tile shape.  What matters is the length of the contiguous piece each bulk copy takes from one worker's row: with
+// W workers the kernel reads 3 W interleaved streams, and DRAM serves long pieces better than short ones.  Measured
+// on B200 at d = 11,173,962 (TB/s of 20 W d bytes; groups per thread x ring slots; piece = 4 KB x groups):
+//   W = 256:  1 x 6  5.72    2 x 4  5.93    4 x 4  6.09    4 x 3  6.13    6 x 2  6.14    8 x 2  6.11
+//   W = 128:  1 x 6  5.70    2 x 4  5.90    4 x 3  6.06        W = 64:  4 x 3  5.91  (plain-load kernel 5.88)
+//   16 consumer warps x 2 groups x 3 slots: 6.12; 4 warps x 8 x 3: 6.01.
+constexpr int KT_VEC = 4;                           // float4 groups per consumer thread and stage
+constexpr int KT_TC = KT_CONSUMERS * 4 * KT_VEC;    // 4096 coordinates per tile: 16 KB pieces
+constexpr int KT_STAGES = 3;                        // ring slots of 3 * 4 * KT_TC = 48 KB each (one CTA per SM)
 
 struct alignas(128) KtSlot { float g[KT_TC]; float u[KT_TC]; float v[KT_TC]; };
 struct KtShared {
@@ -180,18 +187,30 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
         uint32_t n = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
-            const int64_t i0 = tile * KT_TC + 4 * tid;
-            const bool active = i0 < d_main;
-            double x0 = 0., x1 = 0., x2 = 0., x3 = 0.;      // sum over workers of the new v: fp64, worker order
-            const uint32_t pend = active ? pending_bits4(A.pending, i0) : 0u;
+            // this thread's float4 groups of the tile: group v starts at coordinate tile * KT_TC + 4 * (tid + v * KT_CONSUMERS)
+            const int64_t t0 = tile * KT_TC;
+            double xs[KT_VEC][4];                           // sum over workers of the new v: fp64, worker order
+            uint32_t pend[KT_VEC];
+            bool active[KT_VEC];
+#pragma unroll
+            for (int v = 0; v < KT_VEC; ++v) {
+                const int64_t i0 = t0 + 4 * (tid + v * KT_CONSUMERS);
+                active[v] = i0 < d_main;
+                pend[v] = active[v] ? pending_bits4(A.pending, i0) : 0u;
+                xs[v][0] = xs[v][1] = xs[v][2] = xs[v][3] = 0.;
+            }
             for (int w = 0; w < A.W; ++w, ++n) {
                 const int s = n % KT_STAGES;
                 if (!mbar_wait(&S.full[s], (n / KT_STAGES) & 1, &S.abort, A.wait_ns)) { ok = false; break; }
-                if (active) {
-                    const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[4 * tid]);
-                    float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[4 * tid]);
-                    float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[4 * tid]);
-                    if (pend) drop_pending(pend, u4, v4);
+#pragma unroll
+                for (int v = 0; v < KT_VEC; ++v) {
+                    if (!active[v]) continue;
+                    const int at = 4 * (tid + v * KT_CONSUMERS);
+                    const int64_t i0 = t0 + at;
+                    const float4 g4 = *reinterpret_cast<const float4*>(&S.slot[s].g[at]);
+                    float4 u4 = *reinterpret_cast<const float4*>(&S.slot[s].u[at]);
+                    float4 v4 = *reinterpret_cast<const float4*>(&S.slot[s].v[at]);
+                    if (pend[v]) drop_pending(pend[v], u4, v4);
                     float4 un, vn;
                     un.x = __fmaf_rn(A.rho, u4.x, g4.x); vn.x = __fadd_rn(v4.x, un.x);
                     un.y = __fmaf_rn(A.rho, u4.y, g4.y); vn.y = __fadd_rn(v4.y, un.y);
@@ -199,15 +218,18 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
                     un.w = __fmaf_rn(A.rho, u4.w, g4.w); vn.w = __fadd_rn(v4.w, un.w);
                     __stcs(reinterpret_cast<float4*>(A.u + (int64_t)w * A.ld + i0), un);
                     __stcs(reinterpret_cast<float4*>(A.v + (int64_t)w * A.ld + i0), vn);
-                    x0 = __dadd_rn(x0, (double)vn.x); x1 = __dadd_rn(x1, (double)vn.y);
-                    x2 = __dadd_rn(x2, (double)vn.z); x3 = __dadd_rn(x3, (double)vn.w);
+                    xs[v][0] = __dadd_rn(xs[v][0], (double)vn.x); xs[v][1] = __dadd_rn(xs[v][1], (double)vn.y);
+                    xs[v][2] = __dadd_rn(xs[v][2], (double)vn.z); xs[v][3] = __dadd_rn(xs[v][3], (double)vn.w);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&S.empty[s]);
             }
             if (!ok) break;
-            if (active) {
-                const float x[4] = {(float)x0, (float)x1, (float)x2, (float)x3};
+#pragma unroll
+            for (int v = 0; v < KT_VEC; ++v) {
+                if (!active[v]) continue;
+                const int64_t i0 = t0 + 4 * (tid + v * KT_CONSUMERS);
+                const float x[4] = {(float)xs[v][0], (float)xs[v][1], (float)xs[v][2], (float)xs[v][3]};
                 if (A.xsum) __stcs(reinterpret_cast<float4*>(A.xsum + i0), make_float4(x[0], x[1], x[2], x[3]));
 #pragma unroll
                 for (int j = 0; j < R; ++j) {

@@ -338,11 +338,10 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     if (x->insert_mode == SSGD_INSERT_SMEM) return fits ? INS_MERGED_SMEM : -1;
     if (x->insert_mode == SSGD_INSERT_GLOBAL) return INS_MERGED_GLOBAL;
     if (x->insert_mode == SSGD_INSERT_TMA) return INS_MERGED_TMA;
-    // measured on B200: the bulk-copy pipeline wins once a tile's walk over the workers is long
-    // (W = 128: 5.73 vs 5.43 TB/s), plain loads win for short walks (W = 16: 4.93 vs 4.83 TB/s)
-    // measured at C2's d (plain / bulk-copy, TB/s): W = 32 5.98 / 5.36; 96 5.79 / 5.64; 128 5.72 / 5.69; 192 5.53 / 5.71;
-    // 256 5.43 / 5.70 -- the plain kernel's threads loop over the workers 16 at a time, and loop less well than they start
-    return x->W > 128 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
+    // measured on B200 at d = 11,173,962 (plain loads / bulk-copy pipeline, TB/s): W = 32 6.06 / 5.58; 48 5.97 / 5.83;
+    // 64 5.88 / 5.91; 96 5.82 / 6.01; 128 5.75 / 6.06; 256 5.42 / 6.13 -- the plain kernel's threads loop over the
+    // workers 16 at a time, and loop less well than they start
+    return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
 }  // namespace
