@@ -124,8 +124,9 @@ int ssgd_set_wait_limit_ns(ssgd_ctx* ctx, int64_t ns);
 /* Test hook: thread block (block_plus_one - 1) of those kernels leaves without ever arriving at its barriers, so
  * that the others' waits run out (nothing hangs, nothing faults); 0 switches the hook off. */
 int ssgd_test_withhold_block(ssgd_ctx* ctx, int32_t block_plus_one);
-/* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Launches
- * nothing when no deferred step has run since the last flush. */
+/* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Cheap when
+ * nothing is pending (one pass over d/8 bytes).  It always launches: the marks may come from a replayed CUDA
+ * graph, which the host side of the context does not see. */
 int ssgd_flush(ssgd_ctx* ctx, void* stream);
 /* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
  * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up

@@ -242,6 +242,36 @@ def test_misjudged_threshold_reruns_without_pruning(cuda_device, prune):
     assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
 
 
+@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT])
+def test_carried_prune_threshold(cuda_device, prune):
+    """From the second step on the prune threshold is the previous step's exact threshold minus a margin, not a
+    sample.  The candidates never depend on it: when the accumulated vector suddenly shrinks a thousandfold (state
+    reset by the caller, tiny gradients) the carried threshold keeps far fewer than ncand coordinates, the pass is
+    redone without pruning, and the step after that prunes again on the new threshold."""
+    cfg = wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000)
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(prune)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    for t in range(2):                                     # sampled, then carried: both prune without a rerun
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
+        fell_back, survivors, bin_lo = eng.step_used_fallback()
+        assert not fell_back and bin_lo > 0 and cfg.ncand <= survivors < cfg.d // 10
+    eng.flush()
+    u.zero_(); v.zero_()
+    u_o[:] = 0; v_o[:] = 0
+    check_step(orc, eng, wl.gradients(st, 2) * 1e-3, cfg.rho, cfg.ncand, u_o, v_o)
+    fell_back, survivors, bin_lo = eng.step_used_fallback()
+    assert fell_back and survivors == cfg.d and bin_lo > 0  # the carried threshold was far too high: rerun, same result
+    check_step(orc, eng, wl.gradients(st, 3) * 1e-3, cfg.rho, cfg.ncand, u_o, v_o)
+    fell_back, survivors, _ = eng.step_used_fallback()
+    assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
+    # another ncand: the carried threshold belongs to another selection and is not used (a sample decides)
+    check_step(orc, eng, wl.gradients(st, 4) * 1e-3, cfg.rho, cfg.ncand // 2, u_o, v_o)
+    fell_back, survivors, _ = eng.step_used_fallback()
+    assert not fell_back and cfg.ncand // 2 <= survivors < cfg.d // 10
+
+
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_FUSED])
 def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
@@ -289,9 +319,9 @@ def test_fused_tail_lockstep(cuda_device, cfg, steps, zero):
     for t in range(steps):
         check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o, flush=(t == steps - 1))
     # memset + accumulate + tail (+ k_zero when k*W is too large for the tail) per step; check_step adds the dense
-    # stage call (5 launches) and, with the zero-out deferred, the last one a flush
+    # stage call (5 launches) and the last one a flush
     per_step = 3 + (1 if zero == S.ZERO_EAGER and cfg.k * cfg.W > 65536 else 0)
-    assert eng.launch_count() - n0 == steps * (per_step + 5) + (1 if zero == S.ZERO_DEFERRED else 0)
+    assert eng.launch_count() - n0 == steps * (per_step + 5) + 1
 
 
 def test_fused_tail_is_refused_where_it_does_not_apply(cuda_device):
