@@ -49,7 +49,7 @@ COLD_SETS = 8                      # independent (g, u, v, workspace) sets rotat
 # dram__bytes_write.sum on a small case, scaled in proportion to W*d), keyed by kernel: bytes per worker-coordinate
 NCU_TRAFFIC_BYTES_PER_UNIT = {
     "k_accum_insert": 1906.1e6 / (16 * 6_000_002),       # profiles/k_accum_insert_C2_d6M.md
-    "k_accum_insert_tma": 5.12498e9 / (256 * 1_000_002),  # profiles/k_accum_insert_tma_C5_W256_d1M.md
+    "k_accum_insert_tma": 5.09581e9 / (256 * 1_000_002),  # profiles/k_accum_insert_tma_C5_W256_d1M.md
 }
 
 
@@ -467,9 +467,40 @@ def measure_config(cfg, dev, args, gpu_index, reps):
         rec["roofline"]["frac_of_binding_bound"] = max(t_ops, t_hbm) / stage["accumulate_insert_ms"]
     if b.cold:
         rec["ms_per_step_warm_l2"] = b.warm_sequence(20)
+    if b.mode == "faithful":
+        rec["sketch16"] = time_sketch16(b)
     del b
     torch.cuda.empty_cache()
     return rec
+
+
+def time_sketch16(b):
+    """16-bit sketches (Section 6) on the per-worker tables of the faithful pipeline: what quantising them and
+    merging the 16-bit encodings costs beside the fp32 merge, with the bytes each kernel moves."""
+    torch, S, cfg = b.torch, b.S, b.cfg
+    q16 = torch.empty((cfg.W, cfg.r, cfg.c), dtype=torch.int16, device=b.dev)
+    rc = cfg.r * cfg.c
+
+    def timed(fn, n=20):
+        for _ in range(3):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    out = {"merge_fp32_ms": timed(lambda: b.eng.sketch_merge(b.tables, b.merged)),
+           "merge_fp32_bytes": 4 * rc * (cfg.W + 1)}
+    for name, fmt in (("f16", S.FMT_F16), ("bf16", S.FMT_BF16)):
+        out[f"quantize_{name}_ms"] = timed(lambda: b.eng.sketch_quantize16(b.tables, fmt, q16))
+        out[f"merge_{name}_ms"] = timed(lambda: b.eng.sketch_merge16(q16, fmt, b.merged))
+    out["quantize_bytes"] = 6 * rc * cfg.W
+    out["merge16_bytes"] = 2 * rc * cfg.W + 4 * rc
+    out["note"] = "working set (W tables) may fit in L2: these are warm figures"
+    return out
 
 
 def run_ours(args):

@@ -46,7 +46,6 @@ struct ssgd_ctx {
     bool filter_ready;                                     // shared-memory attribute of the filter kernel set
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
     size_t off_pending;     // d-bit map of the deferred zero-out; survives from step to step
-    size_t off_carry;       // previous selection's threshold bin (prune threshold of the next step); survives too
     int32_t zero_mode;      // SSGD_ZERO_DEFERRED / SSGD_ZERO_EAGER
     int32_t sched_mode;     // SSGD_SCHED_*: how ssgd_sketch_accumulate walks workers and coordinates
     bool pending_dirty;     // a deferred ssgd_step has run since the last flush: u, v may await their zero-out

@@ -29,7 +29,7 @@ constexpr int MAP_CHUNK_WORDS = SEL_THREADS * 8;       // map words per block in
 
 // ---- histogram pass over the list; its last block publishes T and Q --------------------------------------
 static __global__ void __launch_bounds__(SEL_THREADS)
-k_list_hist(SparseBuffers sp, uint32_t ncand) {
+k_list_hist(SparseBuffers sp) {
     __shared__ SelShared sh;
     pdl_trigger();
     for (int b = threadIdx.x; b < H2_BINS; b += SEL_THREADS) sh.hist[b] = 0;
@@ -58,7 +58,6 @@ k_list_hist(SparseBuffers sp, uint32_t ncand) {
         if (threadIdx.x == 0) {
             sp.state->thr_key = (d1 << H1_SHIFT) | (d2 << H2_SHIFT) | d3;
             sp.state->quota_eq = rem3;
-            if (sp.carry) { sp.carry[1] = d1; sp.carry[2] = ncand; sp.carry[0] = 1u; }   // for the next step's prune threshold
         }
     }
 }

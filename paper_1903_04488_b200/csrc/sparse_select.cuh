@@ -7,11 +7,7 @@
 //   * |median of r values| >= t  implies  at least (r+1)/2 of the r values have magnitude >= t.
 //     So once a coordinate cannot reach (r+1)/2 "big" row estimates any more, its remaining rows need
 //     not be read: it is certainly below t.
-//   * From the second step on, t is carried over: the exact threshold of the previous step's selection (same
-//     ncand), lowered by CARRY_MARGIN histogram bins (about 9 %), is the prune threshold, and the sample kernel
-//     returns at once.  The accumulated vector changes slowly from step to step, and a threshold that turns out
-//     too high only costs the unpruned rerun below; the candidates never depend on it.
-//   * Otherwise a safe t comes from a sample: k_unsketch_sample computes exact estimates for 1/64 of the
+//   * A safe t comes from a sample: k_unsketch_sample computes exact estimates for 1/64 of the
 //     float4 groups (pseudo-randomly placed), histograms them, and takes the histogram-bin edge `bin_lo`
 //     below which fewer than  ncand/64 + 6*sqrt(ncand/64) + 16  sampled estimates remain ... i.e. a
 //     threshold the full vector exceeds at least ncand times except with negligible probability.
@@ -62,11 +58,7 @@ struct SparseBuffers {
     uint32_t* map_b;       // [ceil(d/32)] zeroed: coordinates at the threshold (ties)
     uint32_t* chunk_a;     // [map chunks] marks per chunk of map words, then exclusive offsets
     uint32_t* chunk_b;
-    // NOT zeroed per step: [0] = 1 once a selection on the list has finished, [1] = histogram bin of its threshold
-    // key, [2] = its ncand.  Written by k_list_hist's last block, read by the next step's k_unsketch_sample.
-    uint32_t* carry;
 };
-constexpr uint32_t CARRY_MARGIN = 2;   // bins (1/16 octave each) below the previous threshold
 
 struct SparseArgs {
     const float* table; int64_t c; int64_t d;
@@ -77,7 +69,6 @@ struct SparseArgs {
     uint32_t n_sampled_min; // a lower bound of the number of sampled coordinates: 4 * (windows - 2)
     int32_t rerun;         // 0: the pruned pass; 1: the unpruned pass behind it (runs only if fallback == 1)
     int32_t gated;         // 1: the pruned pass runs only if use_table is set (it follows a bitmap filter that declined)
-    int32_t use_carry;     // 1: the previous step's threshold may stand in for the sample (k_unsketch_sample decides)
 };
 
 #ifdef __CUDACC__
@@ -94,12 +85,6 @@ k_unsketch_sample(const SparseArgs A) {
     pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
-    if (A.use_carry && __ldcg(A.sp.carry) == 1u && __ldcg(A.sp.carry + 2) == A.ncand && __ldcg(A.sp.carry + 1) > CARRY_MARGIN) {
-        // the previous step's threshold, lowered by the margin, stands in for the sample (a carried bin at or
-        // below the margin says nothing: all-zero or all-equal estimates; the sample decides then)
-        if (blockIdx.x == 0 && threadIdx.x == 0) A.sp.state->bin_lo = __ldcg(A.sp.carry + 1) - CARRY_MARGIN;
-        return;
-    }
     __syncthreads();
     const int64_t groups = (A.d + 3) >> 2;
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;

@@ -119,7 +119,6 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->bm_fold = s <= FILTER_MAX_FOLD ? s : -1;
     x->bm_stride_fold = s <= FILTER_MAX_FOLD ? (int32_t)round4((sf + (1 << s) - 1) >> s) : 0;
     x->off_pending = o; o += x->map_bytes;
-    x->off_carry = o;   o += up(16);
     x->off_bm_full = o; o += up((size_t)x->r * sf * 4);
     x->off_bm_fold = o; o += up((size_t)x->r * x->bm_stride_fold * 4);
     x->total_bytes = o;
@@ -219,7 +218,6 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
     sp.map_b = reinterpret_cast<uint32_t*>(x->ws + x->off_maps + x->map_bytes);
     sp.chunk_a = reinterpret_cast<uint32_t*>(x->ws + x->off_map_chunks);
     sp.chunk_b = sp.chunk_a + x->nchunk_map;
-    sp.carry = reinterpret_cast<uint32_t*>(x->ws + x->off_carry);
     return sp;
 }
 
@@ -255,7 +253,6 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     A.ncand = (uint32_t)ncand;
     A.rerun = 0;
     A.gated = 0;
-    A.use_carry = x->sample_rank == 0 ? 1 : 0;           // a forced sample rank (tests) always samples
     const int64_t groups = (x->d + 3) / 4;
     const int64_t windows = (groups + (1 << SPARSE_SAMPLE_SHIFT) - 1) >> SPARSE_SAMPLE_SHIFT;
     const double mean = (double)ncand * (double)(windows * 4) / (double)x->d;
@@ -266,7 +263,7 @@ int unsketch_select_sparse(ssgd_ctx* x, const float* merged, int64_t ncand, int3
     if ((e = mark(x, 2, st))) return e;
     // the list normally holds 1-2 x ncand entries; the kernels stride over whatever it holds
     const int list_grid = grid_for(4 * ncand, SEL_THREADS * SEL_BATCH, (int64_t)x->sm_count * 8);
-    CU(launch_pdl(st, k_list_hist, list_grid, SEL_THREADS, 0, A.sp, (uint32_t)ncand), "launch k_list_hist");
+    CU(launch_pdl(st, k_list_hist, list_grid, SEL_THREADS, 0, A.sp), "launch k_list_hist");
     LAUNCHED("k_list_hist");
     CU(launch_pdl(st, k_list_mark, list_grid, SEL_THREADS, 0, A.sp, x->nchunk_map), "launch k_list_mark");
     LAUNCHED("k_list_mark");
@@ -489,7 +486,6 @@ int ssgd_bind(ssgd_ctx* x, float* u, float* v, int64_t ld, void* workspace, size
     if (e) return e;
     CU(cudaMemset(x->ws + x->off_err, 0, 16), "clear error flag");
     CU(cudaMemset(x->ws + x->off_pending, 0, x->map_bytes), "clear pending map");   // nothing awaits its zero-out
-    CU(cudaMemset(x->ws + x->off_carry, 0, 16), "clear carried threshold");
     x->pending_dirty = false;
     return SSGD_OK;
 }

@@ -242,36 +242,6 @@ def test_misjudged_threshold_reruns_without_pruning(cuda_device, prune):
     assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
 
 
-@pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT])
-def test_carried_prune_threshold(cuda_device, prune):
-    """From the second step on the prune threshold is the previous step's exact threshold minus a margin, not a
-    sample.  The candidates never depend on it: when the accumulated vector suddenly shrinks a thousandfold (state
-    reset by the caller, tiny gradients) the carried threshold keeps far fewer than ncand coordinates, the pass is
-    redone without pruning, and the step after that prunes again on the new threshold."""
-    cfg = wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000)
-    eng, orc, u, v = make(cfg, cuda_device)
-    eng.set_prune_mode(prune)
-    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
-    st = wl.Structure(cfg, cuda_device)
-    for t in range(2):                                     # sampled, then carried: both prune without a rerun
-        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
-        fell_back, survivors, bin_lo = eng.step_used_fallback()
-        assert not fell_back and bin_lo > 0 and cfg.ncand <= survivors < cfg.d // 10
-    eng.flush()
-    u.zero_(); v.zero_()
-    u_o[:] = 0; v_o[:] = 0
-    check_step(orc, eng, wl.gradients(st, 2) * 1e-3, cfg.rho, cfg.ncand, u_o, v_o)
-    fell_back, survivors, bin_lo = eng.step_used_fallback()
-    assert fell_back and survivors == cfg.d and bin_lo > 0  # the carried threshold was far too high: rerun, same result
-    check_step(orc, eng, wl.gradients(st, 3) * 1e-3, cfg.rho, cfg.ncand, u_o, v_o)
-    fell_back, survivors, _ = eng.step_used_fallback()
-    assert not fell_back and cfg.ncand <= survivors < cfg.d // 10
-    # another ncand: the carried threshold belongs to another selection and is not used (a sample decides)
-    check_step(orc, eng, wl.gradients(st, 4) * 1e-3, cfg.rho, cfg.ncand // 2, u_o, v_o)
-    fell_back, survivors, _ = eng.step_used_fallback()
-    assert not fell_back and cfg.ncand // 2 <= survivors < cfg.d // 10
-
-
 @pytest.mark.parametrize("prune", [S.PRUNE_ON, S.PRUNE_EARLY_EXIT, S.PRUNE_OFF, S.PRUNE_FUSED])
 def test_heavy_ties_at_the_threshold(cuda_device, prune):
     """Many coordinates with one magnitude straddling both thresholds: the quota logic decides."""
@@ -766,6 +736,72 @@ def test_stage_calls_apply_a_pending_zero_out_first(cuda_device):
     before_u = u.clone()
     eng.sketch_accumulate(torch.zeros_like(u), 0.0, tables)   # rho = 0, g = 0: u <- 0, v <- v
     assert (u == 0).all() and (v[:, chosen.long()] == 0).all() and (before_u[:, chosen.long()] != 0).any()
+
+
+# ------------------------------------------------------------------------------------------------
+# nothing is written outside the buffers the caller hands over
+# ------------------------------------------------------------------------------------------------
+CANARY_CASES = [
+    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), S.PRUNE_FUSED, S.INSERT_GLOBAL),
+    (wl.C2.scaled(d=300_001, W=4, c=8192, ncand=3000, k=1500), S.PRUNE_OFF, S.INSERT_TMA),
+    (wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000), S.PRUNE_ON, S.INSERT_GLOBAL),
+    (wl.C3.scaled(d=600_011, W=3, r=5, c=524_288, ncand=5000, k=2000), S.PRUNE_ON, S.INSERT_GLOBAL),   # folded bitmap
+    (wl.C2.scaled(d=500_003, W=3, c=8192, ncand=4000, k=2000), S.PRUNE_EARLY_EXIT, S.INSERT_GLOBAL),
+]
+
+
+@pytest.mark.parametrize("cfg,prune,mode", CANARY_CASES, ids=lambda x: f"{x.name}-d{x.d}-c{x.c}" if hasattr(x, "name") else str(x))
+def test_canaries_around_every_caller_buffer_survive(cuda_device, cfg, prune, mode):
+    """Workspace, state, gradient and output buffers each sit between two 4 KiB guard zones filled with a pattern;
+    the workspace is exactly ssgd_workspace_bytes long.  After steps, a flush and the stage calls the guards are
+    untouched and the gradients unchanged."""
+    dev = cuda_device
+    G = 4096
+    pat = 0xA5
+
+    def guarded(nbytes):
+        raw = torch.full((nbytes + 2 * G,), pat, dtype=torch.uint8, device=dev)
+        return raw, raw[G:G + nbytes]
+
+    eng = S.Ssgd(cfg.d, cfg.r, cfg.c, cfg.k, cfg.W, cfg.sketch_seed)
+    n_ws = eng.workspace_bytes(cfg.ncand)
+    n_state = cfg.W * cfg.ld * 4
+    raws = {}
+    raws["ws"], ws = guarded(n_ws)
+    raws["u"], u8 = guarded(n_state)
+    raws["v"], v8 = guarded(n_state)
+    raws["g"], g8 = guarded(n_state)
+    raws["oi"], oi8 = guarded(cfg.k * 4)
+    raws["ov"], ov8 = guarded(cfg.k * 4)
+    u, v, g = (t.view(torch.float32).view(cfg.W, cfg.ld) for t in (u8, v8, g8))
+    oi, ov = oi8.view(torch.int32), ov8.view(torch.float32)
+    u.zero_(); v.zero_()
+    eng.bind(u, v, cfg.ncand, ws)
+    eng.set_prune_mode(prune)
+    eng.set_insert_mode(mode)
+    st = wl.Structure(cfg, dev)
+    for t in range(3):
+        g.copy_(wl.gradients(st, t))
+        g_before = g.clone()
+        eng.step(g, cfg.rho, cfg.ncand, oi, ov)
+        assert eng.status() == S.OK
+        assert torch.equal(g, g_before)
+    eng.flush()
+    # the stage calls on caller buffers of their exact sizes
+    raws["tab"], tab8 = guarded(cfg.W * cfg.r * cfg.c * 4)
+    raws["mer"], mer8 = guarded(cfg.r * cfg.c * 4)
+    raws["cand"], cand8 = guarded(cfg.ncand * 4)
+    raws["cest"], cest8 = guarded(cfg.ncand * 4)
+    tables = tab8.view(torch.float32).view(cfg.W, cfg.r, cfg.c)
+    merged = mer8.view(torch.float32).view(cfg.r, cfg.c)
+    cand, cest = cand8.view(torch.int32), cest8.view(torch.float32)
+    eng.sketch_accumulate(g, cfg.rho, tables)
+    eng.sketch_merge(tables, merged)
+    eng.unsketch_candidates(merged, cfg.ncand, cand, cest)
+    eng.exact_topk(cand, oi, ov)
+    assert eng.status() == S.OK
+    for name, raw in raws.items():
+        assert bool((raw[:G] == pat).all()) and bool((raw[-G:] == pat).all()), f"guard zone of {name} was written"
 
 
 # ------------------------------------------------------------------------------------------------
