@@ -79,10 +79,11 @@ extern "C" {
 #define SSGD_PRUNE_OFF  1
 #define SSGD_PRUNE_ON   2
 #define SSGD_PRUNE_EARLY_EXIT 3
-/* FUSED: lines 9-13 run as ONE cooperative kernel (dense estimates, exact radix select behind grid barriers, the
- * second round, the final top-k and line 13 by the last block), for problems so small that a chain of short
+/* FUSED: lines 9-13 run as ONE cooperative kernel (dense estimates, exact radix select and ordered candidate emit
+ * behind grid barriers, the second round where a candidate is emitted, the final top-k and line 13 by the last
+ * block), for problems so small that a chain of short
  * launches costs more than the work: needs d <= 2^22 and ncand <= 16384 (SSGD_EINVAL from ssgd_step otherwise).
- * AUTO takes this path for d <= 2^21 and ncand <= 4096.  The results are those of the other modes. */
+ * AUTO takes this path for d <= 2^21 when it applies.  The results are those of the other modes. */
 #define SSGD_PRUNE_FUSED 4
 
 typedef struct ssgd_ctx ssgd_ctx; /* opaque host object; holds no device memory */
@@ -145,10 +146,11 @@ int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
  * out[4] = set bits of the folded bitmap (0 if the bitmap is not folded). */
 int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out5);
 /* Diagnostics of the last ssgd_step that took the FUSED tail (waits for the stream): nanoseconds since the tail
- * kernel's first thread block started, at 12 points -- [0] start, [1] table copied to shared memory (if it is),
- * [2] its estimates done, [3]-[5] past the three grid barriers (all of thread block 0); of the block that finishes
- * the step alone: [6] it knows it is the last, [11] mark counts scanned, [7] candidates emitted, [8] second round
- * done, [9] final threshold known, [10] end.  -1 where no stamp was taken. */
+ * kernel's first thread block started, at 12 points -- [0] start, [1] table rows copied to shared memory (if any),
+ * [2] its estimates done, [3]-[5] past the first three grid barriers (the digits of the threshold), [11] past the
+ * fourth (segment counts complete), all of thread block 0; of the block that finishes the step alone: [6] it knows
+ * it is the last (candidates and their sums are in place), [7], [8] candidates loaded, [9] final threshold known,
+ * [10] end.  -1 where no stamp was taken. */
 int ssgd_tail_trace(ssgd_ctx* ctx, void* stream, int64_t* out12);
 /* For tests and diagnostics: the rank (from the top) in the sample's histogram that sets the prune threshold;
  * 0 = derive it from ncand (mean + 6 sigma + 16).  A rank of 1 puts the threshold at the largest sampled

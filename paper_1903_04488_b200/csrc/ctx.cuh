@@ -37,7 +37,7 @@ struct ssgd_ctx {
     char* ws; size_t ws_bytes; int64_t ncand_max;
     // workspace layout (byte offsets)
     size_t off_table, off_hist_c, off_hist_f, off_state_c, off_state_f, off_err, zero_bytes;
-    size_t off_h19_c, off_h19_f, off_small;
+    size_t off_h19_c, off_h19_f, off_small, zero_small_bytes;
     size_t off_sp_hist, off_sp_state, off_maps, off_map_chunks, off_list_idx, off_list_est;   // early-exit path
     size_t map_bytes;
     int64_t list_cap, nchunk_map;

@@ -1,7 +1,7 @@
 // small_tail.cuh -- Algorithm 3 lines 9-13 in ONE kernel, for problems so small that a chain of short launches
 // costs more than the work itself (d up to a few million coordinates, at most SMALL_MAX_NCAND candidates).
 //
-// The grid is co-resident (one CTA per SM, launched cooperatively) and its CTAs meet at three grid-wide barriers:
+// The grid is co-resident (one CTA per SM, launched cooperatively) and its CTAs meet at four grid-wide barriers:
 //
 //   phase 1   every CTA estimates its share of the coordinates (Algorithm 4 estimate: median of the r signed
 //             buckets), stores est[i] and counts the top 12 bits of |est| in a shared-memory histogram -> H1.
@@ -15,12 +15,15 @@
 //   barrier   -> second digit d2
 //   phase 3   histogram H3 of the last 8 key bits among the items matching the 23-bit prefix
 //   barrier   -> threshold key T and tie quota Q
-//   phase 4   every CTA marks its coordinates above T in a d-bit map A, those equal to T in map B.  The CTA that
-//             draws the last ticket goes on alone (nobody waits for it):
-//   phase 5   ordered walk of the two maps -> cand_idx ascending, ties at T to the smallest coordinates
-//             (line 9); xs[m] = the accumulate kernel's sum over the workers at cand_idx[m] (line 10); exact
-//             top-k of |xs| in shared memory, 12 + 11 + 8 bits, ordered emit of out_idx / out_val (line 11);
+//   phase 4   every warp counts, per segment of 128 consecutive coordinates, those above T and those equal to T
+//   barrier   -> with the counts of everything before it, every warp emits its candidates to their final slots:
+//             cand_idx ascending, ties at T to the smallest coordinates (line 9), and reads each candidate's exact
+//             sum over the workers right there (line 10).  The CTA that draws the last ticket goes on alone
+//             (nobody waits for it):
+//   phase 5   exact top-k of |xs| in shared memory, 12 + 11 + 8 bits, ordered emit of out_idx / out_val (line 11);
 //             line 13 as marks in the pending map (deferred) or as zeros written to u and v (eager, small k*W).
+// (An earlier form marked the candidates in two d-bit maps and let the last CTA walk them in order: 13 us of
+// instruction issue on one SM at d = 2^20, growing with d; the distributed form costs one more barrier.)
 //
 // Every wait at a barrier is bounded: after `wait_ns` the waiting CTA records ERR_TIMEOUT in the error word,
 // raises the abort flag so that the others stop waiting too, and returns.
@@ -46,8 +49,8 @@ struct SmallState {          // zeroed before the step
     uint32_t ticket;         // CTAs that finished phase 4
     uint32_t pad;
     uint64_t trace[12];      // globaltimer stamps of CTA 0 (slots 0-5) and of the last CTA (6-10), for diagnostics
-    // marks per stretch of map words (stretch w = the words warp w of the last CTA walks), counted in phase 4
-    uint32_t chunk_a[ST_WARPS], chunk_b[ST_WARPS];
+    // coordinates above / at the threshold per super-segment (64 segments of 128 coordinates), counted in phase 4
+    uint32_t sup_a[ST_THREADS], sup_b[ST_THREADS];
 };
 
 struct SmallArgs {
@@ -56,7 +59,7 @@ struct SmallArgs {
     float* est;              // [d], 16-byte aligned
     uint32_t* h1; uint32_t* h2; uint32_t* h3;   // global histograms of the candidate selection, zeroed
     SmallState* st;
-    uint32_t* map_a; uint32_t* map_b;           // [ceil(d/32)] words each, zeroed; 16-byte aligned
+    uint32_t* map_a; uint32_t* map_b;           // [>= ceil(d/128)] words each: per-segment counts, written before they are read
     const float* xsum;       // [d] per-coordinate sums over the workers of the new v
     int32_t* cand_idx; float* xs;               // [ncand] (kept for inspection)
     uint32_t ncand, k;
@@ -167,8 +170,6 @@ k_small_tail(const SmallArgs A) {
     const int64_t groups = (A.d + 3) >> 2;
     const int64_t gstride = (int64_t)gridDim.x * ST_THREADS;
     const int64_t gtid = (int64_t)blockIdx.x * ST_THREADS + tid;
-    const int64_t nwords = (A.d + 31) >> 5;                // words of a coordinate map
-    const int64_t per = ((nwords + ST_WARPS - 1) / ST_WARPS + 127) & ~(int64_t)127;   // map words per stretch: whole 512-byte rows
     auto stamp = [&](int slot, bool mine) { if (mine && tid == 0) A.st->trace[slot] = global_ns(); };
     const bool first_cta = blockIdx.x == 0;
     stamp(0, first_cta);
@@ -299,107 +300,110 @@ k_small_tail(const SmallArgs A) {
     if (!small_grid_barrier(A, 3, &s_flag)) return;
     stamp(5, first_cta);
 
-    // ---------------- phase 4: marks ----------------
+    // ---------------- phase 4: ordered candidates (line 9) and the second round (line 10), by every CTA ----------------
+    // A warp owns, in each of its iterations, one SEGMENT of 128 consecutive coordinates (its 32 lanes hold 32
+    // consecutive groups of four).  4a: count the segment's coordinates above T (a) and equal to T (b); the counts go
+    // to seg_a / seg_b and are added to the counters of the segment's SUPER-segment (64 segments).  Grid barrier.
+    // 4b: a candidate's slot is the number of a's before it plus min(number of b's before it, Q) -- ties at T go to the
+    // smallest coordinates -- and "before it" = whole super-segments (block-wide scan of at most 512 counters) +
+    // earlier segments of its super-segment (64 counts, two loads per lane) + earlier lanes of its segment (warp
+    // scan).  The candidate list comes out ascending, each candidate's exact sum is read right where it is emitted.
     block_find_from_top<H3_BINS>(A.h3, rem2, sh, d3, rem3);
     const uint32_t T = (d1 << H1_SHIFT) | (d2 << H2_SHIFT) | d3, Q = rem3;
-    for_my_keys([&](int64_t i0, const uint32_t (&key)[4]) {
-        uint32_t gt = 0, eq = 0;
+    const int lane = tid & 31;
+    uint32_t* seg_a = A.map_a;                             // [ceil(d / 128)] of each, written by the owning warps
+    uint32_t* seg_b = A.map_b;
+    // keys of one segment's share of this lane: gt / eq masks over its four coordinates
+    auto lane_masks = [&](int64_t q, uint32_t& gt, uint32_t& eq) {
+        const int64_t i0 = q << 2;
+        uint32_t key[4];
+        if (i0 + 3 < A.d) {
+            const float4 t = __ldcg(reinterpret_cast<const float4*>(A.est + i0));
+            key[0] = key_of(t.x); key[1] = key_of(t.y); key[2] = key_of(t.z); key[3] = key_of(t.w);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) key[e] = i0 + e < A.d ? key_of(__ldcg(A.est + i0 + e)) : NO_ITEM;
+        }
+        gt = 0; eq = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             if (key[e] == NO_ITEM) continue;
             gt |= (key[e] > T ? 1u : 0u) << e;
             eq |= (key[e] == T ? 1u : 0u) << e;
         }
-        const int sh4 = (int)(i0 & 31);                    // a group of four never straddles a map word
-        if (gt) { atomicOr(A.map_a + (i0 >> 5), gt << sh4); atomicAdd(&A.st->chunk_a[(i0 >> 5) / per], (uint32_t)__popc(gt)); }
-        if (eq) { atomicOr(A.map_b + (i0 >> 5), eq << sh4); atomicAdd(&A.st->chunk_b[(i0 >> 5) / per], (uint32_t)__popc(eq)); }
-    });
+    };
+    for (int64_t q = gtid; q - lane < groups; q += gstride) {          // warp-uniform trip count
+        uint32_t gt, eq;
+        lane_masks(q, gt, eq);
+        const uint32_t ta = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(gt));
+        const uint32_t tb = __reduce_add_sync(0xFFFFFFFFu, (uint32_t)__popc(eq));
+        if (lane == 0) {
+            const int64_t seg = q >> 5;
+            seg_a[seg] = ta; seg_b[seg] = tb;
+            if (ta) atomicAdd(&A.st->sup_a[seg >> 6], ta);
+            if (tb) atomicAdd(&A.st->sup_b[seg >> 6], tb);
+        }
+    }
+    if (!small_grid_barrier(A, 4, &s_flag)) return;
+    stamp(11, first_cta);
+    {
+        uint32_t* s_sup_a = sh.hist;                       // exclusive prefixes over the super-segments
+        uint32_t* s_sup_b = sh.hist + ST_THREADS;
+        const int64_t nsuper = (((A.d + 127) >> 7) + 63) >> 6;         // <= ST_THREADS since d <= SMALL_MAX_D
+        const uint32_t ca = tid < nsuper ? __ldcg(&A.st->sup_a[tid]) : 0u, cb = tid < nsuper ? __ldcg(&A.st->sup_b[tid]) : 0u;
+        uint32_t ea, eb;
+        block_excl_scan2(ca, cb, s_warp_a, s_warp_b, ea, eb);
+        s_sup_a[tid] = ea; s_sup_b[tid] = eb;
+        __syncthreads();
+        for (int64_t q = gtid; q - lane < groups; q += gstride) {
+            uint32_t gt, eq;
+            lane_masks(q, gt, eq);
+            const int64_t seg = (q - lane) >> 5, sup = seg >> 6;
+            const int within = (int)(seg & 63);
+            // a's and b's in the earlier segments of this super-segment
+            uint32_t pa = (lane < within ? __ldcg(seg_a + (sup << 6) + lane) : 0u) + (lane + 32 < within ? __ldcg(seg_a + (sup << 6) + 32 + lane) : 0u);
+            uint32_t pb = (lane < within ? __ldcg(seg_b + (sup << 6) + lane) : 0u) + (lane + 32 < within ? __ldcg(seg_b + (sup << 6) + 32 + lane) : 0u);
+            pa = __reduce_add_sync(0xFFFFFFFFu, pa);
+            pb = __reduce_add_sync(0xFFFFFFFFu, pb);
+            if (__ballot_sync(0xFFFFFFFFu, (gt | eq) != 0u) == 0u) continue;      // nothing to emit in this segment
+            const uint32_t packed = (uint32_t)__popc(gt) | ((uint32_t)__popc(eq) << 16);   // at most 4 each
+            uint32_t incl = packed;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+                if (lane >= off) incl += o;
+            }
+            uint32_t a = s_sup_a[sup] + pa + ((incl - packed) & 0xFFFFu), b = s_sup_b[sup] + pb + ((incl - packed) >> 16);
+            uint32_t bits = gt | eq;
+            while (bits) {
+                const int e = __ffs(bits) - 1;
+                bits &= bits - 1;
+                uint32_t slot = 0xFFFFFFFFu;
+                if ((gt >> e) & 1u) { slot = a + (b < Q ? b : Q); ++a; }
+                else { if (b < Q) slot = a + b; ++b; }
+                if (slot < A.ncand) {
+                    const int64_t coord = (q << 2) + e;
+                    A.cand_idx[slot] = (int32_t)coord;
+                    A.xs[slot] = __ldcg(A.xsum + coord);   // line 10: the accumulate kernel's sum over the workers
+                }
+            }
+        }
+    }
     if (!block_is_last(&A.st->ticket, sh)) return;
 
-    // ---------------- phase 5 (one CTA): candidates, second round, final top-k, line 13 ----------------
+    // ---------------- phase 5 (one CTA): final top-k (line 11) and line 13 ----------------
     stamp(6, true);
     int32_t* cand_s = reinterpret_cast<int32_t*>(st_dyn);
     float* xs_s = reinterpret_cast<float*>(st_dyn) + A.ncand;
-    // Warp w walks stretch w of the maps (how many marks each stretch holds was counted in phase 4), 128 words per
-    // step: lane l holds words 4l .. 4l+3 of the step, so that every load instruction reads 512 contiguous bytes
-    // Order inside a stretch is (step, lane, word, bit) = ascending coordinate.  Measured at d = 2^20 (2 x 128 KiB of
-    // maps, 2,000 marks): 13 us, of which 1.2 us are the loads -- the rest is instruction issue on this one SM (about
-    // 300 warp instructions per step and warp); the same loop not unrolled (batch in local memory) takes 20 us.
-    const int lane = tid & 31, warp = tid >> 5;
-    for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) cand_s[m] = 0;     // consistent histograms fill every slot
-    uint32_t run_a = 0, run_b = 0, mine_a = 0, mine_b = 0;
-    {
-        const uint32_t ca = lane < ST_WARPS ? __ldcg(&A.st->chunk_a[lane]) : 0u;
-        const uint32_t cb = lane < ST_WARPS ? __ldcg(&A.st->chunk_b[lane]) : 0u;
-        for (int w = 0; w < ST_WARPS; ++w) {
-            const uint32_t ta = __shfl_sync(0xFFFFFFFFu, ca, w), tb = __shfl_sync(0xFFFFFFFFu, cb, w);
-            if (w < warp) { run_a += ta; run_b += tb; }
-            if (w == warp) { mine_a = ta; mine_b = tb; }
-        }
-    }
-    __syncthreads();                                       // cand_s is cleared before any warp fills its slots
-    stamp(11, true);
-    const int64_t w_lo = (int64_t)warp * per, w_hi = w_lo + per < nwords ? w_lo + per : nwords;
-    if (mine_a | mine_b) {                                 // warp-uniform
-        for (int64_t w0 = w_lo; w0 < w_hi; w0 += 8 * 128) {
-            // eight steps per round trip to L2.  The loads are unconditional: the maps are padded with zero words to
-            // a multiple of 64 and rows beyond the stretch's end are masked out below
-            uint4 a4[8], b4[8];
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const int64_t w = w0 + q * 128 + 4 * lane;
-                const int64_t wl = w < w_hi ? w : w_lo;
-                a4[q] = __ldcg(reinterpret_cast<const uint4*>(A.map_a + wl));
-                b4[q] = __ldcg(reinterpret_cast<const uint4*>(A.map_b + wl));
-            }
-#pragma unroll
-            for (int q = 0; q < 8; ++q) {
-                const int64_t w = w0 + q * 128 + 4 * lane;
-                uint32_t wa[4] = {a4[q].x, a4[q].y, a4[q].z, a4[q].w}, wb[4] = {b4[q].x, b4[q].y, b4[q].z, b4[q].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (w + e >= w_hi) { wa[e] = 0u; wb[e] = 0u; }
-                const uint32_t na = __popc(wa[0]) + __popc(wa[1]) + __popc(wa[2]) + __popc(wa[3]);
-                const uint32_t nb = __popc(wb[0]) + __popc(wb[1]) + __popc(wb[2]) + __popc(wb[3]);
-                if (__ballot_sync(0xFFFFFFFFu, (na | nb) != 0u) == 0u) continue;        // an empty step
-                uint32_t packed = na | (nb << 16), incl = packed;                        // at most 128 marks per lane
-#pragma unroll
-                for (int off = 1; off < 32; off <<= 1) {
-                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, off);
-                    if (lane >= off) incl += o;
-                }
-                const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                uint32_t a = run_a + ((incl - packed) & 0xFFFFu), b = run_b + ((incl - packed) >> 16);
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    uint32_t bits = wa[e] | wb[e];
-                    while (bits) {
-                        const int bit = __ffs(bits) - 1;
-                        bits &= bits - 1;
-                        uint32_t slot = 0xFFFFFFFFu;
-                        if ((wa[e] >> bit) & 1u) { slot = a + (b < Q ? b : Q); ++a; }
-                        else { if (b < Q) slot = a + b; ++b; }
-                        if (slot < A.ncand) {
-                            const int32_t coord = (int32_t)(((w + e) << 5) + bit);
-                            cand_s[slot] = coord;
-                            A.cand_idx[slot] = coord;
-                        }
-                    }
-                }
-                run_a += tot & 0xFFFFu;
-                run_b += tot >> 16;
-            }
-        }
-    }
     for (int b = tid; b < H1_BINS; b += ST_THREADS) sh.hist[b] = 0;
     __syncthreads();
     stamp(7, true);
-    // line 10: one read per candidate of the sums the accumulate kernel left
     for (uint32_t m = tid; m < A.ncand; m += ST_THREADS) {
-        const uint32_t i = (uint32_t)cand_s[m];
-        const float x = (int64_t)i < A.d ? __ldcg(A.xsum + i) : 0.0f;
+        const uint32_t i = (uint32_t)__ldcg(A.cand_idx + m);
+        const bool ok = (int64_t)i < A.d;                  // consistent histograms fill every slot with a coordinate
+        const float x = ok ? __ldcg(A.xs + m) : 0.0f;
+        cand_s[m] = ok ? (int32_t)i : 0;
         xs_s[m] = x;
-        A.xs[m] = x;
         atomicAdd(&sh.hist[key_of(x) >> H1_SHIFT], 1u);
     }
     __syncthreads();

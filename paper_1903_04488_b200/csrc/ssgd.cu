@@ -48,11 +48,11 @@ constexpr size_t ALIGN = 256;
 constexpr int TIMING_SLOTS = 256;
 // ssgd_sketch_accumulate goes through the workers one launch at a time once all W tables together exceed this
 constexpr size_t WORKER_MAJOR_MIN_BYTES = (size_t)32 << 20;
-// AUTO takes the one-kernel tail up to this many coordinates and candidates.  Measured on B200, whole step,
-// fused / chain of launches: d = 2^20, W = 4, ncand = 2000: 0.109 / 0.127 ms; d = 2^21, W = 4, ncand = 4000: 0.181 /
-// 0.210; d = 2e6, W = 16, ncand = 16000: 0.290 / 0.281 (the last block's serial part grows with ncand)
+// AUTO takes the one-kernel tail up to this many coordinates (and as many candidates as it can hold).  Measured on
+// B200, whole step warm, one kernel / chain of launches: d = 2^20, W = 4, ncand = 2000: 0.097 / 0.128 ms; d = 2^21,
+// W = 4, ncand = 4000: 0.156 / 0.210; d = 2e6, W = 16, ncand = 16000: 0.249 / 0.281.  From 2^21 coordinates on the
+// chain prunes with the bucket bitmap, which the dense estimates of the one-kernel tail do not beat.
 constexpr int64_t SMALL_AUTO_MAX_D = (int64_t)1 << 21;
-constexpr int64_t SMALL_AUTO_MAX_NCAND = 4096;
 constexpr int64_t SMALL_INLINE_ZERO_MAX = 65536;            // eager line 13 inside the tail kernel up to this many k*W
 constexpr int EV_PER_STEP = SSGD_NSTAGES + 1;
 inline size_t up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
@@ -77,15 +77,16 @@ void derive_params(uint64_t seed, int32_t r, HashParams& hp) {
 
 void layout(ssgd_ctx* x, int64_t ncand_max) {
     size_t o = 0;
-    // the head, cleared at the start of every step.  What the one-kernel tail of small problems needs comes first
-    // (table, the two coordinate maps, its barrier state, H1-H3 and state of the candidate selection), so that its
-    // memset stops at off_h19_c
+    // the head, cleared at the start of every step.  What the one-kernel tail of small problems needs cleared comes
+    // first (table, its barrier state and counters, H1-H3 and state of the candidate selection), so that its memset
+    // stops at zero_small_bytes
     x->off_table = o;   o += up((size_t)x->r * x->c * 4);
-    x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
-    x->off_maps = o;    o += 2 * x->map_bytes;
     x->off_small = o;   o += up(sizeof(SmallState));
     x->off_hist_c = o;  o += up((size_t)SEL_HIST_WORDS * 4);
     x->off_state_c = o; o += up(sizeof(SelState));
+    x->zero_small_bytes = o;
+    x->map_bytes = up((size_t)((x->d + 31) / 32) * 4);
+    x->off_maps = o;    o += 2 * x->map_bytes;
     x->off_h19_c = o;   o += up((size_t)H19_BINS * 4);
     x->off_hist_f = o;  o += up((size_t)SEL_HIST_WORDS * 4);
     x->off_h19_f = o;   o += up((size_t)H19_BINS * 4);
@@ -225,8 +226,7 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
 // (measured on B200 against the chain of short launches).
 bool use_small(const ssgd_ctx* x, int64_t ncand) {
     if (x->prune_mode == SSGD_PRUNE_FUSED) return small_tail_applicable(x, ncand);
-    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D &&
-           ncand <= SMALL_AUTO_MAX_NCAND;
+    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D;
 }
 
 // Whether ssgd_step takes the pruned first pass + selection on the survivor list (filter_unsketch.cuh,
@@ -568,8 +568,9 @@ int ssgd_unsketch_candidates(ssgd_ctx* x, const float* merged, int64_t ncand, in
     if (est_all && !aligned16(est_all)) return SSGD_EALIGN;
     if ((e = ensure_device(x))) return e;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->off_hist_f - x->off_hist_c, st), "memset hist");
-    x->launches++;
+    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->zero_small_bytes - x->off_hist_c, st), "memset hist");   // H1-H3, state
+    CU(cudaMemsetAsync(x->ws + x->off_h19_c, 0, x->off_hist_f - x->off_h19_c, st), "memset hist");           // 2^19-bin table
+    x->launches += 2;
     float* est = est_all ? est_all : reinterpret_cast<float*>(x->ws + x->off_est);
     return unsketch_select(x, merged, ncand, cand_idx, cand_est, est, st);
 }
@@ -602,7 +603,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     const bool small = use_small(x, ncand);
     if (x->prune_mode == SSGD_PRUNE_FUSED && !small) return SSGD_EINVAL;
     // table, histograms, selection state: one memset (the error flag is sticky until ssgd_status)
-    CU(cudaMemsetAsync(x->ws, 0, small ? x->off_h19_c : x->off_err, st), "memset workspace head");
+    CU(cudaMemsetAsync(x->ws, 0, small ? x->zero_small_bytes : x->off_err, st), "memset workspace head");
     x->launches++;
     float* merged = reinterpret_cast<float*>(x->ws + x->off_table);
     AccumArgs A;
@@ -739,10 +740,11 @@ int ssgd_heavymix(ssgd_ctx* x, const float* merged, uint64_t fill_seed, int32_t*
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (x->pending_dirty && (e = flush_pending(x, st))) return e;   // line 5 reads v
     // histograms + state of the candidate selection, and the HEAVYMIX state
-    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->off_hist_f - x->off_hist_c, st), "memset hist");
+    CU(cudaMemsetAsync(x->ws + x->off_hist_c, 0, x->zero_small_bytes - x->off_hist_c, st), "memset hist");   // H1-H3, state
+    CU(cudaMemsetAsync(x->ws + x->off_h19_c, 0, x->off_hist_f - x->off_h19_c, st), "memset hist");           // 2^19-bin table
     CU(cudaMemsetAsync(x->ws + x->off_hist_f, 0, x->off_sp_hist - x->off_hist_f, st), "memset hist");
     CU(cudaMemsetAsync(x->ws + x->off_hm, 0, sizeof(HeavymixState), st), "memset heavymix state");
-    x->launches += 3;
+    x->launches += 4;
     HeavymixArgs A;
     A.table = merged; A.c = x->c; A.d = x->d; A.r = x->r; A.hp = x->hp; A.bk = x->bk;
     A.hm = reinterpret_cast<HeavymixState*>(x->ws + x->off_hm);

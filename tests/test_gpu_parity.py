@@ -289,9 +289,9 @@ def test_fused_tail_lockstep(cuda_device, cfg, steps, zero):
     for t in range(steps):
         check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o, flush=(t == steps - 1))
     # memset + accumulate + tail (+ k_zero when k*W is too large for the tail) per step; check_step adds the dense
-    # stage call (5 launches) and the last one a flush
+    # stage call (two memsets and four kernels) and the last one a flush
     per_step = 3 + (1 if zero == S.ZERO_EAGER and cfg.k * cfg.W > 65536 else 0)
-    assert eng.launch_count() - n0 == steps * (per_step + 5) + 1
+    assert eng.launch_count() - n0 == steps * (per_step + 6) + 1
 
 
 def test_fused_tail_is_refused_where_it_does_not_apply(cuda_device):
@@ -736,6 +736,29 @@ def test_stage_calls_apply_a_pending_zero_out_first(cuda_device):
     before_u = u.clone()
     eng.sketch_accumulate(torch.zeros_like(u), 0.0, tables)   # rho = 0, g = 0: u <- 0, v <- v
     assert (u == 0).all() and (v[:, chosen.long()] == 0).all() and (before_u[:, chosen.long()] != 0).any()
+
+
+# ------------------------------------------------------------------------------------------------
+# every call works on the stream it is given
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("prune", [S.PRUNE_FUSED, S.PRUNE_ON, S.PRUNE_OFF])
+def test_steps_on_a_side_stream(cuda_device, prune):
+    """The library only enqueues on the caller's stream (the binding passes torch's current stream): three steps on
+    a non-default stream, with the gradients produced on that stream right before each step and no synchronisation
+    in between, in lock step with the oracle."""
+    cfg = wl.C2.scaled(d=400_003, W=3, c=8192, ncand=3000, k=1500)
+    dev = cuda_device
+    eng, orc, u, v = make(cfg, dev)
+    eng.set_prune_mode(prune)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, dev)
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for t in range(3):
+            g = wl.gradients(st, t)
+            check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o, flush=(t == 2))
+    side.synchronize()
 
 
 # ------------------------------------------------------------------------------------------------
