@@ -123,7 +123,10 @@ int ssgd_set_zero_mode(ssgd_ctx* ctx, int32_t mode);
  * context stays usable. */
 int ssgd_set_wait_limit_ns(ssgd_ctx* ctx, int64_t ns);
 /* Test hook: thread block (block_plus_one - 1) of those kernels leaves without ever arriving at its barriers, so
- * that the others' waits run out (nothing hangs, nothing faults); 0 switches the hook off. */
+ * that the others' waits run out (nothing hangs, nothing faults); 0 switches the hook off.  -1: ssgd_step behaves as
+ * if the device had refused the cooperative launch of the FUSED tail (which happens when it cannot hold one thread
+ * block per SM at once, e.g. with SMs taken by another context): under SSGD_PRUNE_AUTO the step then takes the chain
+ * of ordinary launches, and so do the following steps; under SSGD_PRUNE_FUSED it returns SSGD_ECUDA. */
 int ssgd_test_withhold_block(ssgd_ctx* ctx, int32_t block_plus_one);
 /* Applies a deferred zero-out to u and v now (device pointers bound by ssgd_bind), on `stream`.  Cheap when
  * nothing is pending (one pass over d/8 bytes).  It always launches: the marks may come from a replayed CUDA

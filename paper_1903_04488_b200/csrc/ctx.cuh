@@ -60,6 +60,7 @@ struct ssgd_ctx {
     int device; int sm_count; int max_smem_optin;
     int kt_blocks_per_sm;   // residency of the bulk-copy pipeline kernel (0 = not queried yet)
     int small_grid;         // CTAs of the one-kernel tail (0 = not queried yet)
+    bool small_refused;     // a cooperative launch was refused: AUTO stays with the chain of ordinary launches
     uint64_t wait_ns;       // limit of every device-side wait (grid barriers, mbarriers)
     int32_t withhold;       // test hook: this CTA (1-based; 0 = none) never arrives, so the others' waits run out
     int64_t launches;
@@ -161,6 +162,7 @@ bool use_filter(const ssgd_ctx* x);
 int launch_sparse(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st);
 int launch_heavymix_keys(ssgd_ctx* x, const HeavymixArgs& A, cudaStream_t st);
 // defined in launch_small.cu
+constexpr int SMALL_TAIL_REFUSED = 1;    // launch_small_tail: the cooperative launch does not fit the device right now
 bool small_tail_applicable(const ssgd_ctx* x, int64_t ncand);
 int launch_small_tail(ssgd_ctx* x, SmallArgs& A, cudaStream_t st);
 

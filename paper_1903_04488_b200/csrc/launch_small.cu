@@ -43,7 +43,14 @@ static int launch_small_tail_t(ssgd_ctx* x, SmallArgs& A, cudaStream_t st) {
         x->small_grid = x->sm_count;                       // one CTA per SM: co-resident by the query above
     }
     cfg.gridDim = dim3((unsigned)x->small_grid);
-    CU(cudaLaunchKernelEx(&cfg, kern, A), "launch k_small_tail");
+    const cudaError_t le = A.withhold < 0 ? cudaErrorCooperativeLaunchTooLarge : cudaLaunchKernelEx(&cfg, kern, A);
+    if (le == cudaErrorCooperativeLaunchTooLarge || le == cudaErrorLaunchOutOfResources) {
+        // the device cannot hold one block per SM at once right now (SMs taken by another context, or the test
+        // hook): nothing was launched; the caller takes the chain of ordinary launches instead
+        if (A.withhold >= 0) cudaGetLastError();
+        return SMALL_TAIL_REFUSED;
+    }
+    if (le != cudaSuccess) return cuda_fail(x, le, "launch k_small_tail");
     LAUNCHED("k_small_tail");
     return SSGD_OK;
 }

@@ -226,7 +226,7 @@ SparseBuffers sparse_buffers(ssgd_ctx* x) {
 // (measured on B200 against the chain of short launches).
 bool use_small(const ssgd_ctx* x, int64_t ncand) {
     if (x->prune_mode == SSGD_PRUNE_FUSED) return small_tail_applicable(x, ncand);
-    return x->prune_mode == SSGD_PRUNE_AUTO && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D;
+    return x->prune_mode == SSGD_PRUNE_AUTO && !x->small_refused && small_tail_applicable(x, ncand) && x->d <= SMALL_AUTO_MAX_D;
 }
 
 // Whether ssgd_step takes the pruned first pass + selection on the survivor list (filter_unsketch.cuh,
@@ -365,7 +365,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->insert_mode = SSGD_INSERT_AUTO;
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
-    x->small_grid = 0; x->wait_ns = 2000000000ull; x->withhold = 0;
+    x->small_grid = 0; x->small_refused = false; x->wait_ns = 2000000000ull; x->withhold = 0;
     x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
@@ -642,7 +642,15 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
         T.zero_inline = (!deferred && x->k * (int64_t)x->W <= SMALL_INLINE_ZERO_MAX) ? 1 : 0;
         T.wait_ns = x->wait_ns; T.withhold = x->withhold;
         T.errflag = reinterpret_cast<int32_t*>(x->ws + x->off_err);
-        if ((e = launch_small_tail(x, T, st))) return e;
+        e = launch_small_tail(x, T, st);
+        if (e == SMALL_TAIL_REFUSED) {
+            if (x->prune_mode == SSGD_PRUNE_FUSED) { x->last_error = "cooperative launch refused: the device cannot hold one block per SM at once"; return SSGD_ECUDA; }
+            x->small_refused = true;                       // AUTO: this step and the following ones take the chain
+            CU(cudaMemsetAsync(x->ws + x->zero_small_bytes, 0, x->off_err - x->zero_small_bytes, st), "memset workspace head");
+            x->launches++;
+            goto chain;
+        }
+        if (e) return e;
         if ((e = mark(x, 2, st)) || (e = mark(x, 3, st))) return e;
         if (deferred) {
             x->pending_dirty = true;
@@ -655,6 +663,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
         if (x->timing && x->ev_steps < TIMING_SLOTS) x->ev_steps++;
         return SSGD_OK;
     }
+chain:
     const bool sparse = use_sparse(x, ncand);
     if (sparse) {
         if ((e = unsketch_select_sparse(x, merged, ncand, cand, st, A.xsum))) return e;
@@ -686,7 +695,7 @@ int ssgd_set_wait_limit_ns(ssgd_ctx* x, int64_t ns) {
 }
 
 int ssgd_test_withhold_block(ssgd_ctx* x, int32_t block_plus_one) {
-    if (!x || block_plus_one < 0) return SSGD_EINVAL;
+    if (!x || block_plus_one < -1) return SSGD_EINVAL;
     x->withhold = block_plus_one;
     return SSGD_OK;
 }

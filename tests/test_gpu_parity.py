@@ -309,6 +309,36 @@ def test_fused_tail_is_refused_where_it_does_not_apply(cuda_device):
     assert eng.status() == S.OK
 
 
+def test_refused_cooperative_launch_falls_back_to_the_chain(cuda_device):
+    """If the device cannot hold the one-kernel tail's grid at once, the runtime refuses the cooperative launch
+    (simulated by the test hook: nothing is launched).  Under AUTO the same step goes on as the chain of ordinary
+    launches -- same results -- and later steps do not try again; under FUSED the call reports the refusal."""
+    cfg = wl.C2.scaled(d=300_001, W=3, c=8192, ncand=3000, k=1500)
+    eng, orc, u, v = make(cfg, cuda_device)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    check_step(orc, eng, wl.gradients(st, 0), cfg.rho, cfg.ncand, u_o, v_o)          # AUTO: one kernel
+    eng.test_withhold_block(-1)
+    n0 = eng.launch_count()
+    check_step(orc, eng, wl.gradients(st, 1), cfg.rho, cfg.ncand, u_o, v_o)          # refused: the chain, same step
+    n_refused = eng.launch_count() - n0
+    eng.test_withhold_block(0)
+    n0 = eng.launch_count()
+    check_step(orc, eng, wl.gradients(st, 2), cfg.rho, cfg.ncand, u_o, v_o, flush=True)   # stays with the chain
+    assert eng.launch_count() - n0 - 1 == n_refused - 1        # one memset less than in the step that was refused
+    assert n_refused > 3 + 6
+    eng2, _, _, _ = make(cfg, cuda_device)
+    eng2.set_prune_mode(S.PRUNE_FUSED)
+    eng2.test_withhold_block(-1)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=cuda_device)
+    ov = torch.empty(cfg.k, device=cuda_device)
+    with pytest.raises(S.SsgdError) as e:
+        eng2.step(wl.gradients(st, 0), cfg.rho, cfg.ncand, oi, ov)
+    assert e.value.code == S.ECUDA
+    eng2.test_withhold_block(0)
+    eng2.flush()
+
+
 def test_a_grid_barrier_wait_that_runs_out_is_reported_and_nothing_hangs(cuda_device):
     """One block of the cooperative tail is withheld (it returns before the first grid barrier), so the others'
     bounded waits run out after the configured limit: the kernel returns, ssgd_status reports SSGD_EDEVICE once,
