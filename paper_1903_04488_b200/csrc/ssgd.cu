@@ -14,10 +14,11 @@
 //   list_select.cuh     k_list_hist, k_list_mark, k_map_emit: exact top-ncand of the survivor list
 //   select.cuh          k_sel_pass23 (k_sel_pass2/3), k_sel_count: exact radix select with ordered compaction
 //                       (lines 9, 11)
-//   heavymix.cuh        k_row_sumsq, k_heavymix_keys: Algorithm 1
+//   small_tail.cuh      k_small_tail: lines 9-13 as one cooperative kernel (small problems)
+//   heavymix.cuh        k_row_sumsq, k_heavymix_keys, k_heavymix_rekey: Algorithm 1
 //   hash.cuh, estimate.cuh   the hash family and the median-of-r estimate
-// The kernels instantiated per (rows, power-of-two columns) are launched from launch_accum.cu and
-// launch_unsketch.cu; ctx.cuh holds what the units share.
+// The kernels instantiated per (rows, power-of-two columns) are launched from launch_accum.cu,
+// launch_unsketch.cu and launch_small.cu; ctx.cuh holds what the units share.
 // HBM-bound work is the accumulate+insert kernel (20 bytes per worker-coordinate); nothing here is a dense
 // contraction, so there are no tensor-core instructions.
 #include <cuda_bf16.h>

@@ -26,8 +26,8 @@ constexpr int K3_GRID = 4;
 
 
 // ------------------------------------------------------------------------------------------------
-// K1 (plain-load form): momentum + error accumulation + sketch insert.  ssgd_step's default up to 128 workers
-// (the bulk-copy pipeline of accum_tma.cuh beyond); also the per-worker tables of ssgd_sketch_accumulate and the
+// K1 (plain-load form): momentum + error accumulation + sketch insert.  ssgd_step's default below 64 workers
+// (the bulk-copy pipeline of accum_tma.cuh from there on); also the per-worker tables of ssgd_sketch_accumulate and the
 // shared-memory table variant.
 // ------------------------------------------------------------------------------------------------
 enum InsertMode { INS_MERGED_GLOBAL = 0, INS_PER_WORKER = 1, INS_MERGED_SMEM = 2, INS_MERGED_TMA = 3 };
