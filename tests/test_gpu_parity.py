@@ -666,6 +666,39 @@ def test_step_can_be_captured_in_a_cuda_graph(cuda_device):
         assert int((v[0, :cfg.d] == 0).sum().item()) >= cfg.k
 
 
+def test_one_kernel_tail_can_be_captured_in_a_cuda_graph(cuda_device):
+    """The small-problem step (memset, accumulate kernel, one cooperative kernel) can be captured and replayed too;
+    integer gradients and rho = 1/2 make every operation exact, so a replay from zero state must reproduce the eager
+    step bit for bit."""
+    dev = cuda_device
+    cfg = wl.C2.scaled(d=300_001, W=3, c=8192, ncand=3000, k=1500)
+    gen = torch.Generator(device=dev).manual_seed(77)
+    g = torch.zeros((cfg.W, cfg.ld), device=dev)
+    g[:, :cfg.d] = torch.randint(-30, 31, (cfg.W, cfg.d), generator=gen, device=dev).float()
+    g[:, 11:cfg.d:101] += 64.0
+    eng, _, u, v = make(cfg, dev)
+    eng.set_zero_mode(S.ZERO_EAGER)
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=dev)
+    ov = torch.empty(cfg.k, device=dev)
+    eng.step(g, 0.5, cfg.ncand, oi, ov)                    # warm-up: device queries, function attributes
+    assert eng.status() == S.OK
+    eager_idx, eager_val, eager_v = oi.clone(), ov.clone(), v.clone()
+    stream = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    u.zero_(); v.zero_()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(stream):
+        with torch.cuda.graph(graph, stream=stream):
+            eng.step(g, 0.5, cfg.ncand, oi, ov)
+    for _ in range(2):
+        u.zero_(); v.zero_(); oi.zero_(); ov.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert eng.status() == S.OK
+        assert torch.equal(oi, eager_idx) and torch.equal(ov, eager_val) and torch.equal(v, eager_v)
+
+
 # ------------------------------------------------------------------------------------------------
 # seeded random shapes: every combination of sizes a user could pass, small enough for the oracle
 # ------------------------------------------------------------------------------------------------
