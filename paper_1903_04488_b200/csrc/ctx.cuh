@@ -20,6 +20,7 @@
 #include "estimate.cuh"
 #include "sparse_select.cuh"
 #include "filter_unsketch.cuh"
+#include "rowbits_unsketch.cuh"
 #include "heavymix.cuh"
 #include "step_kernels.cuh"
 #include "small_tail.cuh"
@@ -44,6 +45,9 @@ struct ssgd_ctx {
     size_t off_bm_full, off_bm_fold;                       // bit-per-bucket filter (filter_unsketch.cuh)
     int32_t bm_stride_full, bm_stride_fold, bm_fold;       // bm_fold < 0: the bitmap cannot be folded into shared memory
     bool filter_ready;                                     // shared-memory attribute of the filter kernel set
+    bool rowbits;                                          // the bitmap does not fit as a whole but row by row (rowbits_unsketch.cuh)
+    bool rowbits_ready;                                    // shared-memory attribute of k_row_bits set
+    size_t off_rowbits;                                    // [r][ceil(d/32)] result words of k_row_bits (rowbits only)
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)
     size_t off_pending;     // d-bit map of the deferred zero-out; survives from step to step
     int32_t zero_mode;      // SSGD_ZERO_DEFERRED / SSGD_ZERO_EAGER

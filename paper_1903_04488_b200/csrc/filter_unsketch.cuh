@@ -50,16 +50,34 @@ struct FilterArgs {
     int32_t stride_fold;      // words per row of the folded bitmap, a multiple of 4
     int32_t fold;             // s: a folded bit covers buckets [q << s, (q + 1) << s)
     int32_t r;
+    // 1: the bitmap is used unfolded, row by row (rowbits_unsketch.cuh); k_bitmap_build then counts the set bits and
+    // its last block decides between that filter and the table kernel (k_bitmap_fold does it for folded bitmaps)
+    int32_t decide_in_build;
+    float max_pass;           // decide_in_build: largest expected share of passing coordinates the filter is used for
 };
 
 #ifdef __CUDACC__
+
+// Probability that at least `need` of r independent bits of density p are set.
+__device__ __forceinline__ float binomial_tail(int r, int need, float p) {
+    float tail = 0.f;
+    for (int k = need; k <= r; ++k) {
+        float term = 1.f;                                  // C(r, k) p^k (1-p)^(r-k)
+        for (int t = 0; t < k; ++t) term *= p * (float)(r - t) / (float)(k - t);
+        for (int t = 0; t < r - k; ++t) term *= 1.f - p;
+        tail += term;
+    }
+    return tail;
+}
 
 // ---- bit per bucket ------------------------------------------------------------------------------------------
 // One warp per 32 words (1024 buckets) of one row: 32 coalesced loads, a ballot each; lane k keeps ballot k.
 static __global__ void __launch_bounds__(SEL_THREADS)
 k_bitmap_build(const FilterArgs F) {
+    __shared__ uint32_t s_last;
     pdl_trigger();
     pdl_wait();
+    uint32_t ones = 0;
     const uint32_t bin_lo = __ldcg(&F.A.sp.state->bin_lo);
     const int lane = threadIdx.x & 31;
     const int64_t tasks_per_row = (F.stride_full + 31) / 32;
@@ -83,19 +101,20 @@ k_bitmap_build(const FilterArgs F) {
             if (lane == k) mine = bal;
         }
         if (w0 + lane < F.stride_full) F.bm_full[j * F.stride_full + w0 + lane] = mine;
+        ones += __popc(mine);
     }
-}
-
-// Probability that at least `need` of r independent bits of density p are set.
-__device__ __forceinline__ float binomial_tail(int r, int need, float p) {
-    float tail = 0.f;
-    for (int k = need; k <= r; ++k) {
-        float term = 1.f;                                  // C(r, k) p^k (1-p)^(r-k)
-        for (int t = 0; t < k; ++t) term *= p * (float)(r - t) / (float)(k - t);
-        for (int t = 0; t < r - k; ++t) term *= 1.f - p;
-        tail += term;
+    if (F.decide_in_build) {                               // density of the unfolded bitmap -> filter or table kernel
+        for (int off = 16; off; off >>= 1) ones += __shfl_xor_sync(0xFFFFFFFFu, ones, off);
+        if (lane == 0 && ones) atomicAdd(&F.A.sp.state->fold_ones, ones);
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) s_last = atomicAdd(&F.A.sp.state->ticket[5], 1u) == gridDim.x - 1 ? 1u : 0u;
+        __syncthreads();
+        if (s_last && threadIdx.x == 0) {
+            const float p = fminf(1.f, (float)__ldcg(&F.A.sp.state->fold_ones) / ((float)F.r * (float)F.A.c));
+            F.A.sp.state->use_table = binomial_tail(F.r, (F.r + 1) / 2, p) > F.max_pass ? 1u : 0u;
+        }
     }
-    return tail;
 }
 
 // A folded bitmap is used only if it passes at most this share of the coordinates (estimated from its density as

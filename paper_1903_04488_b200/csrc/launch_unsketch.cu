@@ -21,7 +21,7 @@ int launch_unsketch(ssgd_ctx* x, const UnsketchArgs& A, cudaStream_t st) {
 // The first pass over all coordinates: the bit-per-bucket filter when the (folded) bitmap fits an SM's shared
 // memory, else the early-exit kernel that reads the table.
 bool use_filter(const ssgd_ctx* x) {
-    return x->prune_mode != SSGD_PRUNE_EARLY_EXIT && x->bm_fold >= 0 &&
+    return x->prune_mode != SSGD_PRUNE_EARLY_EXIT && (x->bm_fold >= 0 || x->rowbits) &&
            sizeof(SelShared) + FILTER_QUEUE_BYTES + (size_t)FILTER_MAX_WORDS * 4 <= (size_t)x->max_smem_optin;
 }
 
@@ -39,10 +39,34 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
         F.bm_full = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_full);
         F.bm_fold = reinterpret_cast<uint32_t*>(x->ws + x->off_bm_fold);
         F.stride_full = x->bm_stride_full; F.stride_fold = x->bm_stride_fold; F.fold = x->bm_fold; F.r = x->r;
+        F.decide_in_build = x->rowbits ? 1 : 0; F.max_pass = ROWBITS_MAX_PASS;
         const int64_t build_tasks = (int64_t)x->r * ((x->bm_stride_full + 31) / 32);
         CU(launch_pdl(st, k_bitmap_build, grid_for(build_tasks, SEL_WARPS, (int64_t)x->sm_count * 8), SEL_THREADS, 0, F),
            "launch k_bitmap_build");
         LAUNCHED("k_bitmap_build");
+        if (x->rowbits) {
+            // the bitmap row by row: r x (SMs / r) blocks each hold one row, then the r bits of every coordinate are counted
+            RowBitsArgs B;
+            B.F = F;
+            B.rowbits = reinterpret_cast<uint32_t*>(x->ws + x->off_rowbits);
+            B.words_per_row = (x->d + 31) / 32;
+            B.ranges = x->sm_count / x->r > 0 ? x->sm_count / x->r : 1;
+            auto kern = k_row_bits<POW2>;
+            if (!x->rowbits_ready) {
+                CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)FILTER_MAX_WORDS * 4)),
+                   "smem attribute");
+                x->rowbits_ready = true;
+            }
+            CU(launch_pdl(st, kern, x->r * B.ranges, RB_THREADS, (size_t)F.stride_full * 4, B), "launch k_row_bits");
+            LAUNCHED("k_row_bits");
+            CU(launch_pdl(st, k_rowbits_combine<R, POW2>, grid_for(B.words_per_row, SEL_THREADS, (int64_t)x->sm_count * 8),
+                          SEL_THREADS, 0, B), "launch k_rowbits_combine");
+            LAUNCHED("k_rowbits_combine");
+            SparseArgs G = A;
+            G.gated = 1;                                 // runs only if the bitmap turned out too dense (plain stream order)
+            k_unsketch_pruned<R, POW2><<<pruned_grid, SEL_THREADS, 0, st>>>(G);
+            LAUNCHED("k_unsketch_pruned");
+        } else {
         if (F.fold) {
             CU(launch_pdl(st, k_bitmap_fold, grid_for((int64_t)x->r * F.stride_fold, SEL_THREADS, (int64_t)x->sm_count * 8),
                           SEL_THREADS, 0, F), "launch k_bitmap_fold");
@@ -65,6 +89,7 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
             // resident while the declining filter kernel drains cost 4 ms (d = 9e7)
             k_unsketch_pruned<R, POW2><<<pruned_grid, SEL_THREADS, 0, st>>>(G);
             LAUNCHED("k_unsketch_pruned");
+        }
         }
     } else {
         CU(launch_pdl(st, k_unsketch_pruned<R, POW2>, pruned_grid, SEL_THREADS, 0, A), "launch k_unsketch_pruned");

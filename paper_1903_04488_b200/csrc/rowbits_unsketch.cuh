@@ -1,0 +1,191 @@
+// rowbits_unsketch.cuh -- Algorithm 3 line 9, first pass over all d coordinates, for sketches whose one-bit-per-
+// bucket filter (filter_unsketch.cuh) does not fit one SM's shared memory as a whole but does fit ROW BY ROW.
+//
+// The folded filter of filter_unsketch.cuh ORs neighbouring buckets into one bit until all r rows fit; what passes
+// the coarser test has to be re-checked on the full bitmap in global memory, r scattered L2 reads each, and with 4 or
+// more buckets per bit most coordinates pass.  Here nothing is folded:
+//
+//   k_row_bits          a thread block holds ONE row of the full bitmap (c bits <= 192 KiB) in shared memory and
+//                       evaluates that row's bit for every coordinate of its range: lane l of a warp walks the
+//                       coordinates l, l + 32, l + 64, ... (one add + conditional subtract per hash), a ballot turns
+//                       32 consecutive coordinates into one word, and after 32 ballots the warp stores 32 words
+//                       (1024 coordinates of row j) with one coalesced 128-byte store.  r x (SMs / r) blocks.
+//   k_rowbits_combine   reads the r result words of 32 coordinates (coalesced), counts per coordinate how many rows
+//                       have their bit set with a bit-sliced adder, and for the few coordinates with at least (r+1)/2
+//                       set bits computes the exact estimate from the table and appends it to the survivor list iff
+//                       its own bin is >= bin_lo.
+//
+// The survivor set is exactly { i : bin(|est_i|) >= bin_lo }, as with the other first-pass kernels, and the rest of
+// the stage (too-few-survivors rerun, selection on the list) is unchanged.  k_bitmap_build's last block measures the
+// bitmap's density; if so many buckets are above the threshold that most coordinates would pass, both kernels return
+// at once and the table-reading kernel enqueued behind them does the first pass.
+#pragma once
+#include <stdint.h>
+
+#include "estimate.cuh"
+#include "filter_unsketch.cuh"
+#include "hash.cuh"
+#include "select.cuh"
+#include "sparse_select.cuh"
+
+namespace ssgd {
+
+constexpr int RB_THREADS = 512;
+constexpr int RB_WARPS = RB_THREADS / 32;
+// The row-by-row filter is used if at most this share of the coordinates is expected to pass it (binomial tail of
+// the bitmap's density): beyond, exact estimates for nearly everyone cost more than the early-exit table kernel.
+constexpr float ROWBITS_MAX_PASS = 0.7f;
+
+struct RowBitsArgs {
+    FilterArgs F;
+    uint32_t* rowbits;        // [r][words_per_row]: bit i of row j = "row j's bucket of coordinate i is above the threshold"
+    int64_t words_per_row;    // ceil(d / 32)
+    int32_t ranges;           // blocks per row: block b works on row b % r, coordinate range b / r
+};
+
+#ifdef __CUDACC__
+
+template <bool POW2>
+__global__ void __launch_bounds__(RB_THREADS, 1)
+k_row_bits(const RowBitsArgs B) {
+    extern __shared__ __align__(16) uint32_t rb_bm[];      // row j of the full bitmap
+    const SparseArgs& A = B.F.A;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_trigger();
+    pdl_wait();
+    if (__ldcg(&A.sp.state->use_table) != 0u) return;      // too dense to prune: the table kernel behind runs
+    const int j = (int)(blockIdx.x % (unsigned)B.F.r);
+    const int64_t rho = blockIdx.x / (unsigned)B.F.r;
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(B.F.bm_full + (int64_t)j * B.F.stride_full);
+        const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rb_bm);
+        for (int w = tid; w < B.F.stride_full / 4; w += RB_THREADS)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)w * 16u), "l"(src + w) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
+    __syncthreads();
+    // chunks of 1024 coordinates; this block's chunks, then this warp's share of them (contiguous: the hash runs on)
+    const int64_t nchunks = (A.d + 1023) >> 10;
+    const int64_t per_cta = (nchunks + B.ranges - 1) / B.ranges;
+    const int64_t c_lo = rho * per_cta, c_hi = c_lo + per_cta < nchunks ? c_lo + per_cta : nchunks;
+    if (c_lo >= c_hi) return;
+    const int64_t per_warp = (c_hi - c_lo + RB_WARPS - 1) / RB_WARPS;
+    const int64_t w_lo = c_lo + warp * per_warp, w_hi = w_lo + per_warp < c_hi ? w_lo + per_warp : c_hi;
+    if (w_lo >= w_hi) return;
+    const HashRow hr = A.hp.row[j];
+    uint32_t i = (uint32_t)(w_lo << 10) + (uint32_t)lane;
+    uint32_t y = lin_hash(hr.a, hr.b, i);
+    const uint32_t step = mod_p31((uint64_t)hr.a * 32ull); // (a * 32) mod p: from coordinate i to i + 32
+    const uint32_t d32 = (uint32_t)A.d;
+    uint32_t* out = B.rowbits + (int64_t)j * B.words_per_row;
+    for (int64_t chunk = w_lo; chunk < w_hi; ++chunk) {
+        uint32_t keep = 0;
+#pragma unroll 8
+        for (int t = 0; t < 32; ++t) {
+            const uint32_t b = bucket_of<POW2>(y, A.bk);
+            const uint32_t bit = __funnelshift_r(rb_bm[b >> 5], 0u, b) & 1u;    // shift amount taken mod 32
+            const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit != 0u && i < d32);
+            if (lane == t) keep = word;
+            y = next_hash(y, step);
+            i += 32u;
+        }
+        const int64_t widx = (chunk << 5) + lane;
+        if (widx < B.words_per_row) out[widx] = keep;
+    }
+}
+
+// Exact estimate of one coordinate per lane (for the lanes that `have` one); appended to the survivor list iff its
+// own bin is >= bin_lo.  Every lane of the warp calls.
+template <int R, bool POW2>
+__device__ __forceinline__ void exact_append(const SparseArgs& A, uint32_t bin_lo, uint32_t i, bool have, uint32_t* s_hist) {
+    const int lane = threadIdx.x & 31;
+    float m = 0.f;
+    bool keep = false;
+    if (have) {
+        float rowv[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            uint32_t hb[1];
+            row_hashes<POW2, 1>(A.hp.row[j], A.bk, i, hb);
+            rowv[j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[0] & P31)), hb[0]);
+        }
+        m = median_of<R>(rowv);
+        keep = (key_of(m) >> H1_SHIFT) >= bin_lo;
+    }
+    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
+    if (bal == 0u) return;
+    uint32_t base = 0;
+    if (lane == 0) base = atomicAdd(&A.sp.state->n_surv, (uint32_t)__popc(bal));
+    base = __shfl_sync(0xFFFFFFFFu, base, 0);
+    if (keep) {
+        const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
+        if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)i; A.sp.list_est[pos] = m; }
+        atomicAdd(&s_hist[key_of(m) >> H1_SHIFT], 1u);
+    }
+}
+
+template <int R, bool POW2>
+__global__ void __launch_bounds__(SEL_THREADS)
+k_rowbits_combine(const RowBitsArgs B) {
+    __shared__ SelShared sh;
+    constexpr int NEED = (R + 1) / 2;
+    const SparseArgs& A = B.F.A;
+    const int lane = threadIdx.x & 31;
+    pdl_trigger();
+    for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
+    pdl_wait();
+    if (__ldcg(&A.sp.state->use_table) != 0u) return;
+    const uint32_t bin_lo = __ldcg(&A.sp.state->bin_lo);
+    __syncthreads();
+    const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
+    // warp-uniform trip count: the appends are warp-wide
+    for (int64_t w0 = (int64_t)blockIdx.x * SEL_THREADS + (threadIdx.x & ~31); w0 < B.words_per_row; w0 += stride) {
+        const int64_t w = w0 + lane;
+        // bit-sliced count (4 planes: r <= 15) of the rows whose bit is set, for 32 coordinates at once
+        uint32_t c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+        uint32_t rows[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) rows[j] = w < B.words_per_row ? __ldcs(B.rowbits + (int64_t)j * B.words_per_row + w) : 0u;
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            uint32_t carry = rows[j], t;
+            t = c0 & carry; c0 ^= carry; carry = t;
+            t = c1 & carry; c1 ^= carry; carry = t;
+            t = c2 & carry; c2 ^= carry; carry = t;
+            c3 ^= carry;
+        }
+        // pass = (count >= NEED), compared plane by plane from the top
+        const uint32_t plane[4] = {c0, c1, c2, c3};
+        uint32_t gt = 0u, eq = 0xFFFFFFFFu;
+#pragma unroll
+        for (int p = 3; p >= 0; --p) {
+            if ((NEED >> p) & 1) { eq &= plane[p]; }
+            else { gt |= eq & plane[p]; eq &= ~plane[p]; }
+        }
+        uint32_t pass = gt | eq;
+        while (__ballot_sync(0xFFFFFFFFu, pass != 0u)) {   // one coordinate per lane and round
+            const bool have = pass != 0u;
+            uint32_t i = 0;
+            if (have) { const int bit = __ffs(pass) - 1; pass &= pass - 1; i = (uint32_t)(w << 5) + (uint32_t)bit; }
+            exact_append<R, POW2>(A, bin_lo, i, have, sh.hist);
+        }
+    }
+    __syncthreads();
+    flush_hist<H1_BINS>(sh.hist, A.sp.h1);
+    if (block_is_last(&A.sp.state->ticket[1], sh)) {
+        const uint32_t n = __ldcg(&A.sp.state->n_surv);
+        if (n < A.ncand) {
+            // the sampled threshold was too high: empty the list and its histogram for the unpruned pass
+            for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) A.sp.h1[b] = 0;
+            if (threadIdx.x == 0) { A.sp.state->n_surv = 0; A.sp.state->fallback = 1u; }
+        } else {
+            uint32_t d1 = 0, rem1 = 1;
+            block_find_from_top<H1_BINS>(A.sp.h1, A.ncand, sh, d1, rem1);
+            if (threadIdx.x == 0) { A.sp.state->d1 = d1; A.sp.state->rem1 = rem1; }
+        }
+    }
+}
+
+#endif  // __CUDACC__
+}  // namespace ssgd

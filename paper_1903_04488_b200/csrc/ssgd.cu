@@ -123,6 +123,10 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_pending = o; o += x->map_bytes;
     x->off_bm_full = o; o += up((size_t)x->r * sf * 4);
     x->off_bm_fold = o; o += up((size_t)x->r * x->bm_stride_fold * 4);
+    // a bitmap that needs folding but whose single row fits shared memory is used unfolded, row by row
+    x->rowbits = x->bm_fold != 0 && sf <= FILTER_MAX_WORDS;
+    x->off_rowbits = o;
+    if (x->rowbits) o += up((size_t)x->r * (size_t)((x->d + 31) / 32) * 4);
     x->total_bytes = o;
 }
 
@@ -239,7 +243,7 @@ bool use_sparse(const ssgd_ctx* x, int64_t ncand) {
     if (x->d < (1 << 21) || ncand * 8 > x->d) return false;      // fixed costs outweigh the saving
     // an unfolded bucket bitmap pays for every r; behind a folded one the table kernel may have to run, which was
     // measured to pay for r = 5, 7, 9 only (r = 3: one row can be skipped; r = 15, ncand = 1.6e6: 5.8 vs 4.9 ms)
-    return x->bm_fold == 0 || (x->r >= 5 && x->r <= 9);
+    return x->bm_fold == 0 || (x->r >= 5 && x->r <= 9);   // (the row-by-row filter hands over to the table kernel the same way)
 }
 
 
@@ -367,7 +371,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
     x->small_grid = 0; x->small_refused = false; x->wait_ns = 2000000000ull; x->withhold = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->rowbits = false; x->rowbits_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT;
     *out = x;
     return SSGD_OK;
 }
