@@ -6,14 +6,15 @@
 // more buckets per bit most coordinates pass.  Here nothing is folded:
 //
 //   k_row_bits          a thread block holds ONE row of the full bitmap (c bits <= 192 KiB) in shared memory and
-//                       evaluates that row's bit for every coordinate of its range: lane l of a warp walks the
-//                       coordinates l, l + 32, l + 64, ... (one add + conditional subtract per hash), a ballot turns
-//                       32 consecutive coordinates into one word, and after 32 ballots the warp stores 32 words
-//                       (1024 coordinates of row j) with one coalesced 128-byte store.  r x (SMs / r) blocks.
+//                       evaluates that row's bit for every coordinate of its range: of each 1024 coordinates a
+//                       warp takes, lane l walks the 32 consecutive ones of result word l (one add + conditional
+//                       subtract per hash, one shared-memory load, two funnel shifts to append the bit), then
+//                       the warp stores its 32 words with one coalesced 128-byte store.
 //   k_rowbits_combine   reads the r result words of 32 coordinates (coalesced), counts per coordinate how many rows
 //                       have their bit set with a bit-sliced adder, and for the few coordinates with at least (r+1)/2
-//                       set bits computes the exact estimate from the table and appends it to the survivor list iff
-//                       its own bin is >= bin_lo.
+//                       set bits computes the exact estimate from the table (the warp's passing coordinates are
+//                       compacted in shared memory first, so that every lane has one) and appends it to the
+//                       survivor list iff its own bin is >= bin_lo: one reservation per warp and 1024 coordinates.
 //
 // The survivor set is exactly { i : bin(|est_i|) >= bin_lo }, as with the other first-pass kernels, and the rest of
 // the stage (too-few-survivors rerun, selection on the list) is unchanged.  k_bitmap_build's last block measures the
@@ -30,8 +31,7 @@
 
 namespace ssgd {
 
-constexpr int RB_THREADS = 512;
-constexpr int RB_WARPS = RB_THREADS / 32;
+constexpr int RB_MAX_THREADS = 1024;
 // The row-by-row filter is used if at most this share of the coordinates is expected to pass it (binomial tail of
 // the bitmap's density): beyond, exact estimates for nearly everyone cost more than the early-exit table kernel.
 constexpr float ROWBITS_MAX_PASS = 0.7f;
@@ -46,11 +46,12 @@ struct RowBitsArgs {
 #ifdef __CUDACC__
 
 template <bool POW2>
-__global__ void __launch_bounds__(RB_THREADS, 1)
+__global__ void __launch_bounds__(RB_MAX_THREADS)
 k_row_bits(const RowBitsArgs B) {
     extern __shared__ __align__(16) uint32_t rb_bm[];      // row j of the full bitmap
     const SparseArgs& A = B.F.A;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nthreads = blockDim.x, nwarps = nthreads >> 5;
     pdl_trigger();
     pdl_wait();
     if (__ldcg(&A.sp.state->use_table) != 0u) return;      // too dense to prune: the table kernel behind runs
@@ -59,7 +60,7 @@ k_row_bits(const RowBitsArgs B) {
     {
         const uint4* src = reinterpret_cast<const uint4*>(B.F.bm_full + (int64_t)j * B.F.stride_full);
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rb_bm);
-        for (int w = tid; w < B.F.stride_full / 4; w += RB_THREADS)
+        for (int w = tid; w < B.F.stride_full / 4; w += nthreads)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)w * 16u), "l"(src + w) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -70,68 +71,49 @@ k_row_bits(const RowBitsArgs B) {
     const int64_t per_cta = (nchunks + B.ranges - 1) / B.ranges;
     const int64_t c_lo = rho * per_cta, c_hi = c_lo + per_cta < nchunks ? c_lo + per_cta : nchunks;
     if (c_lo >= c_hi) return;
-    const int64_t per_warp = (c_hi - c_lo + RB_WARPS - 1) / RB_WARPS;
+    const int64_t per_warp = (c_hi - c_lo + nwarps - 1) / nwarps;
     const int64_t w_lo = c_lo + warp * per_warp, w_hi = w_lo + per_warp < c_hi ? w_lo + per_warp : c_hi;
     if (w_lo >= w_hi) return;
+    // lane l owns the 32 consecutive coordinates s .. s + 31 of each chunk, i.e. one result word: the hash advances
+    // by one add and a conditional subtract per coordinate, the bit is shifted into the word from the top
     const HashRow hr = A.hp.row[j];
-    uint32_t i = (uint32_t)(w_lo << 10) + (uint32_t)lane;
-    uint32_t y = lin_hash(hr.a, hr.b, i);
-    const uint32_t step = mod_p31((uint64_t)hr.a * 32ull); // (a * 32) mod p: from coordinate i to i + 32
+    uint32_t s = (uint32_t)(w_lo << 10) + (uint32_t)lane * 32u;
+    uint32_t y = lin_hash(hr.a, hr.b, s);
+    const uint32_t skip = mod_p31((uint64_t)hr.a * 992ull);   // from s + 32 to the lane's word of the next chunk
     const uint32_t d32 = (uint32_t)A.d;
     uint32_t* out = B.rowbits + (int64_t)j * B.words_per_row;
     for (int64_t chunk = w_lo; chunk < w_hi; ++chunk) {
-        uint32_t keep = 0;
-#pragma unroll 8
+        uint32_t word = 0;
+#pragma unroll
         for (int t = 0; t < 32; ++t) {
             const uint32_t b = bucket_of<POW2>(y, A.bk);
-            const uint32_t bit = __funnelshift_r(rb_bm[b >> 5], 0u, b) & 1u;    // shift amount taken mod 32
-            const uint32_t word = __ballot_sync(0xFFFFFFFFu, bit != 0u && i < d32);
-            if (lane == t) keep = word;
-            y = next_hash(y, step);
-            i += 32u;
+            const uint32_t bits = __funnelshift_r(rb_bm[b >> 5], 0u, b);     // bucket b's bit lowest (shift taken mod 32)
+            word = __funnelshift_r(word, bits, 1);                           // word >> 1 | lowest bit of `bits` << 31
+            y = next_hash(y, hr.a);
         }
+        y = next_hash(y, skip);
+        const uint32_t valid = d32 > s ? d32 - s : 0u;       // coordinates of this word below d
+        if (valid < 32u) word &= (1u << valid) - 1u;
         const int64_t widx = (chunk << 5) + lane;
-        if (widx < B.words_per_row) out[widx] = keep;
+        if (widx < B.words_per_row) out[widx] = word;
+        s += 1024u;
     }
 }
 
-// Exact estimate of one coordinate per lane (for the lanes that `have` one); appended to the survivor list iff its
-// own bin is >= bin_lo.  Every lane of the warp calls.
-template <int R, bool POW2>
-__device__ __forceinline__ void exact_append(const SparseArgs& A, uint32_t bin_lo, uint32_t i, bool have, uint32_t* s_hist) {
-    const int lane = threadIdx.x & 31;
-    float m = 0.f;
-    bool keep = false;
-    if (have) {
-        float rowv[R];
-#pragma unroll
-        for (int j = 0; j < R; ++j) {
-            uint32_t hb[1];
-            row_hashes<POW2, 1>(A.hp.row[j], A.bk, i, hb);
-            rowv[j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[0] & P31)), hb[0]);
-        }
-        m = median_of<R>(rowv);
-        keep = (key_of(m) >> H1_SHIFT) >= bin_lo;
-    }
-    const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
-    if (bal == 0u) return;
-    uint32_t base = 0;
-    if (lane == 0) base = atomicAdd(&A.sp.state->n_surv, (uint32_t)__popc(bal));
-    base = __shfl_sync(0xFFFFFFFFu, base, 0);
-    if (keep) {
-        const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
-        if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)i; A.sp.list_est[pos] = m; }
-        atomicAdd(&s_hist[key_of(m) >> H1_SHIFT], 1u);
-    }
-}
+// Per warp: the passing coordinates of 1024 (at most all of them) and the estimates of those that are kept.
+constexpr int RBC_QUEUE = 1024;
+constexpr size_t RBC_SMEM = (size_t)SEL_WARPS * RBC_QUEUE * 2 * 4;
 
 template <int R, bool POW2>
 __global__ void __launch_bounds__(SEL_THREADS)
 k_rowbits_combine(const RowBitsArgs B) {
+    extern __shared__ __align__(16) uint32_t rbc_smem[];
     __shared__ SelShared sh;
     constexpr int NEED = (R + 1) / 2;
     const SparseArgs& A = B.F.A;
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* q = rbc_smem + (size_t)warp * (RBC_QUEUE * 2);          // coordinates: passing ones, then (in place) kept ones
+    float* e = reinterpret_cast<float*>(q + RBC_QUEUE);                 // estimates of the kept ones
     pdl_trigger();
     for (int b = threadIdx.x; b < H1_BINS; b += SEL_THREADS) sh.hist[b] = 0;
     pdl_wait();
@@ -139,7 +121,7 @@ k_rowbits_combine(const RowBitsArgs B) {
     const uint32_t bin_lo = __ldcg(&A.sp.state->bin_lo);
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * SEL_THREADS;
-    // warp-uniform trip count: the appends are warp-wide
+    // warp-uniform trip count: the queue is the warp's
     for (int64_t w0 = (int64_t)blockIdx.x * SEL_THREADS + (threadIdx.x & ~31); w0 < B.words_per_row; w0 += stride) {
         const int64_t w = w0 + lane;
         // bit-sliced count (4 planes: r <= 15) of the rows whose bit is set, for 32 coordinates at once
@@ -164,12 +146,61 @@ k_rowbits_combine(const RowBitsArgs B) {
             else { gt |= eq & plane[p]; eq &= ~plane[p]; }
         }
         uint32_t pass = gt | eq;
-        while (__ballot_sync(0xFFFFFFFFu, pass != 0u)) {   // one coordinate per lane and round
-            const bool have = pass != 0u;
-            uint32_t i = 0;
-            if (have) { const int bit = __ffs(pass) - 1; pass &= pass - 1; i = (uint32_t)(w << 5) + (uint32_t)bit; }
-            exact_append<R, POW2>(A, bin_lo, i, have, sh.hist);
+        // the warp's passing coordinates, compacted: every lane then computes one exact estimate per round
+        const uint32_t mine = (uint32_t)__popc(pass);
+        uint32_t incl = mine;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+            if (lane >= off) incl += up;
         }
+        const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        if (total == 0u) continue;
+        uint32_t at = incl - mine;
+        while (pass) {
+            const int bit = __ffs(pass) - 1;
+            pass &= pass - 1u;
+            q[at++] = (uint32_t)(w << 5) + (uint32_t)bit;
+        }
+        __syncwarp();
+        uint32_t nk = 0;                                     // kept so far (<= coordinates read so far: in place)
+        for (uint32_t t0 = 0; t0 < total; t0 += 32u) {
+            const bool have = t0 + (uint32_t)lane < total;
+            const uint32_t i = have ? q[t0 + lane] : 0u;
+            float m = 0.f;
+            bool keep = false;
+            if (have) {
+                float rowv[R];
+#pragma unroll
+                for (int j = 0; j < R; ++j) {
+                    uint32_t hb[1];
+                    row_hashes<POW2, 1>(A.hp.row[j], A.bk, i, hb);
+                    rowv[j] = apply_sign(table_load(A.table + (int64_t)j * A.c + (hb[0] & P31)), hb[0]);
+                }
+                m = median_of<R>(rowv);
+                keep = (key_of(m) >> H1_SHIFT) >= bin_lo;
+            }
+            const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
+            __syncwarp();
+            if (keep) {
+                const uint32_t pos = nk + (uint32_t)__popc(bal & ((1u << lane) - 1u));
+                q[pos] = i;
+                e[pos] = m;
+                atomicAdd(&sh.hist[key_of(m) >> H1_SHIFT], 1u);
+            }
+            nk += (uint32_t)__popc(bal);
+        }
+        __syncwarp();
+        if (nk) {                                            // one reservation and coalesced stores per 1024 coordinates
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(&A.sp.state->n_surv, nk);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            for (uint32_t t = (uint32_t)lane; t < nk; t += 32u) {
+                const uint32_t pos = base + t;
+                if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)q[t]; A.sp.list_est[pos] = e[t]; }
+            }
+        }
+        __syncwarp();
     }
     __syncthreads();
     flush_hist<H1_BINS>(sh.hist, A.sp.h1);
