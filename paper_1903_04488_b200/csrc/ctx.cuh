@@ -46,6 +46,7 @@ struct ssgd_ctx {
     int32_t bm_stride_full, bm_stride_fold, bm_fold;       // bm_fold < 0: the bitmap cannot be folded into shared memory
     bool filter_ready;                                     // shared-memory attribute of the filter kernel set
     bool rowbits;                                          // the bitmap does not fit as a whole but row by row (rowbits_unsketch.cuh)
+    int rb_slices, rb_slice_words;                         // pieces each of its rows is cut into for that, words per piece
     bool rowbits_ready;                                    // shared-memory attribute of k_row_bits set
     size_t off_rowbits;                                    // [r][ceil(d/32)] result words of k_row_bits (rowbits only)
     uint32_t sample_rank;   // 0: derive the sample rank from ncand; else use this one (tests)

@@ -221,6 +221,21 @@ k_unsketch_filter(const FilterArgs F) {
     }
     __syncthreads();
 
+    // unfolded bitmaps (q3 is free): kept coordinates wait in q3 and go to the list 32 at a time, one reservation
+    // and two coalesced stores each -- reservations all hit one counter, and one per batch with a kept coordinate
+    // in it is what bounds the kernel when many pass (measured at 5 x 180,000, d = 7.3e7)
+    auto flush_kept = [&](int at_least) {
+        while (q3.count >= at_least) {
+            const int n = q3.count < 32 ? q3.count : 32;
+            uint32_t c = 0, mbits = 0;
+            const bool got = q3.pop(c, mbits, lane);
+            uint32_t base = 0;
+            if (lane == 0) base = atomicAdd(&A.sp.state->n_surv, (uint32_t)n);
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            const uint32_t pos = base + (uint32_t)lane;
+            if (got && pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)c; A.sp.list_est[pos] = __uint_as_float(mbits); }
+        }
+    };
     // exact estimate of one queued coordinate; append to the list iff its bin is >= bin_lo
     auto exact = [&](uint32_t i, bool have) {
         float m = 0.f;
@@ -236,6 +251,12 @@ k_unsketch_filter(const FilterArgs F) {
             m = median_of<R>(rowv);
             keep = (key_of(m) >> H1_SHIFT) >= bin_lo;
         }
+        if (keep) atomicAdd(&sh.hist[key_of(m) >> H1_SHIFT], 1u);
+        if (!FOLD) {
+            q3.push(keep, i, __float_as_uint(m), lane);
+            flush_kept(32);
+            return;
+        }
         const uint32_t bal = __ballot_sync(0xFFFFFFFFu, keep);
         if (bal == 0u) return;
         uint32_t base = 0;
@@ -244,7 +265,6 @@ k_unsketch_filter(const FilterArgs F) {
         if (keep) {
             const uint32_t pos = base + __popc(bal & ((1u << lane) - 1u));
             if (pos < A.sp.cap) { A.sp.list_idx[pos] = (int32_t)i; A.sp.list_est[pos] = m; }
-            atomicAdd(&sh.hist[key_of(m) >> H1_SHIFT], 1u);
         }
     };
     // folded bitmaps only: the rows whose folded bit was set (`rows`) are looked up in the full bitmap (global
@@ -309,6 +329,7 @@ k_unsketch_filter(const FilterArgs F) {
     }
     if (q2.count > 0) drain2();
     if (FOLD && q3.count > 0) { uint32_t c = 0, tag = 0; const bool got = q3.pop(c, tag, lane); exact(c, got); }
+    if (!FOLD) flush_kept(1);
 
     __syncthreads();
     flush_hist<H1_BINS>(sh.hist, A.sp.h1);

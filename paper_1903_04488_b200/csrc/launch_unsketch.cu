@@ -50,19 +50,21 @@ int launch_sparse_t(ssgd_ctx* x, const SparseArgs& A, cudaStream_t st) {
             B.F = F;
             B.rowbits = reinterpret_cast<uint32_t*>(x->ws + x->off_rowbits);
             B.words_per_row = (x->d + 31) / 32;
+            B.slices = x->rb_slices; B.slice_words = x->rb_slice_words;
             // two blocks per SM when two rows fit its shared memory (32 registers per thread: 2048 threads are resident)
-            const size_t row_bytes = (size_t)F.stride_full * 4;
+            const size_t row_bytes = B.slices > 1 ? (size_t)B.slice_words * 4 + 16 : (size_t)F.stride_full * 4;   // + the zero word
             const int per_sm = 2 * (row_bytes + 1024) <= (size_t)x->max_smem_optin ? 2 : 1;
-            B.ranges = x->sm_count * per_sm / x->r > 0 ? x->sm_count * per_sm / x->r : 1;
-            auto kern = k_row_bits<POW2>;
+            const int row_blocks = x->r * B.slices;
+            B.ranges = x->sm_count * per_sm / row_blocks > 0 ? x->sm_count * per_sm / row_blocks : 1;
+            auto kern = B.slices > 1 ? k_row_bits<POW2, true> : k_row_bits<POW2, false>;
             if (!x->rowbits_ready) {
-                CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)FILTER_MAX_WORDS * 4)),
+                CU(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)((size_t)FILTER_MAX_WORDS * 4 + 16)),
                    "smem attribute");
                 CU(cudaFuncSetAttribute(k_rowbits_combine<R, POW2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)RBC_SMEM),
                    "smem attribute");
                 x->rowbits_ready = true;
             }
-            CU(launch_pdl(st, kern, x->r * B.ranges, RB_MAX_THREADS, row_bytes, B), "launch k_row_bits");
+            CU(launch_pdl(st, kern, row_blocks * B.ranges, RB_MAX_THREADS, row_bytes, B), "launch k_row_bits");
             LAUNCHED("k_row_bits");
             CU(launch_pdl(st, k_rowbits_combine<R, POW2>, grid_for(B.words_per_row, SEL_THREADS, (int64_t)x->sm_count * 2),
                           SEL_THREADS, RBC_SMEM, B), "launch k_rowbits_combine");

@@ -1,5 +1,6 @@
 // rowbits_unsketch.cuh -- Algorithm 3 line 9, first pass over all d coordinates, for sketches whose one-bit-per-
-// bucket filter (filter_unsketch.cuh) does not fit one SM's shared memory as a whole but does fit ROW BY ROW.
+// bucket filter (filter_unsketch.cuh) does not fit one SM's shared memory as a whole but does fit ROW BY ROW, or a row
+// in up to RB_MAX_SLICES slices.
 //
 // The folded filter of filter_unsketch.cuh ORs neighbouring buckets into one bit until all r rows fit; what passes
 // the coarser test has to be re-checked on the full bitmap in global memory, r scattered L2 reads each, and with 4 or
@@ -9,8 +10,10 @@
 //                       evaluates that row's bit for every coordinate of its range: of each 1024 coordinates a
 //                       warp takes, lane l walks the 32 consecutive ones of result word l (one add + conditional
 //                       subtract per hash, one shared-memory load, two funnel shifts to append the bit), then
-//                       the warp stores its 32 words with one coalesced 128-byte store.
-//   k_rowbits_combine   reads the r result words of 32 coordinates (coalesced), counts per coordinate how many rows
+//                       the warp stores its 32 words with one coalesced 128-byte store.  A row longer than shared
+//                       memory is cut into slices, one block each: a block sets the bits of the coordinates whose
+//                       bucket lies in its slice, into a result row of its own.
+//   k_rowbits_combine   reads the r result words of 32 coordinates (coalesced; ORs a row's slices), counts per coordinate how many rows
 //                       have their bit set with a bit-sliced adder, and for the few coordinates with at least (r+1)/2
 //                       set bits computes the exact estimate from the table (the warp's passing coordinates are
 //                       compacted in shared memory first, so that every lane has one) and appends it to the
@@ -32,23 +35,28 @@
 namespace ssgd {
 
 constexpr int RB_MAX_THREADS = 1024;
+constexpr int RB_MAX_SLICES = 4;       // a row in more slices costs more hash evaluations than the folded filter saves
 // The row-by-row filter is used if at most this share of the coordinates is expected to pass it (binomial tail of
 // the bitmap's density): beyond, exact estimates for nearly everyone cost more than the early-exit table kernel.
 constexpr float ROWBITS_MAX_PASS = 0.7f;
 
 struct RowBitsArgs {
     FilterArgs F;
-    uint32_t* rowbits;        // [r][words_per_row]: bit i of row j = "row j's bucket of coordinate i is above the threshold"
+    uint32_t* rowbits;        // [slices][r][words_per_row]: bit i of row j = "row j's bucket of coordinate i lies in
+                              // this slice and is above the threshold"
     int64_t words_per_row;    // ceil(d / 32)
-    int32_t ranges;           // blocks per row: block b works on row b % r, coordinate range b / r
+    int32_t ranges;           // blocks per row and slice: block b works on row b % r, slice (b / r) % slices,
+                              // coordinate range b / (r * slices)
+    int32_t slices;           // pieces a bitmap row is cut into (1: the row fits shared memory)
+    int32_t slice_words;      // words per slice (a multiple of 4; the last slice may be shorter)
 };
 
 #ifdef __CUDACC__
 
-template <bool POW2>
+template <bool POW2, bool SLICED>
 __global__ void __launch_bounds__(RB_MAX_THREADS)
 k_row_bits(const RowBitsArgs B) {
-    extern __shared__ __align__(16) uint32_t rb_bm[];      // row j of the full bitmap
+    extern __shared__ __align__(16) uint32_t rb_bm[];      // row j of the full bitmap (SLICED: words [lo, lo + nw) of it)
     const SparseArgs& A = B.F.A;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads >> 5;
@@ -56,12 +64,18 @@ k_row_bits(const RowBitsArgs B) {
     pdl_wait();
     if (__ldcg(&A.sp.state->use_table) != 0u) return;      // too dense to prune: the table kernel behind runs
     const int j = (int)(blockIdx.x % (unsigned)B.F.r);
-    const int64_t rho = blockIdx.x / (unsigned)B.F.r;
+    const int sl = SLICED ? (int)((blockIdx.x / (unsigned)B.F.r) % (unsigned)B.slices) : 0;
+    const int64_t rho = blockIdx.x / ((unsigned)B.F.r * (unsigned)(SLICED ? B.slices : 1));
+    const uint32_t lo = (uint32_t)sl * (uint32_t)B.slice_words;
+    const uint32_t nw = SLICED ? ((uint32_t)B.F.stride_full - lo < (uint32_t)B.slice_words ? (uint32_t)B.F.stride_full - lo
+                                                                                          : (uint32_t)B.slice_words)
+                               : (uint32_t)B.F.stride_full;
     {
-        const uint4* src = reinterpret_cast<const uint4*>(B.F.bm_full + (int64_t)j * B.F.stride_full);
+        const uint4* src = reinterpret_cast<const uint4*>(B.F.bm_full + (int64_t)j * B.F.stride_full + lo);
         const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rb_bm);
-        for (int w = tid; w < B.F.stride_full / 4; w += nthreads)
+        for (int w = tid; w < (int)(nw / 4); w += nthreads)
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + (uint32_t)w * 16u), "l"(src + w) : "memory");
+        if (SLICED && tid == 0) rb_bm[nw] = 0u;            // what buckets outside the slice read
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
@@ -81,13 +95,19 @@ k_row_bits(const RowBitsArgs B) {
     uint32_t y = lin_hash(hr.a, hr.b, s);
     const uint32_t skip = mod_p31((uint64_t)hr.a * 992ull);   // from s + 32 to the lane's word of the next chunk
     const uint32_t d32 = (uint32_t)A.d;
-    uint32_t* out = B.rowbits + (int64_t)j * B.words_per_row;
+    uint32_t* out = B.rowbits + ((int64_t)sl * B.F.r + j) * B.words_per_row;
     for (int64_t chunk = w_lo; chunk < w_hi; ++chunk) {
         uint32_t word = 0;
 #pragma unroll
         for (int t = 0; t < 32; ++t) {
             const uint32_t b = bucket_of<POW2>(y, A.bk);
-            const uint32_t bits = __funnelshift_r(rb_bm[b >> 5], 0u, b);     // bucket b's bit lowest (shift taken mod 32)
+            uint32_t bits;                                                   // bucket b's bit lowest (shift taken mod 32)
+            if (SLICED) {
+                const uint32_t wi = (b >> 5) - lo;                           // wraps to a large value below the slice
+                bits = __funnelshift_r(rb_bm[wi < nw ? wi : nw], 0u, b);     // word nw is zero: no branch, a broadcast read
+            } else {
+                bits = __funnelshift_r(rb_bm[b >> 5], 0u, b);
+            }
             word = __funnelshift_r(word, bits, 1);                           // word >> 1 | lowest bit of `bits` << 31
             y = next_hash(y, hr.a);
         }
@@ -128,7 +148,13 @@ k_rowbits_combine(const RowBitsArgs B) {
         uint32_t c0 = 0, c1 = 0, c2 = 0, c3 = 0;
         uint32_t rows[R];
 #pragma unroll
-        for (int j = 0; j < R; ++j) rows[j] = w < B.words_per_row ? __ldcs(B.rowbits + (int64_t)j * B.words_per_row + w) : 0u;
+        for (int j = 0; j < R; ++j) rows[j] = 0u;
+        if (w < B.words_per_row) {
+            for (int sl = 0; sl < B.slices; ++sl) {
+#pragma unroll
+                for (int j = 0; j < R; ++j) rows[j] |= __ldcs(B.rowbits + ((int64_t)sl * R + j) * B.words_per_row + w);
+            }
+        }
 #pragma unroll
         for (int j = 0; j < R; ++j) {
             uint32_t carry = rows[j], t;

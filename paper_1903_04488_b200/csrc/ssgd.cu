@@ -123,10 +123,12 @@ void layout(ssgd_ctx* x, int64_t ncand_max) {
     x->off_pending = o; o += x->map_bytes;
     x->off_bm_full = o; o += up((size_t)x->r * sf * 4);
     x->off_bm_fold = o; o += up((size_t)x->r * x->bm_stride_fold * 4);
-    // a bitmap that needs folding but whose single row fits shared memory is used unfolded, row by row
-    x->rowbits = x->bm_fold != 0 && sf <= FILTER_MAX_WORDS;
+    // a bitmap that needs folding but whose single row fits shared memory in a few slices is used unfolded, row by row
+    x->rb_slices = (int)((sf + FILTER_MAX_WORDS - 1) / FILTER_MAX_WORDS);
+    x->rb_slice_words = x->rb_slices > 0 ? (int)(((sf + x->rb_slices - 1) / x->rb_slices + 3) / 4 * 4) : 0;
+    x->rowbits = x->bm_fold != 0 && x->rb_slices >= 1 && x->rb_slices <= RB_MAX_SLICES;
     x->off_rowbits = o;
-    if (x->rowbits) o += up((size_t)x->r * (size_t)((x->d + 31) / 32) * 4);
+    if (x->rowbits) o += up((size_t)x->rb_slices * x->r * (size_t)((x->d + 31) / 32) * 4);
     x->total_bytes = o;
 }
 

@@ -423,14 +423,17 @@ def test_pruned_path_is_taken_and_prunes(cuda_device, prune):
 FOLD_CASES = [
     wl.C3.scaled(d=600_011, W=3, r=5, c=524_288, ncand=5000, k=2000),       # 5 x 2^19 bits: two buckets per bit
     wl.P1.scaled(d=400_003, W=2, r=15, c=180_000, ncand=8000, k=500),       # the paper's 15 x 180,000: two per bit
-    wl.C4.scaled(d=500_009, W=2, r=5, c=6_000_001, ncand=4000, k=1000),     # 32 buckets per bit, c not a power of two
+    wl.C4.scaled(d=500_009, W=2, r=5, c=6_000_001, ncand=4000, k=1000),     # each row in 4 slices, c not a power of two
+    wl.C4.scaled(d=500_009, W=2, r=5, c=4_194_304, ncand=4000, k=1000),     # C4's own table: each row in 3 slices
+    wl.C4.scaled(d=500_009, W=2, r=5, c=7_000_003, ncand=4000, k=1000),     # folded: 32 buckets per bit
 ]
 
 
 @pytest.mark.parametrize("cfg", FOLD_CASES, ids=lambda c: f"{c.name}-r{c.r}-c{c.c}")
 def test_bucket_bitmap_folded_into_shared_memory(cuda_device, cfg):
-    """Sketches whose one-bit-per-bucket filter exceeds an SM's shared memory: neighbouring buckets share a bit
-    there and the full bitmap is consulted in global memory before the table is read."""
+    """Sketches whose one-bit-per-bucket filter exceeds an SM's shared memory.  Up to four times a row's worth of
+    shared memory per row: the bitmap is evaluated row by row (a row in slices).  Beyond: neighbouring buckets
+    share a bit and the full bitmap is consulted in global memory before the table is read."""
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_prune_mode(S.PRUNE_ON)
     u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
@@ -443,10 +446,12 @@ def test_bucket_bitmap_folded_into_shared_memory(cuda_device, cfg):
         assert not declined and 0 < ones < cfg.r * cfg.c // 8
 
 
-def test_dense_folded_bitmap_hands_over_to_the_table_kernel(cuda_device):
-    """A folded bitmap that would rule out too few coordinates (here: all estimates zero, threshold zero, every
-    bit set) makes the filter kernel return at once; the table kernel enqueued behind it does the first pass."""
-    cfg = wl.C3.scaled(d=300_007, W=2, r=5, c=524_288, ncand=1000, k=500)
+@pytest.mark.parametrize("c,ones_per_row", [(524_288, 524_288), (8_388_608, 8_388_608 // 32)], ids=["rows", "folded"])
+def test_dense_bitmap_hands_over_to_the_table_kernel(cuda_device, c, ones_per_row):
+    """A bitmap that would rule out too few coordinates (here: all estimates zero, threshold zero, every bit set)
+    makes the filter kernels return at once; the table kernel enqueued behind them does the first pass.  Both
+    forms of the filter: row by row (the unfolded bitmap's density decides) and folded (32 buckets per bit)."""
+    cfg = wl.C3.scaled(d=300_007, W=2, r=5, c=c, ncand=1000, k=500)
     eng, orc, u, v = make(cfg, cuda_device)
     eng.set_prune_mode(S.PRUNE_ON)
     g = torch.zeros((cfg.W, cfg.ld), device=cuda_device)
@@ -454,7 +459,7 @@ def test_dense_folded_bitmap_hands_over_to_the_table_kernel(cuda_device):
     idx, val = check_step(orc, eng, g, cfg.rho, cfg.ncand, u_o, v_o)
     fell_back, survivors, bin_lo = eng.step_used_fallback()
     declined, ones = eng.step_first_pass()
-    assert declined and ones == cfg.r * cfg.c              # one row fits shared memory: the unfolded bitmap is counted
+    assert declined and ones == cfg.r * ones_per_row
     assert not fell_back and survivors == cfg.d and bin_lo == 0
     assert idx.tolist() == list(range(cfg.k))
     st = wl.Structure(cfg, cuda_device)                    # a real gradient next: the filter takes over again
