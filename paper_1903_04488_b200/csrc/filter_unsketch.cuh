@@ -293,9 +293,11 @@ k_unsketch_filter(const FilterArgs F) {
         if (FOLD) recheck(c, rows, got); else exact(c, got);
     };
 
-    // this thread's run of consecutive coordinates
+    // this thread's run of consecutive coordinates, 32 at a time: row j's bits of the 32 are shifted into one word
+    // (two funnel shifts per lookup), the rows are counted with a bit-sliced adder, and only the coordinates with
+    // at least NEED set bits are looked at one by one
     const uint32_t total_threads = gridDim.x * FILTER_THREADS;
-    constexpr int NC = FILTER_NC;
+    constexpr uint32_t NC = FILTER_NC;
     const uint32_t per = (uint32_t)((A.d + total_threads - 1) / total_threads + NC - 1) / NC * NC;
     const uint32_t gtid = blockIdx.x * FILTER_THREADS + threadIdx.x;
     const uint64_t begin64 = (uint64_t)gtid * per;
@@ -305,25 +307,57 @@ k_unsketch_filter(const FilterArgs F) {
     const uint32_t* row_base[R];
 #pragma unroll
     for (int j = 0; j < R; ++j) { y[j] = lin_hash(A.hp.row[j].a, A.hp.row[j].b, i_begin); row_base[j] = bm + j * stride_s; }
-    for (uint32_t t = 0; t < per; t += NC) {             // warp-uniform trip count
-        uint32_t rows[NC];                               // bit j: row j's bit is set
+    for (uint32_t t0 = 0; t0 < per; t0 += 32u) {         // warp-uniform trip counts, here and below
+        const uint32_t n_this = per - t0 < 32u ? per - t0 : 32u;     // a multiple of NC
+        uint32_t w[R];                                   // bit e of w[j]: row j's bit of coordinate i_begin + t0 + e
 #pragma unroll
-        for (int e = 0; e < NC; ++e) rows[e] = 0;
+        for (int j = 0; j < R; ++j) w[j] = 0u;
+        for (uint32_t t = 0; t < n_this; t += NC) {
 #pragma unroll
-        for (int e = 0; e < NC; ++e) {
+            for (uint32_t e = 0; e < NC; ++e) {
 #pragma unroll
-            for (int j = 0; j < R; ++j) {
-                const uint32_t b = bucket_of<POW2>(y[j], A.bk) >> fold;
-                const uint32_t bit = __funnelshift_r(row_base[j][b >> 5], 0u, b) & 1u;   // shift amount taken mod 32
-                if (FOLD) rows[e] |= bit << j; else rows[e] += bit;
-                y[j] = next_hash(y[j], A.hp.row[j].a);
+                for (int j = 0; j < R; ++j) {
+                    const uint32_t b = bucket_of<POW2>(y[j], A.bk) >> fold;
+                    const uint32_t bits = __funnelshift_r(row_base[j][b >> 5], 0u, b);   // shift amount taken mod 32
+                    w[j] = __funnelshift_r(w[j], bits, 1);                               // lowest bit of `bits` enters at the top
+                    y[j] = next_hash(y[j], A.hp.row[j].a);
+                }
             }
         }
+        if (n_this < 32u) {
 #pragma unroll
-        for (int e = 0; e < NC; ++e) {
-            const uint32_t i = i_begin + t + e;
-            const int cnt = FOLD ? __popc(rows[e]) : (int)rows[e];
-            q2.push(i < i_end && cnt >= NEED, i, rows[e], lane);
+            for (int j = 0; j < R; ++j) w[j] >>= 32u - n_this;
+        }
+        // bit-sliced count (4 planes: r <= 15) of the rows whose bit is set; pass = count >= NEED
+        uint32_t c0 = 0, c1 = 0, c2 = 0, c3 = 0;
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            uint32_t carry = w[j], x;
+            x = c0 & carry; c0 ^= carry; carry = x;
+            x = c1 & carry; c1 ^= carry; carry = x;
+            x = c2 & carry; c2 ^= carry; carry = x;
+            c3 ^= carry;
+        }
+        const uint32_t plane[4] = {c0, c1, c2, c3};
+        uint32_t gt = 0u, eq = 0xFFFFFFFFu;
+#pragma unroll
+        for (int p = 3; p >= 0; --p) {
+            if ((NEED >> p) & 1) { eq &= plane[p]; }
+            else { gt |= eq & plane[p]; eq &= ~plane[p]; }
+        }
+        const uint32_t first = i_begin + t0;
+        const uint32_t nvalid = i_end > first ? (i_end - first < 32u ? i_end - first : 32u) : 0u;
+        uint32_t pass = (gt | eq) & (nvalid >= 32u ? 0xFFFFFFFFu : (1u << nvalid) - 1u);
+        while (__any_sync(0xFFFFFFFFu, pass != 0u)) {
+            const bool have = pass != 0u;
+            const int bit = have ? __ffs(pass) - 1 : 0;
+            pass &= pass - 1u;                           // (0 stays 0)
+            uint32_t rows = 0u;                          // folded bitmaps: which rows had their folded bit set
+            if (FOLD) {
+#pragma unroll
+                for (int j = 0; j < R; ++j) rows |= ((w[j] >> bit) & 1u) << j;
+            }
+            q2.push(have, first + (uint32_t)bit, rows, lane);
             if (q2.count >= 32) drain2();
         }
     }
