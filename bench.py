@@ -458,7 +458,7 @@ def measure_config(cfg, dev, args, gpu_index, reps):
         k1 = 20.0 * cfg.W * cfg.d / (stage["accumulate_insert_ms"] * 1e-3) / 1e9
         rec["roofline"] = {"bound": "hbm", "kernel": dominant_kernel(cfg), "achieved": k1, "peak": peak, "unit": "GB/s",
                            "frac": k1 / peak, "peak_source": f"of {peak_kind}"}
-        # the operation-rate bound of the accumulate+insert kernel: a reduction into the L2-resident
+        # the operation-rate bound of the accumulate+insert kernel (measured across shapes): a reduction into the L2-resident
         # table costs the L2 about what a 32-byte sector of the stream costs; 2.6e11 such operations per second
         ops = 20.0 * cfg.W * cfg.d / 32.0 + float(cfg.d) * cfg.r
         t_ops = ops / 2.6e11 * 1e3
