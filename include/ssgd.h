@@ -69,12 +69,13 @@ extern "C" {
 /* How ssgd_step evaluates Algorithm 3 line 9 (ssgd_set_prune_mode).  A median of r values reaches a magnitude
  * only if (r+1)/2 of them do, so with a threshold taken from a sample of the estimates most coordinates can be
  * ruled out from "is this bucket's magnitude above the threshold" alone.  ON: that test is precomputed as one bit
- * per bucket and kept in shared memory (if r*c bits, OR-folded up to 32 buckets per bit, fit; otherwise as
- * EARLY_EXIT).  EARLY_EXIT: the test is applied to the table values themselves and a coordinate stops reading
+ * per bucket and kept in shared memory: all r*c bits at once if they fit; else one row (or one of up to four
+ * slices of a row) per thread block, the r bits of every coordinate being combined afterwards; else OR-folded up
+ * to 32 buckets per bit; otherwise as EARLY_EXIT.  EARLY_EXIT: the test is applied to the table values themselves and a coordinate stops reading
  * rows once it cannot pass.  OFF: every coordinate reads all r rows.  The candidates are identical in all modes.
  * AUTO is ON when d >= 2^21, ncand <= d/8 (below that the fixed costs outweigh the saving) and either the bitmap
- * fits unfolded or 5 <= r <= 9; else OFF.  Behind a folded bitmap ON measures the bitmap's density each step and
- * runs the EARLY_EXIT kernel instead when the folded bits would rule out too few coordinates. */
+ * fits as a whole or 5 <= r <= 9; else OFF.  Unless the bitmap fits as a whole, ON measures its density each step
+ * and runs the EARLY_EXIT kernel instead when its bits would rule out too few coordinates. */
 #define SSGD_PRUNE_AUTO 0
 #define SSGD_PRUNE_OFF  1
 #define SSGD_PRUNE_ON   2
@@ -145,8 +146,9 @@ int ssgd_set_table_persistence(ssgd_ctx* ctx, int32_t enable);
 /* Diagnostics of the last ssgd_step's pruned path (waits for the stream), five values: out[0] != 0 if the
  * sampled threshold kept fewer than ncand coordinates and the pass was redone without pruning, out[1] = number
  * of coordinates on the survivor list, out[2] = the prune threshold as a histogram-bin index (0: nothing
- * pruned), out[3] = 1 if a folded bucket bitmap was too dense and the first pass read the table instead,
- * out[4] = set bits of the folded bitmap (0 if the bitmap is not folded). */
+ * pruned), out[3] = 1 if the bucket bitmap was too dense and the first pass read the table instead,
+ * out[4] = set bits of the bitmap that was measured (the unfolded one if it is used row by row, else the folded
+ * one; 0 if the bitmap fits shared memory as a whole and is not measured). */
 int ssgd_step_used_fallback(ssgd_ctx* ctx, void* stream, int32_t* out5);
 /* Diagnostics of the last ssgd_step that took the FUSED tail (waits for the stream): nanoseconds since the tail
  * kernel's first thread block started, at 12 points -- [0] start, [1] table rows copied to shared memory (if any),

@@ -40,8 +40,9 @@ struct SparseState {                              // zeroed before the step
     uint32_t thr_key;      // T: the exact 31-bit threshold key
     uint32_t quota_eq;     // Q: how many items with key == T are selected (smallest coordinates first)
     uint32_t ticket[6];    // finished-block counters: sample, first pass, unpruned rerun, list histogram, map count, fold
-    uint32_t fold_ones;    // set bits of the folded bucket bitmap (filter_unsketch.cuh)
-    uint32_t use_table;    // 1: the folded bitmap is too dense to prune; the first pass reads the table instead
+    uint32_t fold_ones;    // set bits of the bucket bitmap whose density is measured: the folded one, or the unfolded one
+                           // when it is used row by row (filter_unsketch.cuh, rowbits_unsketch.cuh)
+    uint32_t use_table;    // 1: that bitmap is too dense to prune; the first pass reads the table instead
     uint32_t pad[1];
 };
 

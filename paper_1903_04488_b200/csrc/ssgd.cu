@@ -9,6 +9,8 @@
 //   accum_tma.cuh       k_accum_insert_tma: lines 5-7 as a bulk-copy (TMA) + mbarrier pipeline
 //   filter_unsketch.cuh k_bitmap_build, k_bitmap_fold, k_unsketch_filter: line 9 decided per coordinate on a
 //                       one-bit-per-bucket copy of the table in shared memory
+//   rowbits_unsketch.cuh k_row_bits, k_rowbits_combine: the same decision when that copy fits shared memory only
+//                       one row (or a slice of a row) at a time
 //   sparse_select.cuh   k_unsketch_sample, k_unsketch_pruned: the sampled threshold; line 9 with early exit on
 //                       the table itself
 //   list_select.cuh     k_list_hist, k_list_mark, k_map_emit: exact top-ncand of the survivor list

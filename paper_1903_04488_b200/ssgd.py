@@ -198,7 +198,7 @@ class Ssgd:
         return bool(out[0]), int(out[1]), int(out[2])
 
     def step_first_pass(self):
-        """(folded bitmap declined and the table was read instead?, set bits of the folded bitmap) of the last step."""
+        """(bucket bitmap too dense and the table was read instead?, set bits of the measured bitmap) of the last step."""
         out = (_i32 * 5)()
         self._chk(self._lib.ssgd_step_used_fallback(self._h, _stream(), out), "ssgd_step_used_fallback")
         return bool(out[3]), int(out[4])
