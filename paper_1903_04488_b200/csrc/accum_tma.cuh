@@ -10,6 +10,8 @@
 // After the last worker each consumer thread hashes its four coordinates and issues the r reductions
 // per coordinate into the L2-resident merged table (sum_w S(v_w) = S(sum_w v_w), Section 3).
 // The producer runs ahead into the next tile while the consumers issue a tile's reductions.
+// Tiles are dealt out round robin, so that at any moment the CTAs read neighbouring tiles: one contiguous range
+// per CTA (no partial last round) measured slower, 9.45 against 9.38 ms at W = 256 and 4.81 against 4.71 at W = 128.
 //
 // Every mbarrier wait is bounded: after `wait_ns` nanoseconds (an argument; ssgd_set_wait_limit_ns) the waiter
 // records ERR_TIMEOUT in the error word, raises the CTA's abort flag and leaves; whatever happened, the producer
