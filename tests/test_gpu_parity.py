@@ -446,6 +446,20 @@ def test_bucket_bitmap_folded_into_shared_memory(cuda_device, cfg):
         assert not declined and 0 < ones < cfg.r * cfg.c // 8
 
 
+@pytest.mark.parametrize("d", [1, 31, 33, 1023, 1025, 40_001])
+@pytest.mark.parametrize("c", [1_048_576, 2_000_003, 4_194_304], ids=["row", "2slices", "3slices"])
+def test_row_bitmap_ragged_ends(cuda_device, d, c):
+    """The row-by-row bitmap on coordinate counts around its units (a 32-coordinate result word, a warp's 1024
+    coordinates): far fewer coordinates than blocks, partial last words, pruning forced on."""
+    cfg = wl.C3.scaled(d=d, W=2, r=5, c=c, ncand=max(1, d // 7), k=max(1, d // 20))
+    eng, orc, u, v = make(cfg, cuda_device)
+    eng.set_prune_mode(S.PRUNE_ON)
+    u_o, v_o = u.cpu().numpy(), v.cpu().numpy()
+    st = wl.Structure(cfg, cuda_device)
+    for t in range(2):
+        check_step(orc, eng, wl.gradients(st, t), cfg.rho, cfg.ncand, u_o, v_o)
+
+
 @pytest.mark.parametrize("c,ones_per_row", [(524_288, 524_288), (8_388_608, 8_388_608 // 32)], ids=["rows", "folded"])
 def test_dense_bitmap_hands_over_to_the_table_kernel(cuda_device, c, ones_per_row):
     """A bitmap that would rule out too few coordinates (here: all estimates zero, threshold zero, every bit set)
