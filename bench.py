@@ -469,6 +469,7 @@ def measure_config(cfg, dev, args, gpu_index, reps):
         rec["ms_per_step_warm_l2"] = b.warm_sequence(20)
     if b.mode == "faithful":
         rec["sketch16"] = time_sketch16(b)
+        rec["heavymix"] = time_heavymix(b)
     del b
     torch.cuda.empty_cache()
     return rec
@@ -501,6 +502,27 @@ def time_sketch16(b):
     out["merge16_bytes"] = 2 * rc * cfg.W + 4 * rc
     out["note"] = "working set (W tables) may fit in L2: these are warm figures"
     return out
+
+
+def time_heavymix(b):
+    """Algorithm 1 (HEAVYMIX) on the merged table the faithful pipeline left behind: the other way from a sketch to k
+    coordinates (norm estimate, heavy set, seeded random fill, exact values of the chosen ones)."""
+    torch, cfg = b.torch, b.cfg
+    oi = torch.empty(cfg.k, dtype=torch.int32, device=b.dev)
+    ov = torch.empty(cfg.k, dtype=torch.float32, device=b.dev)
+    l2 = torch.empty(1, dtype=torch.float64, device=b.dev)
+    nh = torch.empty(1, dtype=torch.int32, device=b.dev)
+    for _ in range(3):
+        b.eng.heavymix(b.merged, 12345, oi, ov, l2, nh)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    n = 10
+    for _ in range(n):
+        b.eng.heavymix(b.merged, 12345, oi, ov, l2, nh)
+    e1.record()
+    torch.cuda.synchronize()
+    return {"ms": e0.elapsed_time(e1) / n, "heavy": int(nh.item()), "k": cfg.k,
+            "note": "one call of ssgd_heavymix on the merged table (L2-warm), d*r table reads + selection over d keys"}
 
 
 def run_ours(args):
