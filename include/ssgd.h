@@ -138,6 +138,14 @@ int ssgd_flush(ssgd_ctx* ctx, void* stream);
  * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
  * which leaves tables up to that size untouched). */
 int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
+/* Cache operator of the plain-load accumulate+insert kernel's reads of g, u, v (ssgd_step, W < 64).  AUTO:
+ * evict-first (ld.global.cs) when the sketch table has 16 MiB or more and W >= 8 (the stream then leaves the table's lines
+ * in L2 alone), else L2_ONLY (ld.global.cg: not kept in L1, normal priority in L2).  The result of a step does
+ * not depend on it. */
+#define SSGD_STREAM_AUTO        0
+#define SSGD_STREAM_EVICT_FIRST 1
+#define SSGD_STREAM_L2_ONLY     2
+int ssgd_set_stream_loads(ssgd_ctx* ctx, int32_t mode);
 /* Opt-in: reserve part of L2 for the sketch table while the accumulate+insert kernel streams g, u, v past it
  * (cudaLimitPersistingL2CacheSize of this process's CUDA context is raised to the table size, capped by the
  * device; the launches then carry an access-policy window over the table).  Off by default because the limit

@@ -12,7 +12,9 @@
 // The producer runs ahead into the next tile while the consumers issue a tile's reductions.
 // Tiles are dealt out round robin, so that at any moment the CTAs read neighbouring tiles: one contiguous range
 // per CTA (no partial last round) measured slower, 9.45 against 9.38 ms at W = 256 and 4.81 against 4.71 at W = 128.
-// The results leave through 128-bit streaming stores of the consumer threads: written into the slot in place and
+// Cache hints, measured at W = 256 / 128 (ms per step): bulk loads with an L2 evict-first policy and streaming
+// (.cs) stores 9.53 / 4.86; loads without a hint 9.47 / 4.81; loads without a hint and plain stores 9.43 / 4.80 (kept).
+// The results leave through 128-bit stores of the consumer threads: written into the slot in place and
 // sent by bulk stores (16 KB pieces, issued by the producer before it refills the slot) measured 9.40 ms with 3
 // slots and 9.46 ms with 4 against 9.37 ms at W = 256.
 //
@@ -39,6 +41,9 @@ struct AccumArgs {
     HashParams hp; Bucketizer bk;
     // plain-load merged mode only: insert rows [0, rows_here) in this kernel (k_insert_rows does the others)
     int32_t rows_here;
+    // plain-load kernel: 1 = read g, u, v with the evict-first operator (.cs), 0 = cached in L2 only (.cg); see
+    // STREAM_CS_MIN_TABLE_BYTES
+    int32_t loads_evict_first;
     // merged modes: if not NULL, the per-coordinate sum over workers of the new v (fp64 accumulation in worker
     // order, rounded once) is also written to xsum[d]: the second round's exact sums, and k_insert_rows' input
     float* xsum;
@@ -125,16 +130,11 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         }
     }
 }
-__device__ __forceinline__ uint64_t policy_evict_first() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
 // global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar, uint64_t pol) {
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol) : "memory");
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 template <int R, bool POW2>
@@ -158,7 +158,6 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
     if (warp == KT_CONSUMER_WARPS) {
         // ---------------- producer warp: one thread feeds the ring ----------------
         if (lane == 0) {
-            const uint64_t pol = policy_evict_first();
             uint32_t n = 0;
             bool ok = true;
             const bool withheld = A.withhold && (int)blockIdx.x == A.withhold - 1;
@@ -169,9 +168,9 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
                     const int s = n % KT_STAGES;
                     if (n >= KT_STAGES && !mbar_wait(&S.empty[s], ((n / KT_STAGES) - 1) & 1, &S.abort, A.wait_ns)) { ok = false; break; }
                     mbar_expect_tx(&S.full[s], 3 * bytes);
-                    bulk_load(S.slot[s].g, A.g + (int64_t)w * A.ld_g + i0, bytes, &S.full[s], pol);
-                    bulk_load(S.slot[s].u, A.u + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
-                    bulk_load(S.slot[s].v, A.v + (int64_t)w * A.ld + i0, bytes, &S.full[s], pol);
+                    bulk_load(S.slot[s].g, A.g + (int64_t)w * A.ld_g + i0, bytes, &S.full[s]);
+                    bulk_load(S.slot[s].u, A.u + (int64_t)w * A.ld + i0, bytes, &S.full[s]);
+                    bulk_load(S.slot[s].v, A.v + (int64_t)w * A.ld + i0, bytes, &S.full[s]);
                 }
             }
             if (!ok) {                                     // give up: report and tell the consumers
@@ -221,8 +220,8 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
                     un.y = __fmaf_rn(A.rho, u4.y, g4.y); vn.y = __fadd_rn(v4.y, un.y);
                     un.z = __fmaf_rn(A.rho, u4.z, g4.z); vn.z = __fadd_rn(v4.z, un.z);
                     un.w = __fmaf_rn(A.rho, u4.w, g4.w); vn.w = __fadd_rn(v4.w, un.w);
-                    __stcs(reinterpret_cast<float4*>(A.u + (int64_t)w * A.ld + i0), un);
-                    __stcs(reinterpret_cast<float4*>(A.v + (int64_t)w * A.ld + i0), vn);
+                    *reinterpret_cast<float4*>(A.u + (int64_t)w * A.ld + i0) = un;
+                    *reinterpret_cast<float4*>(A.v + (int64_t)w * A.ld + i0) = vn;
                     xs[v][0] = __dadd_rn(xs[v][0], (double)vn.x); xs[v][1] = __dadd_rn(xs[v][1], (double)vn.y);
                     xs[v][2] = __dadd_rn(xs[v][2], (double)vn.z); xs[v][3] = __dadd_rn(xs[v][3], (double)vn.w);
                 }

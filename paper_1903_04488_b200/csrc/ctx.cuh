@@ -58,6 +58,7 @@ struct ssgd_ctx {
     int32_t prune_mode;
     size_t persist_bytes;   // > 0: launches that touch the table carry an L2 access-policy window of this size
     size_t split_bytes;     // > 0: ssgd_step inserts at most this many bytes of table rows per kernel
+    int stream_loads;       // SSGD_STREAM_*: cache operator of the plain-load kernel's reads of g, u, v
     size_t off_xsum;        // per-coordinate sums over the workers of the new v, written by ssgd_step's accumulate kernel
     size_t off_est, off_chunk_c, off_chunk_f, off_cand, off_xs, off_oidx, off_oval, total_bytes;
     int64_t nchunk_c, nchunk_f;

@@ -375,7 +375,7 @@ int ssgd_create(ssgd_ctx** out, int64_t d, int32_t r, int64_t c, int64_t k, int3
     x->u = x->v = nullptr; x->ws = nullptr; x->ld = 0; x->ws_bytes = 0; x->ncand_max = 0;
     x->device = -1; x->sm_count = 0; x->max_smem_optin = 0; x->launches = 0; x->kt_blocks_per_sm = 0;
     x->small_grid = 0; x->small_refused = false; x->wait_ns = 2000000000ull; x->withhold = 0;
-    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->rowbits = false; x->rowbits_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT;
+    x->timing = false; x->ev = nullptr; x->ev_steps = 0; x->prune_mode = SSGD_PRUNE_AUTO; x->list_cap = 0; x->sample_rank = 0; x->filter_ready = false; x->rowbits = false; x->rowbits_ready = false; x->bm_fold = -1; x->zero_mode = SSGD_ZERO_DEFERRED; x->pending_dirty = false; x->sched_mode = SSGD_SCHED_AUTO; x->persist_bytes = 0; x->split_bytes = SPLIT_BYTES_DEFAULT; x->stream_loads = SSGD_STREAM_AUTO;
     *out = x;
     return SSGD_OK;
 }
@@ -433,6 +433,12 @@ int ssgd_set_table_persistence(ssgd_ctx* x, int32_t enable) {
 int ssgd_set_prune_sample_rank(ssgd_ctx* x, int64_t rank) {
     if (!x || rank < 0 || rank > 0x7FFFFFFF) return SSGD_EINVAL;
     x->sample_rank = (uint32_t)rank;
+    return SSGD_OK;
+}
+
+int ssgd_set_stream_loads(ssgd_ctx* x, int32_t mode) {
+    if (!x || mode < SSGD_STREAM_AUTO || mode > SSGD_STREAM_L2_ONLY) return SSGD_EINVAL;
+    x->stream_loads = mode;
     return SSGD_OK;
 }
 
@@ -519,6 +525,7 @@ int ssgd_sketch_accumulate(ssgd_ctx* x, const float* g, int64_t ld_g, float rho,
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = tables; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr; A.pending = nullptr;
+    A.loads_evict_first = 1;
     A.wait_ns = x->wait_ns; A.withhold = 0;
     const size_t all_tables = (size_t)x->W * x->r * x->c * 4;
     const bool worker_major = x->sched_mode == SSGD_SCHED_WORKER_MAJOR ||
@@ -618,6 +625,8 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
+    A.loads_evict_first = x->stream_loads == SSGD_STREAM_AUTO ? ((size_t)x->r * (size_t)x->c * 4 >= STREAM_CS_MIN_TABLE_BYTES && x->W >= 8 ? 1 : 0)
+                                                              : (x->stream_loads == SSGD_STREAM_EVICT_FIRST ? 1 : 0);
     A.pending = pending_map(x);      // the previous step's deferred zero-out, applied while u and v stream past
     A.wait_ns = x->wait_ns; A.withhold = x->withhold;
     // a table that cannot stay in L2 next to the stream is inserted a slice of rows at a time

@@ -18,6 +18,12 @@ namespace ssgd {
 // (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each): 1 row per kernel 6.43 ms, 2 rows 6.25, 3 rows 6.60,
 // 4 rows 6.89, all 5 rows in one kernel 7.80.
 constexpr size_t SPLIT_BYTES_DEFAULT = (size_t)40 << 20;
+// The plain-load kernel reads g, u, v with the evict-first operator (ld.global.cs) when the table it scatters into
+// is at least this large and W >= 8 (the stream then leaves the table's lines alone), else cached in L2 with the normal
+// priority (ld.global.cg).  Measured on B200, whole step in ms with .cs / .cg: 5 MB table W = 32 1.350 / 1.293,
+// W = 16 0.768 / 0.753, W = 8 0.574 / 0.571; 3.6 MB (W = 4, d = 7.3e7) 2.720 / 2.707; 20 MB W = 32 2.264 / 2.315,
+// (W = 4, d = 9e7) 3.459 / 3.444; 80 MB in row slices 7.238 / 7.590.
+constexpr size_t STREAM_CS_MIN_TABLE_BYTES = (size_t)16 << 20;
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
@@ -74,13 +80,25 @@ k_accum_insert(const AccumArgs A) {
             constexpr int U = MODE == INS_PER_WORKER ? K1_UNROLL_PW : UM;
             for (int w0 = 0; w0 < A.W; w0 += U) {
                 float4 gg[U], uu[U], vv[U];
+                if (A.loads_evict_first) {              // the same for the whole grid
 #pragma unroll
-                for (int s = 0; s < U; ++s) {
-                    if (w0 + s < A.W) {
-                        const int64_t w = w0 + s;
-                        gg[s] = __ldcs(reinterpret_cast<const float4*>(A.g + w * A.ld_g + i0));
-                        uu[s] = __ldcs(reinterpret_cast<const float4*>(A.u + w * A.ld + i0));
-                        vv[s] = __ldcs(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
+                    for (int s = 0; s < U; ++s) {
+                        if (w0 + s < A.W) {
+                            const int64_t w = w0 + s;
+                            gg[s] = __ldcs(reinterpret_cast<const float4*>(A.g + w * A.ld_g + i0));
+                            uu[s] = __ldcs(reinterpret_cast<const float4*>(A.u + w * A.ld + i0));
+                            vv[s] = __ldcs(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int s = 0; s < U; ++s) {
+                        if (w0 + s < A.W) {
+                            const int64_t w = w0 + s;
+                            gg[s] = __ldcg(reinterpret_cast<const float4*>(A.g + w * A.ld_g + i0));
+                            uu[s] = __ldcg(reinterpret_cast<const float4*>(A.u + w * A.ld + i0));
+                            vv[s] = __ldcg(reinterpret_cast<const float4*>(A.v + w * A.ld + i0));
+                        }
                     }
                 }
                 const uint32_t pend = pending_bits4(A.pending, i0);   // after the wide loads are on their way

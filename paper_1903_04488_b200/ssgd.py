@@ -18,6 +18,7 @@ OK, EINVAL, EALIGN, ENOTBOUND, EWORKSPACE, ECUDA, EDEVICE, ENOMEM, ETOOBIG, EPEN
 STATIC_MAX_NCAND = 262144
 INSERT_AUTO, INSERT_GLOBAL, INSERT_SMEM, INSERT_TMA = 0, 1, 2, 3
 PRUNE_AUTO, PRUNE_OFF, PRUNE_ON, PRUNE_EARLY_EXIT, PRUNE_FUSED = 0, 1, 2, 3, 4
+STREAM_AUTO, STREAM_EVICT_FIRST, STREAM_L2_ONLY = 0, 1, 2
 ZERO_DEFERRED, ZERO_EAGER = 0, 1
 SCHED_AUTO, SCHED_COORDINATE_MAJOR, SCHED_WORKER_MAJOR = 0, 1, 2
 FMT_F16, FMT_BF16 = 0, 1
@@ -34,6 +35,7 @@ SIGNATURES = {
     "ssgd_set_prune_mode": [_vp, _i32],
     "ssgd_set_accumulate_schedule": [_vp, _i32],
     "ssgd_set_insert_split": [_vp, _i64],
+    "ssgd_set_stream_loads": [_vp, _i32],
     "ssgd_set_prune_sample_rank": [_vp, _i64],
     "ssgd_set_table_persistence": [_vp, _i32],
     "ssgd_step_used_fallback": [_vp, _vp, C.POINTER(_i32)],
@@ -170,6 +172,9 @@ class Ssgd:
 
     def set_prune_sample_rank(self, rank: int) -> None:
         self._chk(self._lib.ssgd_set_prune_sample_rank(self._h, rank), "ssgd_set_prune_sample_rank")
+
+    def set_stream_loads(self, mode: int) -> None:
+        self._chk(self._lib.ssgd_set_stream_loads(self._h, mode), "ssgd_set_stream_loads")
 
     def set_insert_split(self, nbytes: int) -> None:
         self._chk(self._lib.ssgd_set_insert_split(self._h, nbytes), "ssgd_set_insert_split")
