@@ -49,7 +49,7 @@ COLD_SETS = 8                      # independent (g, u, v, workspace) sets rotat
 # dram__bytes_write.sum on a small case, scaled in proportion to W*d), keyed by kernel: bytes per worker-coordinate
 NCU_TRAFFIC_BYTES_PER_UNIT = {
     "k_accum_insert": 1906.1e6 / (16 * 6_000_002),       # profiles/k_accum_insert_C2_d6M.md
-    "k_accum_insert_tma": 5.09581e9 / (256 * 1_000_002),  # profiles/k_accum_insert_tma_C5_W256_d1M.md
+    "k_accum_insert_tma": 5.11767e9 / (256 * 1_000_002),  # profiles/k_accum_insert_tma_C5_W256_d1M.md
 }
 
 
@@ -296,7 +296,7 @@ def step_bytes(cfg) -> float:
 
 
 def dominant_kernel(cfg) -> str:
-    return "k_accum_insert_tma" if cfg.W >= 64 else "k_accum_insert"
+    return "k_accum_insert_tma" if cfg.W >= (176 if cfg.r * cfg.c * 4 < (16 << 20) else 64) else "k_accum_insert"
 
 
 # ---------------------------------------------------------------------------------------------------

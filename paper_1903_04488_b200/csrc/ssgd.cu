@@ -349,8 +349,13 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     if (x->insert_mode == SSGD_INSERT_TMA) return INS_MERGED_TMA;
     // measured on B200 at d = 11,173,962 (plain loads / bulk-copy pipeline, TB/s): W = 32 6.06 / 5.58; 48 5.97 / 5.83;
     // 64 5.88 / 5.91; 96 5.82 / 6.01; 128 5.75 / 6.06; 256 5.42 / 6.13 -- the plain kernel's threads loop over the
-    // workers 16 at a time, and loop less well than they start
-    return x->W >= 64 ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
+    // workers 16 at a time, and loop less well than they start.  Those figures are for evict-first loads in the plain
+    // kernel, which it uses for tables of 16 MiB and more; below that it reads with .cg and holds out longer (ms per
+    // step, plain / bulk-copy): W = 64 2.49 / 2.63; 96 3.70 / 3.86; 128 4.94 / 5.03; 160 6.20 / 6.23; 192 7.51 / 7.41;
+    // 256 10.05 / 9.80
+    const bool plain_reads_cg = x->stream_loads == SSGD_STREAM_L2_ONLY ||
+                                (x->stream_loads == SSGD_STREAM_AUTO && table_bytes < STREAM_CS_MIN_TABLE_BYTES);
+    return x->W >= (plain_reads_cg ? 176 : 64) ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
 }  // namespace
