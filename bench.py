@@ -296,7 +296,7 @@ def step_bytes(cfg) -> float:
 
 
 def dominant_kernel(cfg) -> str:
-    return "k_accum_insert_tma" if cfg.W >= (176 if cfg.r * cfg.c * 4 < (16 << 20) else 64) else "k_accum_insert"
+    return "k_accum_insert_tma" if cfg.W >= 144 else "k_accum_insert"
 
 
 # ---------------------------------------------------------------------------------------------------

@@ -61,8 +61,7 @@ extern "C" {
 #define SSGD_MAX_R 15
 
 /* Insert variants of ssgd_step (ssgd_set_insert_mode) */
-#define SSGD_INSERT_AUTO   0  /* SSGD_INSERT_TMA when W >= 176 (W >= 64 for tables of 16 MiB and more), else
-                               * SSGD_INSERT_GLOBAL (measured)                                           */
+#define SSGD_INSERT_AUTO   0  /* SSGD_INSERT_TMA when W >= 144, else SSGD_INSERT_GLOBAL (measured)           */
 #define SSGD_INSERT_GLOBAL 1  /* plain 128-bit loads; reductions straight into the L2-resident table    */
 #define SSGD_INSERT_SMEM   2  /* per-block table in shared memory, flushed once; needs r*c*4 <= 200 KiB */
 #define SSGD_INSERT_TMA    3  /* bulk-copy (TMA) + mbarrier pipeline; reductions into the L2 table      */
@@ -136,12 +135,12 @@ int ssgd_test_withhold_block(ssgd_ctx* ctx, int32_t block_plus_one);
 int ssgd_flush(ssgd_ctx* ctx, void* stream);
 /* For tables too large to stay in L2 next to the streamed g, u, v: let the streaming kernel insert only as
  * many rows as fit in `bytes` and insert the remaining rows from the per-coordinate sums in follow-up
- * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 40 MiB,
+ * launches of at most `bytes` of table each (plain-load insert variant only; 0 = never split; default 24 MiB,
  * which leaves tables up to that size untouched). */
 int ssgd_set_insert_split(ssgd_ctx* ctx, int64_t bytes);
-/* Cache operator of the plain-load accumulate+insert kernel's reads of g, u, v (ssgd_step with SSGD_INSERT_GLOBAL).  AUTO:
- * evict-first (ld.global.cs) when the sketch table has 16 MiB or more and W >= 8 (the stream then leaves the table's lines
- * in L2 alone), else L2_ONLY (ld.global.cg: not kept in L1, normal priority in L2).  The result of a step does
+/* Cache operator of the plain-load accumulate+insert kernel's reads of g, u, v (ssgd_step with
+ * SSGD_INSERT_GLOBAL).  AUTO = L2_ONLY (ld.global.cg: not kept in L1, normal priority in L2; the table's lines are
+ * protected by the evict-last policy of the reductions).  EVICT_FIRST: ld.global.cs.  The result of a step does
  * not depend on it. */
 #define SSGD_STREAM_AUTO        0
 #define SSGD_STREAM_EVICT_FIRST 1

@@ -41,8 +41,7 @@ struct AccumArgs {
     HashParams hp; Bucketizer bk;
     // plain-load merged mode only: insert rows [0, rows_here) in this kernel (k_insert_rows does the others)
     int32_t rows_here;
-    // plain-load kernel: 1 = read g, u, v with the evict-first operator (.cs), 0 = cached in L2 only (.cg); see
-    // STREAM_CS_MIN_TABLE_BYTES
+    // plain-load kernel: 1 = read g, u, v with the evict-first operator (.cs), 0 = cached in L2 only (.cg)
     int32_t loads_evict_first;
     // merged modes: if not NULL, the per-coordinate sum over workers of the new v (fp64 accumulation in worker
     // order, rounded once) is also written to xsum[d]: the second round's exact sums, and k_insert_rows' input
@@ -93,6 +92,15 @@ __device__ __forceinline__ void drop_pending(uint32_t bits, float4& u4, float4& 
 
 __device__ __forceinline__ void red_add(float* addr, float x) {
     asm volatile("red.global.add.f32 [%0], %1;" ::"l"(addr), "f"(x) : "memory");
+}
+// The same with an L2 eviction policy for the line it touches (table_policy: the table's lines are the last to go)
+__device__ __forceinline__ void red_add_hint(float* addr, float x, uint64_t policy) {
+    asm volatile("red.global.add.L2::cache_hint.f32 [%0], %1, %2;" ::"l"(addr), "f"(x), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t table_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -188,6 +196,7 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
         }
     } else {
         // ---------------- consumer warps ----------------
+        const uint64_t tpol = table_policy();
         uint32_t n = 0;
         bool ok = true;
         for (int64_t tile = blockIdx.x; tile < ntiles && ok; tile += gridDim.x) {
@@ -241,7 +250,7 @@ k_accum_insert_tma(const AccumArgs A, int32_t* __restrict__ errflag) {
                     row_hashes<POW2, 4>(A.hp.row[j], A.bk, (uint32_t)i0, hb);
 #pragma unroll
                     for (int e = 0; e < 4; ++e)
-                        if (x[e] != 0.0f) red_add(A.table + (int64_t)j * A.c + (hb[e] & P31), apply_sign(x[e], hb[e]));
+                        if (x[e] != 0.0f) red_add_hint(A.table + (int64_t)j * A.c + (hb[e] & P31), apply_sign(x[e], hb[e]), tpol);
                 }
             }
         }

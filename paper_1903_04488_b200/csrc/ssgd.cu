@@ -350,12 +350,10 @@ int resolve_insert_mode(const ssgd_ctx* x) {
     // measured on B200 at d = 11,173,962 (plain loads / bulk-copy pipeline, TB/s): W = 32 6.06 / 5.58; 48 5.97 / 5.83;
     // 64 5.88 / 5.91; 96 5.82 / 6.01; 128 5.75 / 6.06; 256 5.42 / 6.13 -- the plain kernel's threads loop over the
     // workers 16 at a time, and loop less well than they start.  Those figures are for evict-first loads in the plain
-    // kernel, which it uses for tables of 16 MiB and more; below that it reads with .cg and holds out longer (ms per
-    // step, plain / bulk-copy): W = 64 2.49 / 2.63; 96 3.70 / 3.86; 128 4.94 / 5.03; 160 6.20 / 6.23; 192 7.51 / 7.41;
-    // 256 10.05 / 9.80
-    const bool plain_reads_cg = x->stream_loads == SSGD_STREAM_L2_ONLY ||
-                                (x->stream_loads == SSGD_STREAM_AUTO && table_bytes < STREAM_CS_MIN_TABLE_BYTES);
-    return x->W >= (plain_reads_cg ? 176 : 64) ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
+    // kernel; reading with .cg (its default) it holds out longer (ms per step, plain / bulk-copy): W = 128
+    // 4.88 / 4.91; 160 6.11 / 6.08; 256 9.86 / 9.59
+    const bool plain_reads_cg = x->stream_loads != SSGD_STREAM_EVICT_FIRST;
+    return x->W >= (plain_reads_cg ? 144 : 64) ? INS_MERGED_TMA : INS_MERGED_GLOBAL;
 }
 
 }  // namespace
@@ -630,8 +628,7 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     AccumArgs A;
     A.g = g; A.ld_g = ld_g; A.u = x->u; A.v = x->v; A.ld = x->ld; A.W = x->W; A.d = x->d; A.rho = rho;
     A.table = merged; A.c = x->c; A.hp = x->hp; A.bk = x->bk; A.rows_here = x->r; A.xsum = nullptr;
-    A.loads_evict_first = x->stream_loads == SSGD_STREAM_AUTO ? ((size_t)x->r * (size_t)x->c * 4 >= STREAM_CS_MIN_TABLE_BYTES && x->W >= 8 ? 1 : 0)
-                                                              : (x->stream_loads == SSGD_STREAM_EVICT_FIRST ? 1 : 0);
+    A.loads_evict_first = x->stream_loads == SSGD_STREAM_EVICT_FIRST ? 1 : 0;
     A.pending = pending_map(x);      // the previous step's deferred zero-out, applied while u and v stream past
     A.wait_ns = x->wait_ns; A.withhold = x->withhold;
     // a table that cannot stay in L2 next to the stream is inserted a slice of rows at a time

@@ -14,16 +14,20 @@
 
 namespace ssgd {
 
+// Every reduction into the merged table carries an L2 evict-last policy (red_add_hint): the table's lines then
+// outlive the stream that passes through L2 beside them.  Measured on B200 with it / without (whole step, ms; the
+// streamed loads as they were best in each case): 20 MB table, W = 32 2.166 / 2.238; 80 MB 7.11 / 7.24; 5 MB
+// W = 256 (bulk-copy kernel) 9.59 / 9.80, W = 32 1.287 / 1.294, W = 16 0.749 / 0.751.
+//
 // Table bytes one insert kernel may scatter into; larger tables are inserted in row slices.  Measured on B200
-// (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each): 1 row per kernel 6.43 ms, 2 rows 6.25, 3 rows 6.60,
-// 4 rows 6.89, all 5 rows in one kernel 7.80.
-constexpr size_t SPLIT_BYTES_DEFAULT = (size_t)40 << 20;
-// The plain-load kernel reads g, u, v with the evict-first operator (ld.global.cs) when the table it scatters into
-// is at least this large and W >= 8 (the stream then leaves the table's lines alone), else cached in L2 with the normal
-// priority (ld.global.cg).  Measured on B200, whole step in ms with .cs / .cg: 5 MB table W = 32 1.350 / 1.293,
-// W = 16 0.768 / 0.753, W = 8 0.574 / 0.571; 3.6 MB (W = 4, d = 7.3e7) 2.720 / 2.707; 20 MB W = 32 2.264 / 2.315,
-// (W = 4, d = 9e7) 3.459 / 3.444; 80 MB in row slices 7.238 / 7.590.
-constexpr size_t STREAM_CS_MIN_TABLE_BYTES = (size_t)16 << 20;
+// (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each; whole step, ms): 1 row per kernel 7.11, 2 rows 7.27,
+// 3 rows 7.52, 4 rows 8.20, all 5 rows in one kernel 9.20.
+constexpr size_t SPLIT_BYTES_DEFAULT = (size_t)24 << 20;
+// The plain-load kernel reads g, u, v cached in L2 only (ld.global.cg); the evict-first operator (ld.global.cs)
+// can be chosen instead (ssgd_set_stream_loads).  Measured on B200, whole step in ms with .cs / .cg: 5 MB table
+// W = 32 1.349 / 1.287, W = 16 0.768 / 0.749, W = 8 0.573 / 0.571; 3.6 MB (W = 4, d = 7.3e7) 2.709 / 2.715; 20 MB
+// W = 32 2.235 / 2.166, (W = 4, d = 9e7) 3.449 / 3.442; 80 MB, one row per kernel 7.25 / 7.11.  (Before the
+// reductions carried their evict-last policy, .cs was the better choice for tables of 20 MB and more.)
 // Blocks per SM of the two unsketch kernels: one resident wave.  Measured on B200 (C2): the dense kernel
 // takes 0.222 ms with 4 or 6 blocks per SM in the grid and 0.246 ms with 8 (6 fit: the last third of a
 // second wave runs alone); the early-exit kernel 0.205-0.210 ms with 2 or 4, 0.232 ms with 16.
@@ -65,6 +69,7 @@ k_accum_insert(const AccumArgs A) {
     }
     const int64_t groups = (A.d + 3) >> 2;
     const int64_t stride = (int64_t)gridDim.x * K1_THREADS;
+    const uint64_t tpol = table_policy();
     for (int64_t q = (int64_t)blockIdx.x * K1_THREADS + threadIdx.x; q < groups; q += stride) {
         const int64_t i0 = q << 2;
         uint32_t hb[R][4];
@@ -174,7 +179,7 @@ k_accum_insert(const AccumArgs A) {
                     if (i0 + e < A.d && x[e] != 0.0f) {
                         const float sx = apply_sign(x[e], h1[e]);
                         if (MODE == INS_MERGED_SMEM) atomicAdd(&s_table[(int64_t)j * A.c + (h1[e] & P31)], sx);
-                        else red_add(A.table + (int64_t)j * A.c + (h1[e] & P31), sx);
+                        else red_add_hint(A.table + (int64_t)j * A.c + (h1[e] & P31), sx, tpol);
                     }
                 }
             }
@@ -202,6 +207,7 @@ k_insert_rows(const float* __restrict__ xsum, int64_t d, float* __restrict__ tab
     pdl_wait();
     const int64_t groups = (d + 3) >> 2;
     const int64_t stride = (int64_t)gridDim.x * 256;
+    const uint64_t tpol = table_policy();
     for (int64_t q = (int64_t)blockIdx.x * 256 + threadIdx.x; q < groups; q += stride) {
         const int64_t i0 = q << 2;
         float x[4] = {0.f, 0.f, 0.f, 0.f};
@@ -218,7 +224,7 @@ k_insert_rows(const float* __restrict__ xsum, int64_t d, float* __restrict__ tab
             row_hashes<POW2, 4>(hp.row[j], bk, (uint32_t)i0, hb);
 #pragma unroll
             for (int e = 0; e < 4; ++e)
-                if (i0 + e < d && x[e] != 0.0f) red_add(table + (int64_t)j * c + (hb[e] & P31), apply_sign(x[e], hb[e]));
+                if (i0 + e < d && x[e] != 0.0f) red_add_hint(table + (int64_t)j * c + (hb[e] & P31), apply_sign(x[e], hb[e]), tpol);
         }
     }
 }
