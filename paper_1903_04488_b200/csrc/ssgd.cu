@@ -639,9 +639,12 @@ int ssgd_step(ssgd_ctx* x, const float* g, int64_t ld_g, float rho, int64_t ncan
     if (split) A.rows_here = rows_fit;
     if ((e = mark(x, 0, st))) return e;
     if ((e = mode == INS_MERGED_TMA ? launch_accum_tma(x, A, st) : launch_accum(x, A, mode, st))) return e;
-    if (split)
-        for (int lo = rows_fit; lo < x->r; lo += rows_fit)
-            if ((e = launch_insert_rows(x, A.xsum, merged, lo, lo + rows_fit < x->r ? lo + rows_fit : x->r, st))) return e;
+    if (split) {
+        // the follow-up passes have only the per-coordinate sums streaming beside the table: more rows per pass
+        const int pass_rows = (int)(INSERT_PASS_BYTES / row_bytes) > rows_fit ? (int)(INSERT_PASS_BYTES / row_bytes) : rows_fit;
+        for (int lo = rows_fit; lo < x->r; lo += pass_rows)
+            if ((e = launch_insert_rows(x, A.xsum, merged, lo, lo + pass_rows < x->r ? lo + pass_rows : x->r, st))) return e;
+    }
     if ((e = mark(x, 1, st))) return e;
     int32_t* cand = reinterpret_cast<int32_t*>(x->ws + x->off_cand);
     float* est = reinterpret_cast<float*>(x->ws + x->off_est);

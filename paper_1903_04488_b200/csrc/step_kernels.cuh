@@ -23,6 +23,11 @@ namespace ssgd {
 // (C4: d = 9e7, W = 16, 5 rows of 4,194,304 = 16 MiB each; whole step, ms): 1 row per kernel 7.11, 2 rows 7.27,
 // 3 rows 7.52, 4 rows 8.20, all 5 rows in one kernel 9.20.
 constexpr size_t SPLIT_BYTES_DEFAULT = (size_t)24 << 20;
+// Table bytes one k_insert_rows pass scatters into: beside it only the per-coordinate sums stream through L2.
+// Measured at C4 (whole step, ms; one row in the streaming kernel): passes of 1 row 7.11, 2 rows 7.04, 3 + 1 rows
+// 7.02, all 4 remaining rows in one pass 6.93; no row in the streaming kernel and all 5 in one pass 7.32; 2 rows in
+// the streaming kernel and 3 in one pass 7.21.
+constexpr size_t INSERT_PASS_BYTES = (size_t)64 << 20;
 // The plain-load kernel reads g, u, v cached in L2 only (ld.global.cg); the evict-first operator (ld.global.cs)
 // can be chosen instead (ssgd_set_stream_loads).  Measured on B200, whole step in ms with .cs / .cg: 5 MB table
 // W = 32 1.349 / 1.287, W = 16 0.768 / 0.749, W = 8 0.573 / 0.571; 3.6 MB (W = 4, d = 7.3e7) 2.709 / 2.715; 20 MB
